@@ -1,0 +1,521 @@
+"""Pins of the CPU oracle against what the paper and the mathematics fix (no GPU needed).
+
+Each test is chosen so that a plausible mistake in the oracle (a dropped term, a wrong sign or index,
+a transposed operand, an off-by-one in the window or in the schedule) fails at least one of them.
+"""
+import math
+import os
+import subprocess
+import sys
+
+import numpy as np
+import pytest
+from scipy.special import expit, log_expit
+
+import oracle
+from oracle import Oracle, StalenessBook
+from paper_2211_10280_b200 import synth
+
+LN2 = math.log(2.0)
+
+
+# ------------------------------------------------------------------ Philox
+def test_philox_known_answers(golden_dir):
+    n = 0
+    for line in open(golden_dir / "philox4x32_10_kat.txt"):
+        if line.startswith("#") or not line.strip():
+            continue
+        w = [int(x, 16) for x in line.split()]
+        assert oracle.philox4x32_10(w[:4], w[4:6]) == w[6:]
+        n += 1
+    assert n == 3
+
+
+def test_philox_counter_words_are_not_interchangeable():
+    # every counter and key word matters, and in its own position
+    base = oracle.philox4x32_10([1, 2, 3, 4], [5, 6])
+    seen = {tuple(base)}
+    for pos in range(4):
+        c = [1, 2, 3, 4]
+        c[pos] ^= 1
+        seen.add(tuple(oracle.philox4x32_10(c, [5, 6])))
+    seen.add(tuple(oracle.philox4x32_10([2, 1, 3, 4], [5, 6])))
+    seen.add(tuple(oracle.philox4x32_10([1, 2, 3, 4], [6, 5])))
+    assert len(seen) == 7
+
+
+# ------------------------------------------------------------------ alias table
+def _alias_mass(thresh, alias):
+    """Probability mass of every outcome, in units of 2^-32 / V, as exact Python integers."""
+    V = thresh.size
+    mass = [0] * V
+    for i in range(V):
+        t = int(thresh[i])
+        if t == 0xFFFFFFFF:
+            mass[i] += 1 << 32
+        else:
+            mass[i] += t
+            mass[int(alias[i])] += (1 << 32) - t
+    return mass
+
+
+@pytest.mark.parametrize("V,seed", [(7, 0), (100, 1), (5000, 2)])
+def test_alias_reconstructs_count_pow_075(V, seed):
+    rng = np.random.default_rng(seed)
+    counts = (rng.zipf(1.3, V).astype(np.uint64) % 100000) + 1
+    thresh, alias = oracle.build_alias(counts)
+    mass = _alias_mass(thresh, alias)
+    assert sum(mass) == V << 32
+    w = counts.astype(np.float64) ** 0.75
+    want = w * V / w.sum() * 2.0 ** 32
+    # floor() quantisation loses < 1 unit per small entry; an outcome collects at most V of them
+    assert np.max(np.abs(np.array(mass, dtype=np.float64) - want)) <= V + 1e-6 * want.max()
+    assert np.all(alias < V)
+
+
+def test_alias_equal_counts_accept_always():
+    thresh, alias = oracle.build_alias(np.full(64, 9, dtype=np.uint64))
+    assert np.all(thresh == 0xFFFFFFFF)
+    assert np.array_equal(alias, np.arange(64, dtype=np.uint32))
+
+
+def test_alias_two_outcomes_by_hand():
+    # counts 1 and 16 -> weights 1 and 8 -> scaled p = 2/9 and 16/9: slot 0 keeps 2/9, rest goes to 1
+    thresh, alias = oracle.build_alias(np.array([1, 16], dtype=np.uint64))
+    assert int(thresh[0]) == (2 << 32) // 9 and int(alias[0]) == 1
+    assert int(thresh[1]) == 0xFFFFFFFF
+
+
+def test_draws_follow_unigram_pow_075_chi_square():
+    V, k = 50, 8
+    counts = (np.arange(V, dtype=np.uint64)[::-1] + 1) ** 2
+    o = Oracle(V=V, d=2, window=2, k=k, batch=256, counts=counts, seed=11)
+    hist = np.zeros(V)
+    rng = np.random.default_rng(0)
+    for b in range(40):
+        rc, _, _ = o.train_batch(0, rng.integers(0, V, 256), b)
+        assert rc == 0
+        hist += np.bincount(o.read_negatives().ravel(), minlength=V)
+    p = counts.astype(np.float64) ** 0.75
+    p /= p.sum()
+    n = hist.sum()
+    chi2 = float(((hist - n * p) ** 2 / (n * p)).sum())
+    # 49 degrees of freedom: mean 49, sd ~9.9; 120 is beyond 7 sigma
+    assert n == 40 * synth.n_pairs(256, 2) * k
+    assert chi2 < 120.0, chi2
+
+
+def test_negative_draw_uses_both_halves_of_a_philox_call():
+    counts = np.arange(1, 1001, dtype=np.uint64)
+    thresh, alias = oracle.build_alias(counts)
+    seed, rep, b, p = 0x1234567890ABCDEF, 3, 77, 41
+    for j in range(6):
+        out = oracle.philox4x32_10([p, j >> 1, b, (1 << 24) | rep], [seed & 0xFFFFFFFF, seed >> 32])
+        ra, rb = (out[2], out[3]) if j & 1 else (out[0], out[1])
+        slot = (ra * 1000) >> 32
+        want = slot if (thresh[slot] == 0xFFFFFFFF or rb < thresh[slot]) else int(alias[slot])
+        assert oracle.negative(seed, rep, b, p, j, thresh, alias) == want
+
+
+# ------------------------------------------------------------------ pairs
+def _pairs_brute(tokens, w):
+    n = len(tokens)
+    return [(q, c) for q in range(n) for c in range(q - w, q + w + 1) if 0 <= c < n and c != q]
+
+
+@pytest.mark.parametrize("n,w", [(0, 2), (1, 2), (2, 5), (3, 1), (5, 5), (6, 5), (7, 3), (11, 5), (12, 5), (40, 5)])
+def test_pair_count_matches_enumeration(n, w):
+    V = 50
+    o = Oracle(V=V, d=2, window=w, k=2, batch=max(n, 1))
+    toks = np.arange(n, dtype=np.int32) % V
+    rc, loss, nrows = o.train_batch(0, toks, 0)
+    assert rc == 0
+    brute = _pairs_brute(toks, w)
+    assert o.last_pairs() == len(brute) == synth.n_pairs(n, w)
+    if n > w:
+        assert len(brute) == 2 * w * n - w * (w + 1)
+    if n < 2:
+        assert nrows == 0 and loss == 0.0
+
+
+# ------------------------------------------------------------------ gradient: closed forms
+def _dense_reference(o, tokens, w, k, V, d, lr, neg, t_in, t_out):
+    """Dense fp64 evaluation of one batch from the per-pair closed form; returns loss, new tables, touched ids."""
+    g_in = np.zeros((V, d))
+    g_out = np.zeros((V, d))
+    touched = set()
+    loss = 0.0
+    for p, (q, c) in enumerate(_pairs_brute(tokens, w)):
+        vc = t_in[tokens[q]].astype(np.float64)
+        ctx = int(tokens[c])
+        uo = t_out[ctx].astype(np.float64)
+        s0 = expit(uo @ vc)
+        loss -= log_expit(uo @ vc)
+        g_in[tokens[q]] += (s0 - 1.0) * uo          # dL/dv_c, positive term
+        g_out[ctx] += (s0 - 1.0) * vc               # dL/du_o
+        touched.update([int(tokens[q]), V + ctx])
+        for j in range(k):
+            r = int(neg[p, j])
+            if r == ctx:
+                continue
+            un = t_out[r].astype(np.float64)
+            sj = expit(un @ vc)
+            loss -= log_expit(-(un @ vc))
+            g_in[tokens[q]] += sj * un              # dL/dv_c, negative terms
+            g_out[r] += sj * vc                     # dL/du_n
+            touched.add(V + r)
+    return loss, g_in, g_out, sorted(touched)
+
+
+def test_single_batch_matches_per_pair_closed_form():
+    V, d, w, k, n, lr = 12, 3, 2, 4, 9, 0.05
+    t_in, t_out = synth.random_tables(V, d, seed=5, scale=1.0)
+    o = Oracle(V=V, d=d, window=w, k=k, batch=n, lr=lr, seed=3, init_in=t_in, init_out=t_out,
+               counts=np.arange(1, V + 1, dtype=np.uint64))
+    toks = np.array([3, 3, 7, 0, 11, 3, 5, 5, 1], dtype=np.int32)
+    rc, loss, nrows = o.train_batch(0, toks, 4)
+    assert rc == 0
+    neg = o.read_negatives()
+    want_loss, g_in, g_out, touched = _dense_reference(o, toks, w, k, V, d, lr, neg, t_in, t_out)
+    ids, delta = o.read_message(0, 4)
+    assert ids.tolist() == touched and nrows == len(touched)
+    assert loss == pytest.approx(want_loss, rel=1e-12)
+    lr32 = float(np.float32(lr))
+    dense = np.concatenate([g_in, g_out])
+    np.testing.assert_allclose(delta, (-lr32 * dense[ids]).astype(np.float32), rtol=2e-7, atol=1e-12)
+    new_in, new_out = o.read_embeddings(0, 0), o.read_embeddings(0, 1)
+    np.testing.assert_allclose(new_in, t_in - lr32 * g_in, rtol=3e-7, atol=1e-9)
+    np.testing.assert_allclose(new_out, t_out - lr32 * g_out, rtol=3e-7, atol=1e-9)
+
+
+def test_two_tokens_one_negative_by_hand():
+    # tokens [a, b], window 1: pairs (a<-b) and (b<-a).  All output rows zero except the ones set here.
+    V, d = 4, 2
+    t_in = np.zeros((V, d), np.float32)
+    t_out = np.zeros((V, d), np.float32)
+    t_in[0] = [1.0, 2.0]
+    t_in[1] = [-1.0, 0.5]
+    t_out[1] = [0.5, -0.25]      # u_b . v_a = 0  -> sigma = 1/2 exactly
+    t_out[0] = [2.0, 4.0]        # u_a . v_b = 0  -> sigma = 1/2 exactly
+    o = Oracle(V=V, d=d, window=1, k=1, batch=2, lr=0.5, seed=9, init_in=t_in, init_out=t_out)
+    rc, loss, _ = o.train_batch(0, np.array([0, 1], np.int32), 0)
+    assert rc == 0
+    neg = o.read_negatives()
+    g = o.read_g()
+    # positives: sigma(0) - 1 = -1/2
+    assert g[0, 0] == -0.5 and g[1, 0] == -0.5
+    want_in = t_in.astype(np.float64).copy()
+    want_out = t_out.astype(np.float64).copy()
+    terms = 2
+    for p, (c, ctx) in enumerate([(0, 1), (1, 0)]):
+        want_in[c] -= 0.5 * (-0.5) * t_out[ctx]
+        want_out[ctx] -= 0.5 * (-0.5) * t_in[c]
+        r = int(neg[p, 0])
+        if r != ctx:
+            x = float(t_out[r].astype(np.float64) @ t_in[c].astype(np.float64))
+            s = 1.0 / (1.0 + math.exp(-x))
+            assert g[p, 1] == pytest.approx(s, rel=1e-7)
+            want_in[c] -= 0.5 * s * t_out[r]
+            want_out[r] -= 0.5 * s * t_in[c]
+            terms += 1 if x == 0.0 else 0
+        else:
+            assert g[p, 1] == 0.0
+    np.testing.assert_allclose(o.read_embeddings(0, 0), want_in, rtol=1e-6, atol=1e-7)
+    np.testing.assert_allclose(o.read_embeddings(0, 1), want_out, rtol=1e-6, atol=1e-7)
+    assert loss >= 2 * LN2
+
+
+@pytest.mark.parametrize("wl", [synth.scaled(synth.TINY, batches=1),
+                                synth.scaled(synth.MID, V=20000, batch=1024, batches=1)])
+def test_first_batch_closed_form(wl):
+    """With zero output rows every dot product is 0 and every sigmoid is 1/2."""
+    toks = synth.token_stream(wl, 0)[0]
+    counts = synth.stream_counts([toks], wl.V)
+    t_in, _ = synth.init_tables(wl.V, wl.d, 123)
+    o = Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, lr=wl.lr, seed=wl.seed,
+               counts=counts, init_in=t_in)
+    rc, loss, nrows = o.train_batch(0, toks, 0)
+    assert rc == 0
+    neg = o.read_negatives()
+    pairs = np.array(_pairs_brute(toks, wl.window))
+    assert len(pairs) == wl.pairs_per_batch
+    centre, ctx = toks[pairs[:, 0]], toks[pairs[:, 1]]
+    live = neg != ctx[:, None].astype(np.uint32)
+    assert loss == pytest.approx((len(pairs) + int(live.sum())) * LN2, rel=1e-12)
+    # input table bit-unchanged (all deltas are -lr * 0)
+    assert np.array_equal(o.read_embeddings(0, 0).view(np.uint32), t_in.view(np.uint32))
+    lr32 = float(np.float32(wl.lr))
+    want = np.zeros((wl.V, wl.d))
+    np.add.at(want, ctx, 0.5 * lr32 * t_in[centre].astype(np.float64))
+    for j in range(wl.k):
+        m = live[:, j]
+        np.add.at(want, neg[m, j], -0.5 * lr32 * t_in[centre[m]].astype(np.float64))
+    got = o.read_embeddings(0, 1)
+    np.testing.assert_allclose(got, want, rtol=2e-7, atol=1e-12)
+    touched_out = set(ctx.tolist()) | set(neg[live].tolist())
+    ids, _ = o.read_message(0, 0)
+    assert ids.tolist() == sorted(set(centre.tolist())) + [wl.V + r for r in sorted(touched_out)]
+    assert nrows == ids.size
+
+
+def test_gradient_matches_central_finite_differences():
+    V, d, w, k, n, lr = 8, 4, 2, 3, 6, 0.25
+    rng = np.random.default_rng(42)
+    # entries on a 2^-10 grid so that +-h is exact in fp32
+    t_in = (rng.integers(-1024, 1024, (V, d)) / 1024.0).astype(np.float32)
+    t_out = (rng.integers(-1024, 1024, (V, d)) / 1024.0).astype(np.float32)
+    toks = np.array([1, 5, 1, 0, 7, 2], dtype=np.int32)
+    o = Oracle(V=V, d=d, window=w, k=k, batch=n, lr=lr, seed=77, init_in=t_in, init_out=t_out)
+    h = 2.0 ** -9
+    fd = np.zeros((2, V, d))
+    for which, tab in ((0, t_in), (1, t_out)):
+        for r in range(V):
+            for e in range(d):
+                row = tab[r:r + 1].copy()
+                row[0, e] = tab[r, e] + np.float32(h)
+                o.write_embeddings(0, which, r, row)
+                lp = o.batch_loss(0, toks, 3)
+                row[0, e] = tab[r, e] - np.float32(h)
+                o.write_embeddings(0, which, r, row)
+                lm = o.batch_loss(0, toks, 3)
+                o.write_embeddings(0, which, r, tab[r:r + 1])
+                fd[which, r, e] = (lp - lm) / (2 * h)
+    rc, loss, _ = o.train_batch(0, toks, 3)
+    assert rc == 0
+    ids, delta = o.read_message(0, 3)
+    grad = np.zeros((2 * V, d))
+    grad[ids] = -delta.astype(np.float64) / lr
+    fd = fd.reshape(2 * V, d)
+    assert np.max(np.abs(fd)) > 0.1
+    np.testing.assert_allclose(grad, fd, rtol=0, atol=2e-5)
+    # rows outside the message have zero finite difference too
+    mask = np.ones(2 * V, bool)
+    mask[ids] = False
+    assert np.all(fd[mask] == 0.0)
+
+
+# ------------------------------------------------------------------ message invariants
+def test_message_covers_exactly_touched_rows_and_rest_is_bit_unchanged():
+    wl = synth.scaled(synth.TINY, V=3000, batches=3)
+    stream = synth.token_stream(wl, 0)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 8, scale=0.3)
+    o = Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, lr=wl.lr, seed=5,
+               counts=synth.stream_counts([stream], wl.V), init_in=t_in, init_out=t_out)
+    for b in range(3):
+        before_in, before_out = o.read_embeddings(0, 0), o.read_embeddings(0, 1)
+        rc, _, nrows = o.train_batch(0, stream[b], b)
+        assert rc == 0
+        neg = o.read_negatives()
+        pairs = np.array(_pairs_brute(stream[b], wl.window))
+        ctx = stream[b][pairs[:, 1]]
+        live = neg != ctx[:, None].astype(np.uint32)
+        want = sorted(set(stream[b].tolist())) + [wl.V + r for r in sorted(set(ctx.tolist()) | set(neg[live].tolist()))]
+        ids, delta = o.read_message(0, b)
+        assert ids.tolist() == want and np.all(np.diff(ids.astype(np.int64)) > 0)
+        after = np.concatenate([o.read_embeddings(0, 0), o.read_embeddings(0, 1)])
+        before = np.concatenate([before_in, before_out])
+        untouched = np.ones(2 * wl.V, bool)
+        untouched[ids] = False
+        assert np.array_equal(after[untouched].view(np.uint32), before[untouched].view(np.uint32))
+        assert np.array_equal(after[ids], before[ids] + delta)   # one fp32 addition per element
+
+
+def test_masked_negative_contributes_nothing():
+    # V = 2 with a huge count on token 1: nearly every draw for a pair whose context is 1 is masked
+    V, d = 2, 2
+    t_in = np.array([[0.5, -1.0], [0.25, 0.75]], np.float32)
+    t_out = np.array([[1.0, 1.0], [-0.5, 2.0]], np.float32)
+    o = Oracle(V=V, d=d, window=1, k=6, batch=2, lr=0.1, seed=1, init_in=t_in, init_out=t_out,
+               counts=np.array([1, 10 ** 9], np.uint64))
+    rc, loss, _ = o.train_batch(0, np.array([0, 1], np.int32), 0)
+    neg, g = o.read_negatives(), o.read_g()
+    assert np.all(neg[0] == 1)           # pair 0: centre 0, context 1: every draw hits the context
+    assert np.all(g[0, 1:] == 0.0)
+    x = float(t_out[1].astype(np.float64) @ t_in[0].astype(np.float64))
+    # pair 1 (centre 1, context 0) keeps its negatives on row 1
+    y = float(t_out[1].astype(np.float64) @ t_in[1].astype(np.float64))
+    z = float(t_out[0].astype(np.float64) @ t_in[1].astype(np.float64))
+    n1 = int(np.sum(neg[1] == 1))
+    want = -log_expit(x) - log_expit(z) - n1 * log_expit(-y)
+    assert loss == pytest.approx(want, rel=1e-12)
+
+
+def test_bad_token_changes_nothing():
+    o = Oracle(V=10, d=2, window=1, k=1, batch=4)
+    before = o.read_embeddings(0, 0)
+    rc, _, _ = o.train_batch(0, np.array([1, 10, 2, 3], np.int32), 0)
+    assert rc == -1
+    rc, _, _ = o.train_batch(0, np.array([1, -1, 2, 3], np.int32), 0)
+    assert rc == -1
+    assert np.array_equal(before, o.read_embeddings(0, 0))
+    assert np.all(o.sampler()[2] == 1)
+
+
+def test_seeded_init_is_uniform_in_half_over_d():
+    V, d = 4000, 16
+    t = oracle.init_input_table(99, V, d)
+    assert t.dtype == np.float32 and np.all(np.abs(t) < 0.5 / d)
+    assert abs(float(t.mean())) < 3 * (1.0 / d) / math.sqrt(12 * V * d)
+    assert float(t.std()) == pytest.approx((1.0 / d) / math.sqrt(12), rel=0.02)
+    assert len(np.unique(t)) > 0.99 * V * d
+    o = Oracle(V=V, d=d, window=1, k=1, batch=4, W=2, seed=99)
+    assert np.array_equal(o.read_embeddings(1, 0), t) and not o.read_embeddings(1, 1).any()
+
+
+# ------------------------------------------------------------------ DASGD protocol
+def test_fig2_staleness_values(golden_dir):
+    want = {}
+    for line in open(golden_dir / "fig2_staleness.txt"):
+        if line.startswith("#") or not line.strip():
+            continue
+        ev, model, grad, val = line.split()
+        want[(ev, grad)] = int(val)
+    book = StalenessBook(3)   # models 1, 2, 3 -> indices 0, 1, 2
+    red = book.compute(0)
+    blue = book.compute(1)
+    green = book.compute(2)
+    yellow = book.compute(1)
+    assert want[("local_apply", "blue")] == 0     # local application has staleness 0 by definition
+    assert book.size(1) == want[("size_before_apply", "green")]
+    assert book.apply(1, green) == want[("staleness", "green")]
+    assert book.size(1) == want[("size_before_apply", "red")]
+    assert book.apply(1, red) == want[("staleness", "red")]
+    assert {blue, yellow} == {1, 3}
+
+
+def test_single_replica_is_plain_sgd():
+    wl = synth.scaled(synth.TINY, V=500, batches=4)
+    stream = synth.token_stream(wl, 0)
+    o = Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=1, max_delay=2)
+    for b in range(4):
+        assert o.train_batch(0, stream[b], b)[0] == 0
+        assert o.apply_messages(0, b) == 0 and o.pending(0) == 0
+    assert o.drain() == 0 and o.delivery_log(0).shape[0] == 0
+
+
+def _run_dasgd(W, max_delay, steps, seed=21, V=400, d=8):
+    wl = synth.scaled(synth.TINY, V=V, d=d, batch=64, W=W, batches=steps, stream_seeds=tuple(range(50, 50 + W)),
+                      max_delay=max_delay)
+    streams = synth.all_streams(wl)
+    t_in, t_out = synth.random_tables(V, d, 2, scale=0.2)
+    o = Oracle(V=V, d=d, window=wl.window, k=wl.k, batch=wl.batch, W=W, lr=wl.lr, max_delay=max_delay,
+               seed=seed, counts=synth.stream_counts(streams, V), init_in=t_in, init_out=t_out)
+    msgs = {}
+    for t in range(steps):
+        for i in range(W):
+            assert o.train_batch(i, streams[i][t], t)[0] == 0
+            msgs[(i, t)] = o.read_message(i, t)
+        for j in range(W):
+            o.apply_messages(j, t)
+    return o, msgs, (t_in, t_out)
+
+
+def test_every_message_is_delivered_once_in_order_and_within_the_delay_bound():
+    W, D, T = 4, 2, 12
+    o, msgs, _ = _run_dasgd(W, D, T)
+    delays = set()
+    for j in range(W):
+        log = o.delivery_log(j)
+        prev = None
+        for origin, sender, due, at, _ in log.tolist():
+            assert sender != j and due == at and 0 <= due - origin <= D
+            assert due == origin + o.delay(origin, sender, j)
+            delays.add(due - origin)
+            if prev is not None and prev[0] == at:
+                assert (prev[1], prev[2]) < (origin, sender)    # (origin step, sender) order in a step
+            prev = (at, origin, sender)
+    assert delays == {0, 1, 2}
+    pending = sum(o.pending(j) for j in range(W))
+    assert o.drain() == pending
+    for j in range(W):
+        log = o.delivery_log(j)
+        got = sorted((int(s), int(t)) for t, s, *_ in log.tolist())
+        assert got == sorted((i, t) for i in range(W) if i != j for t in range(T))
+
+
+def test_staleness_log_matches_set_arithmetic():
+    W, D, T = 3, 2, 8
+    o, _, _ = _run_dasgd(W, D, T)
+    o.drain()
+    G = [set() for _ in range(W)]
+    snap = {}
+    inbox = [[] for _ in range(W)]
+    want = [[] for _ in range(W)]
+    for t in range(T):
+        for i in range(W):
+            snap[(i, t)] = set(G[i])
+            G[i].add((i, t))
+            for j in range(W):
+                if j != i:
+                    inbox[j].append((t + o.delay(t, i, j), t, i))
+        for j in range(W):
+            due = sorted([x for x in inbox[j] if x[0] <= t], key=lambda x: (x[1], x[2]))
+            inbox[j] = [x for x in inbox[j] if x[0] > t]
+            for _, ot, s in due:
+                want[j].append(len(snap[(s, ot)] ^ G[j]))
+                G[j].add((s, ot))
+    for j in range(W):
+        for _, ot, s in sorted(inbox[j]):
+            want[j].append(len(snap[(s, ot)] ^ G[j]))
+            G[j].add((s, ot))
+        assert o.delivery_log(j)[:, 4].tolist() == want[j]
+    assert max(max(w) for w in want) > 0
+
+
+def test_replicas_agree_after_drain_and_equal_init_plus_all_messages():
+    W, D, T = 4, 2, 6
+    o, msgs, (t_in, t_out) = _run_dasgd(W, D, T)
+    o.drain()
+    V = o.V
+    total = np.concatenate([t_in, t_out]).astype(np.float64)
+    for (i, t), (ids, delta) in msgs.items():
+        total[ids] += delta
+    ref = np.concatenate([o.read_embeddings(0, 0), o.read_embeddings(0, 1)])
+    np.testing.assert_allclose(ref, total, rtol=0, atol=2e-6)
+    for j in range(1, W):
+        other = np.concatenate([o.read_embeddings(j, 0), o.read_embeddings(j, 1)])
+        np.testing.assert_allclose(other, ref, rtol=0, atol=2e-6)
+    assert not np.array_equal(ref[:V], t_in)
+
+
+def test_zero_delay_keeps_replicas_in_lockstep():
+    # with every delay 0 all replicas hold theta + sum_i delta_i(theta) after each step:
+    # N models with batch b behave like one model with batch N*b
+    W, T = 3, 3
+    o, msgs, (t_in, t_out) = _run_dasgd(W, 0, T)
+    for j in range(W):
+        assert o.pending(j) == 0 and np.all(o.delivery_log(j)[:, 2] == o.delivery_log(j)[:, 0])
+    a = o.read_embeddings(0, 1)
+    for j in range(1, W):
+        np.testing.assert_allclose(o.read_embeddings(j, 1), a, rtol=0, atol=1e-6)
+
+
+def test_loss_starts_at_ln2_per_term_and_decreases():
+    wl = synth.TINY
+    stream = synth.token_stream(wl, 0)
+    o = Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, lr=wl.lr, seed=wl.seed,
+               counts=synth.stream_counts([stream], wl.V))
+    losses = [o.train_batch(0, stream[b], b)[1] for b in range(60)]
+    P = wl.pairs_per_batch
+    assert losses[0] <= P * (1 + wl.k) * LN2 and losses[0] > P * (1 + wl.k) * LN2 * 0.99
+    assert np.mean(losses[-10:]) < 0.95 * losses[0]
+
+
+def test_result_does_not_depend_on_thread_count(tmp_path):
+    code = (
+        "import sys, numpy as np; sys.path.insert(0, %r)\n"
+        "from oracle import Oracle\n"
+        "from paper_2211_10280_b200 import synth\n"
+        "wl = synth.scaled(synth.TINY, V=2000, batches=2)\n"
+        "s = synth.token_stream(wl, 0)\n"
+        "o = Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, seed=3)\n"
+        "l = [o.train_batch(0, s[b], b)[1] for b in range(2)]\n"
+        "np.save(sys.argv[1], np.concatenate([o.read_embeddings(0,0).ravel(), o.read_embeddings(0,1).ravel(), l]))\n"
+    ) % str(os.path.dirname(os.path.dirname(os.path.abspath(__file__))))
+    outs = []
+    for nt in ("1", "4"):
+        f = tmp_path / f"t{nt}.npy"
+        env = dict(os.environ, OMP_NUM_THREADS=nt)
+        subprocess.check_call([sys.executable, "-c", code, str(f)], env=env)
+        outs.append(np.load(f))
+    assert np.array_equal(outs[0].view(np.uint64), outs[1].view(np.uint64))
