@@ -1,0 +1,246 @@
+/*
+ * tensair.h - C ABI of the SGNS / DASGD hot path on one GPU.
+ *
+ * The library trains W logical replicas of a skip-gram negative-sampling (SGNS) word-embedding
+ * model that live in one GPU's memory and exchange sparse gradient messages the way the Model
+ * operator of Algorithm 1 does:
+ *
+ *   tensair_train_batch     train(msg), mini-batch branch of Algorithm 1: gradient calculation at
+ *                           the snapshot theta_t (Eq. 1), local gradient application, then "send":
+ *                           the sparse gradient message is filed for every other replica.
+ *   tensair_apply_messages  train(msg), gradient branch of Algorithm 1: gradient application of the
+ *                           messages another replica sent, in the order Section 3.1 fixes (after
+ *                           the local step, received gradients one by one).
+ *
+ * Conventions for every call
+ *   - Return value: TENSAIR_OK (0) or a negative TENSAIR_E* code; nothing throws or aborts across
+ *     this boundary.  tensair_strerror() names a code, tensair_last_error() gives detail.
+ *   - "device pointer" means memory of the GPU named in tensair_config.device; "host pointer" means
+ *     ordinary process memory (pinned or pageable).
+ *   - All GPU work is enqueued on the stream given at tensair_init, in call order.  Calls are
+ *     asynchronous unless stated; a context must be used from one thread at a time.
+ *   - The library allocates no device memory: tables, message pool and scratch are caller-owned and
+ *     must stay valid until tensair_destroy.
+ *
+ * Layouts
+ *   - Tables: replica r owns 2*V rows of row_stride floats, input (centre-word) rows [0,V) followed
+ *     by output (context-word) rows [V,2V); replicas are consecutive.  Only the first d floats of a
+ *     row are meaningful.  A "row id" in [0,2V) names a row of this unified table.
+ *   - Sparse gradient message (the payload of Algorithm 1's send_gradients; Section 4 notes that a
+ *     word-embedding mini-batch changes few of the model's variables, so only touched rows travel):
+ *     a row count n, n strictly ascending row ids, n delta rows (already scaled by -lr).  Applying
+ *     it is table[id] += delta, one fp32 addition per element.
+ */
+#ifndef TENSAIR_H
+#define TENSAIR_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#if defined(__GNUC__)
+#define TENSAIR_API __attribute__((visibility("default")))
+#else
+#define TENSAIR_API
+#endif
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef struct tensair_ctx tensair_ctx;
+typedef struct tensair_schedule tensair_schedule;
+
+/* How the batch loss L(X, theta) of Eq. 1 combines the per-pair losses (the paper does not say). */
+enum { TENSAIR_SUM = 0, TENSAIR_MEAN = 1 };
+
+enum {
+    TENSAIR_OK = 0,
+    TENSAIR_EINVAL = -1,    /* bad argument or unsupported configuration */
+    TENSAIR_ENOMEM = -2,    /* a caller-provided buffer is too small */
+    TENSAIR_ECUDA = -3,     /* a CUDA call failed; see tensair_last_error */
+    TENSAIR_EBADTOKEN = -4, /* a batch held a token id outside [0,V) */
+    TENSAIR_EPENDING = -5,  /* a message slot still has undelivered recipients */
+    TENSAIR_ENOTFOUND = -6  /* the requested message is no longer held */
+};
+
+/* Model, batch and exchange shape (Algorithm 1's constructor arguments plus the SGNS shape). */
+typedef struct tensair_config {
+    uint32_t V;               /* vocabulary size, 2 <= V <= 2^30 */
+    uint32_t d;               /* embedding dimension, multiple of 4, 4 <= d <= 1024 */
+    uint32_t window;          /* symmetric context window w, 1 <= w <= 16 */
+    uint32_t k;               /* negatives per pair, 1 <= k <= 64 */
+    uint32_t batch;           /* maximum centre tokens per mini-batch */
+    uint32_t W;               /* logical replicas ("Model instances"), 1 <= W <= 256 */
+    float lr;                 /* learning rate alpha of Eq. 1 */
+    uint32_t max_grad_buffer; /* Algorithm 1's maxGradBuffer; only 1 is supported */
+    uint32_t max_delay;       /* messages are delivered 0..max_delay whole steps after their origin step */
+    uint32_t row_stride;      /* floats between consecutive rows; 0 = d rounded up to a multiple of 8 */
+    uint64_t seed;            /* key of the counter-based generator (negatives, delays, seeded init) */
+    int32_t device;           /* CUDA device ordinal */
+    uint32_t reduction;       /* TENSAIR_SUM: L(X) = sum of the pair losses; TENSAIR_MEAN: their mean over the batch's pairs */
+} tensair_config;
+
+typedef struct tensair_sizes {
+    uint64_t tables_bytes;    /* W * 2V * row_stride * 4 */
+    uint64_t pool_bytes;      /* W * (max_delay + 1) message slots of worst-case size */
+    uint64_t scratch_bytes;   /* sort buffers, gradient scalars, partial sums, sampler table, counts */
+    uint32_t row_stride;      /* the stride the library will use */
+    uint32_t max_pairs;       /* pairs of a full batch: 2*w*batch - w*(w+1) when batch > w */
+    uint32_t max_rows;        /* most rows a message can have */
+    uint32_t reserved;
+} tensair_sizes;
+
+/* Caller-owned device memory and stream.  All three pointers must be 256-byte aligned. */
+typedef struct tensair_buffers {
+    void* tables;
+    uint64_t tables_bytes;
+    void* pool;
+    uint64_t pool_bytes;
+    void* scratch;
+    uint64_t scratch_bytes;
+    void* stream;             /* cudaStream_t; NULL = the legacy default stream */
+} tensair_buffers;
+
+typedef struct tensair_msg_info {
+    uint32_t n_rows;          /* rows in the message */
+    uint32_t n_in_rows;       /* of which input rows (ids < V) */
+    uint32_t n_pairs;         /* (centre, context) pairs of the batch */
+    uint32_t slot;            /* pool slot the message occupies */
+    uint64_t pool_offset;     /* byte offset of that slot in the pool */
+} tensair_msg_info;
+
+/* One entry of a receiver's delivery log. */
+typedef struct tensair_delivery {
+    uint64_t origin_step;     /* step at which the sender computed the gradient */
+    uint64_t sender;
+    uint64_t due_step;        /* origin_step + delay */
+    uint64_t applied_at;      /* step argument of the apply call that delivered it */
+    uint64_t staleness;       /* |G_i u G_j| - |G_i n G_j| of Section 3.1 */
+} tensair_delivery;
+
+/* Sizes the caller must allocate for a configuration.  No GPU is touched. */
+TENSAIR_API int tensair_workspace_bytes(const tensair_config* cfg, tensair_sizes* out);
+
+/*
+ * Constructor of Algorithm 1 for all W replicas at once: every replica starts from the same model
+ * (data parallelism as Section 2.2 describes it: identical initial replicas, disjoint data).
+ *   counts_host   host, uint64[V] unigram counts for the count^0.75 negative sampler, or NULL = all 1.
+ *                 Counts must be >= 1.  They also seed the running counts that train_batch increments.
+ *   init_in_host  host, float[V*d] dense input rows, or NULL = seeded U(-0.5/d, 0.5/d).
+ *   init_out_host host, float[V*d] dense output rows, or NULL = zeros.
+ * Host arrays are read during the call only.  Synchronous.  The context borrows `bufs`.
+ */
+TENSAIR_API int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const uint64_t* counts_host,
+                 const float* init_in_host, const float* init_out_host, tensair_ctx** out);
+
+/* Frees host state only; synchronises the stream first. */
+TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
+
+/*
+ * One mini-batch on one replica (Algorithm 1, train, mini-batch branch; Eq. 1):
+ *   pairs      every (centre position q, context position c) with 0 < |q-c| <= window inside the
+ *              batch's own n_tokens tokens, in (q ascending, c ascending) order;
+ *   negatives  k per pair from the counter-based sampler; one equal to the pair's context word is dropped;
+ *   gradient   of the SGNS loss of the whole batch (sum or mean of the pair losses, see `reduction`) at
+ *              the replica's tables as they are when the call starts (nothing is updated mid-batch);
+ *              dot products, sigmoids and row sums are taken in fp64 from the fp32 tables;
+ *   message    one delta row fp32(-lr * gradient) per touched row, ids ascending;
+ *   local GA   the message is applied to the replica at once (staleness 0);
+ *   send       it is filed for every other replica at step batch_index + delay(batch_index, replica, j).
+ * tokens_dev   device, int32[n_tokens], borrowed until the stream has passed this call; n_tokens <= batch.
+ * batch_index  the global step t of this batch (< 2^32); it selects the random draws and the message slot.
+ * loss_out     host, nullable.  Non-NULL: receives the sum of the batch's pair losses and the call synchronises.
+ * info         host, nullable.  Non-NULL: filled, and the call synchronises.
+ * A token id outside [0,V) leaves tables, counts and pool untouched and raises TENSAIR_EBADTOKEN at
+ * the next synchronising call (this one if loss_out or info is given); batches enqueued after the
+ * bad one and before that call are dropped too.
+ * TENSAIR_EPENDING: the slot of step batch_index - (max_delay+1) still has undelivered recipients
+ * (tensair_apply_messages was not called for them).
+ */
+TENSAIR_API int tensair_train_batch(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_dev, uint32_t n_tokens,
+                        uint64_t batch_index, double* loss_out, tensair_msg_info* info);
+
+/* Same step with the batch in HOST memory: copies tokens_host to the device on the stream first
+ * (asynchronously if the memory is pinned).  tokens_host must stay valid until the stream passes. */
+TENSAIR_API int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_host, uint32_t n_tokens,
+                             uint64_t batch_index, double* loss_out, tensair_msg_info* info);
+
+/*
+ * Algorithm 1, train, gradient branch, for one receiver: applies every pending message whose due step
+ * is <= step, in (origin step, sender) order - the order in which Section 3.1 has a Model work off
+ * the gradients that arrived while it was busy.  Call it for step t after every replica has run
+ * tensair_train_batch for step t.  A second call for the same (replica, step) applies nothing.
+ * n_applied: host, nullable.
+ */
+TENSAIR_API int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint64_t step, uint32_t* n_applied);
+
+/* End of a run: delivers everything still pending, per receiver in (due step, origin step, sender)
+ * order, so that all replicas have applied the same gradients.  n_applied: host, nullable. */
+TENSAIR_API int tensair_drain(tensair_ctx* ctx, uint32_t* n_applied);
+
+/* Rebuilds the negative sampler's alias table from the running unigram counts (initial counts plus
+ * every token trained on so far).  Synchronises; the table is built by one host thread. */
+TENSAIR_API int tensair_update_sampler(tensair_ctx* ctx);
+
+/* Waits for the stream; returns and clears a pending TENSAIR_EBADTOKEN. */
+TENSAIR_API int tensair_sync(tensair_ctx* ctx);
+
+/* Copies rows [row0, row0+nrows) of a replica's input (which=0) or output (which=1) table into
+ * host_dst as dense float[nrows*d].  Synchronises.  (For this model "prediction" is this lookup.) */
+TENSAIR_API int tensair_read_embeddings(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows,
+                            float* host_dst);
+/* The reverse copy (restore from a dump).  Synchronises. */
+TENSAIR_API int tensair_write_embeddings(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows,
+                             const float* host_src);
+
+/* ---- parity taps (synchronous; for tests and diagnostics) ---- */
+
+/* Raw negative draws of the last train_batch call: host uint32[n_pairs*k] (nullable); n_pairs nullable. */
+TENSAIR_API int tensair_read_negatives(tensair_ctx* ctx, uint32_t* host_neg, uint32_t* n_pairs);
+/* Gradient scalars g[p][0..k] of the last train_batch call (dropped negatives read 0): host double[n_pairs*(k+1)]. */
+TENSAIR_API int tensair_read_scalars(tensair_ctx* ctx, double* host_g);
+/* Message of (replica, batch_index) while its slot has not been reused: n_rows (nullable), ids
+ * host uint32[n_rows] (nullable), delta host float[n_rows*d] dense (nullable). */
+TENSAIR_API int tensair_read_message(tensair_ctx* ctx, uint32_t replica, uint64_t batch_index, uint32_t* n_rows,
+                         uint32_t* host_ids, float* host_delta);
+/* Sampler state: any of thresh uint32[V], alias uint32[V], counts uint64[V] (host, nullable). */
+TENSAIR_API int tensair_read_sampler(tensair_ctx* ctx, uint32_t* thresh, uint32_t* alias, uint64_t* counts);
+/* Delivery log of one receiver, oldest first: up to max_records entries into host `out`; n receives the count held. */
+TENSAIR_API int tensair_read_delivery_log(tensair_ctx* ctx, uint32_t replica, uint64_t max_records, tensair_delivery* out,
+                              uint64_t* n);
+/* Messages filed for a receiver and not yet applied. */
+TENSAIR_API int tensair_pending(tensair_ctx* ctx, uint32_t replica, uint64_t* n);
+/* Kernels launched by this context so far. */
+TENSAIR_API uint64_t tensair_kernel_launches(const tensair_ctx* ctx);
+
+TENSAIR_API const char* tensair_strerror(int code);
+TENSAIR_API const char* tensair_last_error(const tensair_ctx* ctx);
+
+/* ---- host-only pieces, usable without a GPU ---- */
+
+/* Walker/Vose alias table over weights count^0.75 (counts NULL = all 1): host in, host out. */
+TENSAIR_API int tensair_build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias);
+/* Philox4x32-10: counter[4], key[2] -> out[4]. */
+TENSAIR_API void tensair_philox4x32_10(const uint32_t counter[4], const uint32_t key[2], uint32_t out[4]);
+/* Delivery delay, in whole steps, of the message (sender, step) to `receiver`: uniform in 0..max_delay. */
+TENSAIR_API uint32_t tensair_delay(uint64_t seed, uint32_t max_delay, uint64_t step, uint32_t sender, uint32_t receiver);
+
+/*
+ * The delivery schedule and staleness bookkeeping on their own (the context owns one of these).
+ * on_train   records that `replica` computed and locally applied gradient (replica, step) and files
+ *            it for every other replica; TENSAIR_EPENDING if the slot it would reuse is still pending.
+ * take_due   pops the receiver's deliveries with due step <= step in (origin step, sender) order (or,
+ *            with drain != 0, all of them in (due, origin, sender) order), marks them applied at `step`
+ *            (at their due step when draining) and writes up to max_records of them; n = how many popped.
+ */
+TENSAIR_API int tensair_schedule_create(uint32_t W, uint32_t max_delay, uint64_t seed, tensair_schedule** out);
+TENSAIR_API void tensair_schedule_destroy(tensair_schedule* s);
+TENSAIR_API int tensair_schedule_on_train(tensair_schedule* s, uint32_t replica, uint64_t step);
+TENSAIR_API int tensair_schedule_take_due(tensair_schedule* s, uint32_t receiver, uint64_t step, int drain,
+                              uint64_t max_records, tensair_delivery* out, uint64_t* n);
+TENSAIR_API int tensair_schedule_pending(const tensair_schedule* s, uint32_t receiver, uint64_t* n);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* TENSAIR_H */

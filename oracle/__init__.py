@@ -41,7 +41,7 @@ def lib():
             "orc_build_alias": (None, [vp, u32, vp, vp]),
             "orc_negative": (u32, [u64, u32, u64, u32, u32, vp, vp, u32]),
             "orc_init_input_table": (None, [u64, u32, u32, vp]),
-            "orc_create": (vp, [u32, u32, u32, u32, u32, u32, f32, u32, u64, vp, vp, vp]),
+            "orc_create": (vp, [u32, u32, u32, u32, u32, u32, f32, u32, u64, u32, vp, vp, vp]),
             "orc_destroy": (None, [vp]),
             "orc_update_sampler": (None, [vp]),
             "orc_get_sampler": (None, [vp, vp, vp, vp]),
@@ -112,7 +112,7 @@ class Oracle:
     """The oracle's model replicas, sampler and message exchange."""
 
     def __init__(self, V, d, window, k, batch, W=1, lr=0.025, max_delay=0, seed=0,
-                 counts=None, init_in=None, init_out=None):
+                 counts=None, init_in=None, init_out=None, reduction=0):
         self.V, self.d, self.window, self.k, self.batch, self.W = V, d, window, k, batch, W
         self.seed = seed
         if counts is not None:
@@ -124,7 +124,7 @@ class Oracle:
         if init_out is not None:
             init_out = np.ascontiguousarray(init_out, dtype=np.float32)
             assert init_out.shape == (V, d)
-        self._h = lib().orc_create(V, d, window, k, batch, W, lr, max_delay, seed,
+        self._h = lib().orc_create(V, d, window, k, batch, W, lr, max_delay, seed, reduction,
                                    _ptr(counts), _ptr(init_in), _ptr(init_out))
 
     def close(self):
@@ -186,7 +186,7 @@ class Oracle:
         return out
 
     def read_g(self):
-        out = np.empty((self.last_pairs(), self.k + 1), dtype=np.float32)
+        out = np.empty((self.last_pairs(), self.k + 1), dtype=np.float64)
         lib().orc_read_g(self._h, _ptr(out))
         return out
 

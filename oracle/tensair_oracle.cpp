@@ -18,8 +18,10 @@
 //     default skip-gram model"): per pair  -log s(u_o.v_c) - sum_j log s(-u_nj.v_c).
 //
 // Arithmetic: tables are stored in fp32; every dot product, sigmoid, loss term and gradient sum is
-// taken in fp64 from those fp32 values; a delta row is fp32(-(double)lr * sum); applying a delta is
-// one fp32 addition per element.
+// taken in fp64 from those fp32 values; a delta row is fp32(-scale * sum) with scale = (double)lr when
+// the batch loss is the sum of the pair losses and (double)lr / (number of pairs) when it is their
+// mean (the paper does not say which; its footnoted Keras model averages over the batch); applying a
+// delta is one fp32 addition per element.
 //
 // Pins (see tests/): Philox known-answer vectors; alias-table exact reconstruction, equal-count
 // special case and chi-square; single-pair closed form; batch-0 closed form; central finite
@@ -125,7 +127,7 @@ struct Delivery { uint64_t due, origin; uint32_t sender; };
 struct LogRec { uint64_t origin, due, applied_at; uint32_t sender, staleness; };
 
 struct Oracle {
-    uint32_t V, d, window, k, batch, W, max_delay;
+    uint32_t V, d, window, k, batch, W, max_delay, reduction;
     float lr;
     uint64_t seed;
     std::vector<std::vector<float>> tin, tout;   // per replica V*d
@@ -137,7 +139,7 @@ struct Oracle {
     std::vector<std::vector<LogRec>> log;                     // per receiver
     // taps of the last train_batch
     std::vector<uint32_t> last_neg;                           // P*k raw draws
-    std::vector<float> last_g;                                // P*(1+k), masked -> 0
+    std::vector<double> last_g;                               // P*(1+k), masked -> 0
     uint32_t last_pairs = 0;
     std::pair<uint32_t, uint64_t> last_key{0, 0};
 };
@@ -209,11 +211,11 @@ void orc_init_input_table(uint64_t seed, uint32_t V, uint32_t d, float* dst) {
 }
 
 Oracle* orc_create(uint32_t V, uint32_t d, uint32_t window, uint32_t k, uint32_t batch, uint32_t W,
-                   float lr, uint32_t max_delay, uint64_t seed, const uint64_t* counts,
+                   float lr, uint32_t max_delay, uint64_t seed, uint32_t reduction, const uint64_t* counts,
                    const float* init_in, const float* init_out) {
     Oracle* o = new Oracle();
     o->V = V; o->d = d; o->window = window; o->k = k; o->batch = batch; o->W = W;
-    o->lr = lr; o->max_delay = max_delay; o->seed = seed;
+    o->lr = lr; o->max_delay = max_delay; o->seed = seed; o->reduction = reduction;
     const size_t n = (size_t)V * d;
     o->tin.assign(W, std::vector<float>());
     o->tout.assign(W, std::vector<float>());
@@ -320,8 +322,7 @@ int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t
     }
     double loss = 0.0;
     for (size_t p = 0; p < P; ++p) loss += pair_loss[p];
-    o->last_g.resize(P * K1);
-    for (size_t i = 0; i < P * K1; ++i) o->last_g[i] = (float)g[i];
+    o->last_g = g;
     o->last_pairs = (uint32_t)P;
 
     // every live (pair, j) term adds g*u to the centre's input row and g*v to the output row
@@ -341,6 +342,7 @@ int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t
     const size_t U = seg.size();
     seg.push_back(terms.size());
 
+    const double scale = o->reduction ? (double)o->lr / (double)P : (double)o->lr;
     Message m;
     m.ids.resize(U);
     m.delta.resize(U * d);
@@ -353,7 +355,7 @@ int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t
             for (uint32_t e = 0; e < d; ++e) sum[e] += terms[i].g * (double)src[e];
         }
         m.ids[r] = terms[seg[r]].id;
-        for (uint32_t e = 0; e < d; ++e) m.delta[r * d + e] = (float)(-(double)o->lr * sum[e]);
+        for (uint32_t e = 0; e < d; ++e) m.delta[r * d + e] = (float)(-scale * sum[e]);
     }
 
     // local apply (staleness 0), then send to every other replica
@@ -415,7 +417,7 @@ void orc_write_embeddings(Oracle* o, uint32_t replica, int which, uint32_t row0,
 
 uint32_t orc_last_pairs(Oracle* o) { return o->last_pairs; }
 void orc_read_negatives(Oracle* o, uint32_t* dst) { std::copy(o->last_neg.begin(), o->last_neg.end(), dst); }
-void orc_read_g(Oracle* o, float* dst) { std::copy(o->last_g.begin(), o->last_g.end(), dst); }
+void orc_read_g(Oracle* o, double* dst) { std::copy(o->last_g.begin(), o->last_g.end(), dst); }
 
 // Message (replica, batch_index): returns its row count, or -1 when it is no longer held.
 int64_t orc_read_message(Oracle* o, uint32_t replica, uint64_t batch_index, uint32_t* ids, float* delta) {

@@ -1,0 +1,64 @@
+// Gradient application of a sparse message: table[id] += delta for every row of the message.
+//
+// Pure streaming scatter-add: the delta rows are contiguous, the ids ascend, so the table rows are
+// visited in address order.  One warp per row, 128-bit accesses, rows taken in a grid-stride loop
+// by a grid sized to the machine; the row count is read from the message header on the device.
+#include "kernels.h"
+
+namespace tensair {
+
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_apply(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids, const float4* __restrict__ delta,
+        float4* __restrict__ table, uint32_t d4, uint32_t stride4, int input_rows_only) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t limit = input_rows_only ? hdr->n_in_rows : hdr->n_rows;
+    for (uint32_t m = warp; m < limit; m += nwarps) {
+        const uint32_t id = __ldg(ids + m);
+        const float4* __restrict__ src = delta + (size_t)m * stride4;
+        float4* __restrict__ dst = table + (size_t)id * stride4;
+        float4 a[NV], b[NV];
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const uint32_t e = lane + 32 * i;
+            if (e < d4) {
+                a[i] = __ldg(src + e);
+                b[i] = dst[e];
+            }
+        }
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const uint32_t e = lane + 32 * i;
+            if (e < d4) {
+                b[i].x += a[i].x; b[i].y += a[i].y; b[i].z += a[i].z; b[i].w += a[i].w;
+                dst[e] = b[i];
+            }
+        }
+    }
+}
+
+cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
+                              float* table, const Shape& s, int input_rows_only) {
+    const uint32_t stride4 = s.stride / 4;
+    const int blocks = L.sms * 8;
+    const float4* d4p = reinterpret_cast<const float4*>(delta);
+    float4* t4 = reinterpret_cast<float4*>(table);
+#define TENSAIR_APPLY(NV) k_apply<NV><<<blocks, 256, 0, L.stream>>>(hdr, ids, d4p, t4, s.d4, stride4, input_rows_only)
+    if (s.d4 <= 32) TENSAIR_APPLY(1);
+    else if (s.d4 <= 64) TENSAIR_APPLY(2);
+    else if (s.d4 <= 96) TENSAIR_APPLY(3);
+    else if (s.d4 <= 128) TENSAIR_APPLY(4);
+    else TENSAIR_APPLY(8);
+#undef TENSAIR_APPLY
+    ++*L.launches;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_apply(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
+                         float* table, const Shape& s) {
+    return launch_apply_rows(L, hdr, ids, delta, table, s, 0);
+}
+
+}  // namespace tensair

@@ -1,0 +1,63 @@
+// Shared device-side definitions of the SGNS / DASGD kernels.
+#pragma once
+#include <cuda_runtime.h>
+#include <stdint.h>
+
+namespace tensair {
+
+// One sort item: key (row id in the unified [0,2V) space, or 2V for a dropped negative) in the
+// high word, payload in the low word.  Payload: the centre position q for an input-row item, the
+// contribution index c = p*(k+1)+j for an output-row item.
+typedef unsigned long long item_t;
+__host__ __device__ inline uint32_t item_key(item_t it) { return (uint32_t)(it >> 32); }
+__host__ __device__ inline uint32_t item_payload(item_t it) { return (uint32_t)it; }
+__host__ __device__ inline item_t make_item(uint32_t key, uint32_t payload) {
+    return ((item_t)key << 32) | payload;
+}
+
+// Gradient scalar of one contribution and the centre token whose input row it multiplies.
+struct Rec {
+    double g;
+    uint32_t centre;
+    uint32_t pad;
+};
+
+// Message slot header (the slot is: header, ids, delta rows).
+struct MsgHeader {
+    uint32_t n_rows;     // distinct touched rows
+    uint32_t n_in_rows;  // of which input rows
+    uint32_t n_items;    // sort items that are not dropped negatives
+    uint32_t pad;
+};
+constexpr uint32_t kHeaderBytes = 256;
+
+// A long row (more contributions than one warp takes in one go) and its chunk partials.
+struct LongRow {
+    uint32_t m;          // message row index
+    uint32_t base;       // first partial slot
+    uint32_t nchunks;
+};
+struct ChunkItem {
+    uint32_t m;
+    uint32_t chunk;
+};
+constexpr uint32_t kChunk = 128;   // contributions per chunk; rows with more than this go the long way
+
+// Sum over i < x of min(i, w): how many left (or, mirrored, right) neighbours the first x positions have.
+__host__ __device__ inline uint64_t neighbours_before(uint64_t x, uint64_t w) {
+    return x <= w + 1 ? x * (x - (x ? 1 : 0)) / 2 : w * (w + 1) / 2 + (x - w - 1) * w;
+}
+// Index of the first pair of centre position q in a batch of n tokens with window w,
+// pairs enumerated by (q ascending, context position ascending).
+__host__ __device__ inline uint32_t pair_offset(uint32_t q, uint32_t n, uint32_t w) {
+    return (uint32_t)(neighbours_before(q, w) + neighbours_before(n, w) - neighbours_before(n - q, w));
+}
+__host__ __device__ inline uint32_t pair_count(uint32_t n, uint32_t w) {
+    return (uint32_t)(2 * neighbours_before(n, w));
+}
+
+struct Shape {
+    uint32_t V, d, d4, stride, w, k, K1;
+};
+
+}  // namespace tensair

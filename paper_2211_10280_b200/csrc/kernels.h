@@ -1,0 +1,51 @@
+// Host-side launchers of the kernels; each enqueues on L.stream and returns the launch status.
+#pragma once
+#include "common.cuh"
+
+namespace tensair {
+
+struct Launcher {
+    cudaStream_t stream;
+    uint64_t* launches;   // incremented once per kernel launch
+    int sms;              // multiprocessors of the device
+};
+
+// sampler.cu
+cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, uint32_t V, uint32_t* err);
+cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, uint32_t replica,
+                           uint32_t batch_lo, uint64_t seed, const uint2* alias_tab, uint32_t* rows,
+                           item_t* items, unsigned long long* counts, const uint32_t* err);
+cudaError_t launch_init_input_table(const Launcher& L, float* table, const Shape& s, uint64_t seed);
+void build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias);
+
+// radix_sort.cu
+// Stable least-significant-digit radix sort of `n` items by the low `key_bits` bits of their keys.
+// `a` holds the input; `b` and `hist` are scratch.  *sorted receives whichever of a / b holds the result.
+cudaError_t launch_sort(const Launcher& L, item_t* a, item_t* b, uint32_t n, uint32_t key_bits, uint32_t* hist,
+                        item_t** sorted);
+uint32_t sort_tiles(uint32_t n);
+uint32_t sort_hist_words(uint32_t n);
+
+// forward.cu
+cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
+                           const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, const uint32_t* err);
+cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err);
+
+// message.cu
+uint32_t heads_tiles(uint32_t n_items);
+cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
+                         MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
+                         const uint32_t* err);
+cudaError_t launch_reduce(const Launcher& L, const item_t* sorted, const MsgHeader* hdr, const uint32_t* ids,
+                          const uint32_t* seg_start, const Rec* rec, const double* gin_pos, float* table,
+                          float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
+                          ChunkItem* chunk_items, double* partials);
+
+// apply.cu
+cudaError_t launch_apply(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
+                         float* table, const Shape& s);
+// Same, restricted to the message's input rows when input_rows_only != 0.
+cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
+                              float* table, const Shape& s, int input_rows_only);
+
+}  // namespace tensair

@@ -1,0 +1,387 @@
+// Building the sparse gradient message from the row-sorted contributions, fused with the local
+// gradient application of its output rows.
+//
+// After the stable sort all contributions to one row are contiguous and in a fixed order.  "Heads"
+// (first item of each distinct key) give the message's ascending id list and the segment bounds.
+// A warp then owns a row: it adds coefficient * source row over the segment (source = the centre's
+// input row and coefficient g for an output row; source = a position's partial centre gradient and
+// coefficient 1 for an input row), scales by -lr, writes the delta row into the message and, for an
+// output row, adds it to the table in the same pass.  Input rows are NOT updated here: they are the
+// sources of every output-row sum and must keep their snapshot values until all sums are done.
+// Rows with more than kChunk contributions are split into chunks that run on separate warps; their
+// partial sums are combined in chunk order, so every sum has a fixed association.  All sums are
+// accumulated in fp64 from the fp32 scalars and rows.
+#include "kernels.h"
+
+namespace tensair {
+
+constexpr int kHeadThreads = 256;
+constexpr int kHeadItems = 8;
+constexpr int kHeadTile = kHeadThreads * kHeadItems;
+
+uint32_t heads_tiles(uint32_t n_items) { return (n_items + kHeadTile - 1) / kHeadTile; }
+
+__device__ inline uint32_t head_flags(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t first,
+                                      uint32_t keys[kHeadItems]) {
+    uint32_t flags = 0;
+    uint32_t prev = first > 0 && first <= n_items ? item_key(sorted[first - 1]) : 0xFFFFFFFFu;
+#pragma unroll
+    for (int i = 0; i < kHeadItems; ++i) {
+        const uint32_t idx = first + i;
+        keys[i] = idx < n_items ? item_key(sorted[idx]) : 0xFFFFFFFFu;
+        if (idx < n_items && (idx == 0 || keys[i] != prev)) flags |= 1u << i;
+        prev = keys[i];
+    }
+    return flags;
+}
+
+__global__ void __launch_bounds__(kHeadThreads)
+k_heads_count(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t* __restrict__ tile_counts,
+              const uint32_t* __restrict__ err) {
+    if (*err) return;
+    __shared__ uint32_t warp_sum[kHeadThreads / 32];
+    uint32_t keys[kHeadItems];
+    const uint32_t first = blockIdx.x * kHeadTile + threadIdx.x * kHeadItems;
+    uint32_t c = __popc(head_flags(sorted, n_items, first, keys));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+        for (int i = 0; i < kHeadThreads / 32; ++i) t += warp_sum[i];
+        tile_counts[blockIdx.x] = t;
+    }
+}
+
+// One block: exclusive scan of the tile counts, message header, counters of the long-row lists.
+__global__ void __launch_bounds__(1024)
+k_heads_scan(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, uint32_t* __restrict__ tile_counts,
+             uint32_t tiles, MsgHeader* __restrict__ hdr, uint32_t* __restrict__ seg_start,
+             uint32_t* __restrict__ long_counters, const uint32_t* __restrict__ err) {
+    __shared__ uint32_t warp_tot[32];
+    __shared__ uint32_t carry_s;
+    if (threadIdx.x == 0) {
+        long_counters[0] = 0;
+        long_counters[1] = 0;
+        carry_s = 0;
+    }
+    if (*err) {
+        if (threadIdx.x == 0) *hdr = MsgHeader{0, 0, 0, 0};
+        return;
+    }
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (uint32_t base = 0; base < tiles; base += 1024) {
+        const uint32_t idx = base + threadIdx.x;
+        const uint32_t v = idx < tiles ? tile_counts[idx] : 0;
+        uint32_t incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= (uint32_t)o) incl += t;
+        }
+        if (lane == 31) warp_tot[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            const uint32_t t = warp_tot[lane];
+            uint32_t ti = t;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, ti, o);
+                if (lane >= (uint32_t)o) ti += u;
+            }
+            warp_tot[lane] = ti - t;
+        }
+        __syncthreads();
+        const uint32_t carry = carry_s;
+        if (idx < tiles) tile_counts[idx] = carry + warp_tot[wid] + incl - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = carry + warp_tot[wid] + incl;
+        __syncthreads();
+    }
+    if (threadIdx.x == 0) {
+        const uint32_t heads = carry_s;
+        const bool dropped = n_items > 0 && item_key(sorted[n_items - 1]) == 2 * V;
+        const uint32_t n_rows = heads - (dropped ? 1u : 0u);
+        hdr->n_rows = n_rows;
+        hdr->pad = 0;
+        seg_start[heads] = n_items;
+        if (!dropped) hdr->n_items = n_items;   // otherwise written by the head of the dropped run
+    }
+}
+
+__global__ void __launch_bounds__(kHeadThreads)
+k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, const uint32_t* __restrict__ tile_base,
+              MsgHeader* __restrict__ hdr, uint32_t* __restrict__ ids, uint32_t* __restrict__ seg_start,
+              const uint32_t* __restrict__ err) {
+    if (*err) return;
+    __shared__ uint32_t warp_tot[kHeadThreads / 32];
+    uint32_t keys[kHeadItems];
+    const uint32_t first = blockIdx.x * kHeadTile + threadIdx.x * kHeadItems;
+    const uint32_t flags = head_flags(sorted, n_items, first, keys);
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    const uint32_t c = __popc(flags);
+    uint32_t incl = c;
+#pragma unroll
+    for (int o = 1; o < 32; o <<= 1) {
+        const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+        if (lane >= (uint32_t)o) incl += t;
+    }
+    if (lane == 31) warp_tot[wid] = incl;
+    __syncthreads();
+    uint32_t m = tile_base[blockIdx.x] + incl - c;
+    for (uint32_t x = 0; x < wid; ++x) m += warp_tot[x];
+    uint32_t prev = first > 0 && first <= n_items ? item_key(sorted[first - 1]) : 0u;
+#pragma unroll
+    for (int i = 0; i < kHeadItems; ++i) {
+        if (flags & (1u << i)) {
+            const uint32_t key = keys[i];
+            seg_start[m] = first + i;
+            if (key < 2 * V) ids[m] = key;
+            else hdr->n_items = first + i;                       // first dropped negative
+            if (key >= V && (first + i == 0 || prev < V)) hdr->n_in_rows = m;   // first output row
+            ++m;
+        }
+        prev = keys[i];
+    }
+}
+
+cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
+                         MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
+                         const uint32_t* err) {
+    const uint32_t tiles = heads_tiles(n_items);
+    if (tiles) {
+        k_heads_count<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, tile_counts, err);
+        ++*L.launches;
+    }
+    k_heads_scan<<<1, 1024, 0, L.stream>>>(sorted, n_items, V, tile_counts, tiles, hdr, seg_start, long_counters, err);
+    ++*L.launches;
+    if (tiles) {
+        k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, err);
+        ++*L.launches;
+    }
+    return cudaGetLastError();
+}
+
+// ---------------------------------------------------------------------------------------------
+// per-row sums
+// ---------------------------------------------------------------------------------------------
+constexpr int kTermsInFlight = 4;
+
+// One lane's share of a row sum: fp64 accumulators for its NV float4 slices.
+template <int NV>
+struct RowSum {
+    double a[NV][4];
+    __device__ inline void clear() {
+#pragma unroll
+        for (int i = 0; i < NV; ++i) a[i][0] = a[i][1] = a[i][2] = a[i][3] = 0.0;
+    }
+};
+
+// Adds coefficient * source over sorted[beg, end) in item order.  Sources and coefficients are fp32;
+// products and sums are taken in fp64, so the result does not feel the cancellation between the
+// positive and negative terms of a row.
+template <int NV>
+__device__ inline void accumulate_segment(const item_t* __restrict__ sorted, uint32_t beg, uint32_t end, bool input_row,
+                                          const Rec* __restrict__ rec, const double* __restrict__ gin_pos,
+                                          const float4* __restrict__ table, uint32_t d4, uint32_t stride4,
+                                          uint32_t lane, RowSum<NV>& sum) {
+    if (input_row) {
+        // sources are the fp64 partial centre gradients of the positions holding this token
+        for (uint32_t i = beg; i < end; ++i) {
+            const double2* src = reinterpret_cast<const double2*>(gin_pos + (size_t)item_payload(sorted[i]) * stride4 * 4);
+#pragma unroll
+            for (int j = 0; j < NV; ++j) {
+                const uint32_t e = lane + 32 * j;
+                if (e < d4) {
+                    const double2 lo = src[2 * e], hi = src[2 * e + 1];
+                    sum.a[j][0] += lo.x; sum.a[j][1] += lo.y; sum.a[j][2] += hi.x; sum.a[j][3] += hi.y;
+                }
+            }
+        }
+        return;
+    }
+    for (uint32_t i0 = beg; i0 < end; i0 += kTermsInFlight) {
+        const float4* src[kTermsInFlight];
+        double coef[kTermsInFlight];
+#pragma unroll
+        for (int t = 0; t < kTermsInFlight; ++t) {
+            coef[t] = 0.0;
+            src[t] = table;
+            if (i0 + t < end) {
+                const Rec r = rec[item_payload(sorted[i0 + t])];
+                coef[t] = r.g;
+                src[t] = table + (size_t)r.centre * stride4;
+            }
+        }
+        float4 x[kTermsInFlight][NV];
+#pragma unroll
+        for (int t = 0; t < kTermsInFlight; ++t)
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const uint32_t e = lane + 32 * i;
+                x[t][i] = (i0 + t < end && e < d4) ? src[t][e] : make_float4(0.f, 0.f, 0.f, 0.f);
+            }
+#pragma unroll
+        for (int t = 0; t < kTermsInFlight; ++t)
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                sum.a[i][0] = fma(coef[t], (double)x[t][i].x, sum.a[i][0]);
+                sum.a[i][1] = fma(coef[t], (double)x[t][i].y, sum.a[i][1]);
+                sum.a[i][2] = fma(coef[t], (double)x[t][i].z, sum.a[i][2]);
+                sum.a[i][3] = fma(coef[t], (double)x[t][i].w, sum.a[i][3]);
+            }
+    }
+}
+
+// delta = fp32(-scale * sum); the delta row goes into the message and, for an output row, onto the table.
+template <int NV>
+__device__ inline void finish_row(const RowSum<NV>& sum, uint32_t m, uint32_t id, uint32_t V, double scale,
+                                  float4* __restrict__ table, float4* __restrict__ delta, uint32_t d4,
+                                  uint32_t stride4, uint32_t lane) {
+    const double nlr = -scale;
+#pragma unroll
+    for (int i = 0; i < NV; ++i) {
+        const uint32_t e = lane + 32 * i;
+        if (e < d4) {
+            const float4 dl = make_float4((float)(nlr * sum.a[i][0]), (float)(nlr * sum.a[i][1]),
+                                          (float)(nlr * sum.a[i][2]), (float)(nlr * sum.a[i][3]));
+            delta[(size_t)m * stride4 + e] = dl;
+            if (id >= V) {
+                float4 t = table[(size_t)id * stride4 + e];
+                t.x += dl.x; t.y += dl.y; t.z += dl.z; t.w += dl.w;
+                table[(size_t)id * stride4 + e] = t;
+            }
+        }
+    }
+}
+
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_reduce_rows(const item_t* __restrict__ sorted, const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids,
+              const uint32_t* __restrict__ seg_start, const Rec* __restrict__ rec, const double* __restrict__ gin_pos,
+              float4* __restrict__ table, float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4,
+              double scale, uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows,
+              ChunkItem* __restrict__ chunk_items) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t n_rows = hdr->n_rows;
+    for (uint32_t m = warp; m < n_rows; m += nwarps) {
+        const uint32_t beg = seg_start[m], end = seg_start[m + 1];
+        const uint32_t id = ids[m];
+        if (end - beg > kChunk) {
+            const uint32_t nch = (end - beg + kChunk - 1) / kChunk;
+            uint32_t base = 0;
+            if (lane == 0) {
+                const uint32_t slot = atomicAdd(long_counters, 1u);
+                base = atomicAdd(long_counters + 1, nch);
+                long_rows[slot] = LongRow{m, base, nch};
+            }
+            base = __shfl_sync(0xFFFFFFFFu, base, 0);
+            for (uint32_t c = lane; c < nch; c += 32) chunk_items[base + c] = ChunkItem{m, c};
+            continue;
+        }
+        RowSum<NV> sum;
+        sum.clear();
+        accumulate_segment<NV>(sorted, beg, end, id < V, rec, gin_pos, table, d4, stride4, lane, sum);
+        finish_row<NV>(sum, m, id, V, scale, table, delta, d4, stride4, lane);
+    }
+}
+
+// Partial sums of the chunks of long rows, one warp per chunk; partials are kept in fp64.
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_reduce_chunks(const item_t* __restrict__ sorted, const uint32_t* __restrict__ ids, const uint32_t* __restrict__ seg_start,
+                const Rec* __restrict__ rec, const double* __restrict__ gin_pos, const float4* __restrict__ table,
+                uint32_t V, uint32_t d4, uint32_t stride4, const uint32_t* __restrict__ long_counters,
+                const ChunkItem* __restrict__ chunk_items, double* __restrict__ partials) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t n_chunks = long_counters[1];
+    for (uint32_t x = warp; x < n_chunks; x += nwarps) {
+        const ChunkItem ci = chunk_items[x];
+        const uint32_t beg = seg_start[ci.m] + ci.chunk * kChunk;
+        const uint32_t seg_end = seg_start[ci.m + 1];
+        const uint32_t end = beg + kChunk < seg_end ? beg + kChunk : seg_end;
+        RowSum<NV> sum;
+        sum.clear();
+        accumulate_segment<NV>(sorted, beg, end, ids[ci.m] < V, rec, gin_pos, table, d4, stride4, lane, sum);
+        double* out = partials + (size_t)x * stride4 * 4;
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const uint32_t e = lane + 32 * i;
+            if (e < d4) {
+                reinterpret_cast<double2*>(out)[2 * e] = make_double2(sum.a[i][0], sum.a[i][1]);
+                reinterpret_cast<double2*>(out)[2 * e + 1] = make_double2(sum.a[i][2], sum.a[i][3]);
+            }
+        }
+    }
+}
+
+// Long rows: the chunk partials are added in chunk order, then the row is finished like a short one.
+template <int NV>
+__global__ void __launch_bounds__(256)
+k_reduce_long(const uint32_t* __restrict__ ids, const double* __restrict__ partials, float4* __restrict__ table,
+              float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4, double scale,
+              const uint32_t* __restrict__ long_counters, const LongRow* __restrict__ long_rows) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    const uint32_t n_long = long_counters[0];
+    for (uint32_t x = warp; x < n_long; x += nwarps) {
+        const LongRow row = long_rows[x];
+        RowSum<NV> sum;
+        sum.clear();
+        for (uint32_t c = 0; c < row.nchunks; ++c) {
+            const double2* in = reinterpret_cast<const double2*>(partials + (size_t)(row.base + c) * stride4 * 4);
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const uint32_t e = lane + 32 * i;
+                if (e < d4) {
+                    const double2 lo = in[2 * e], hi = in[2 * e + 1];
+                    sum.a[i][0] += lo.x; sum.a[i][1] += lo.y; sum.a[i][2] += hi.x; sum.a[i][3] += hi.y;
+                }
+            }
+        }
+        finish_row<NV>(sum, row.m, ids[row.m], V, scale, table, delta, d4, stride4, lane);
+    }
+}
+
+template <int NV>
+static cudaError_t reduce_all(const Launcher& L, const item_t* sorted, const MsgHeader* hdr, const uint32_t* ids,
+                              const uint32_t* seg_start, const Rec* rec, const double* gin_pos, float* table,
+                              float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
+                              ChunkItem* chunk_items, double* partials) {
+    const uint32_t stride4 = s.stride / 4;
+    const int blocks = L.sms * 8;
+    float4* t4 = reinterpret_cast<float4*>(table);
+    float4* d4p = reinterpret_cast<float4*>(delta);
+    k_reduce_rows<NV><<<blocks, 256, 0, L.stream>>>(sorted, hdr, ids, seg_start, rec, gin_pos, t4, d4p, s.V, s.d4, stride4,
+                                                    scale, long_counters, long_rows, chunk_items);
+    k_reduce_chunks<NV><<<blocks, 256, 0, L.stream>>>(sorted, ids, seg_start, rec, gin_pos, t4, s.V, s.d4, stride4,
+                                                      long_counters, chunk_items, partials);
+    k_reduce_long<NV><<<L.sms * 2, 256, 0, L.stream>>>(ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters,
+                                                       long_rows);
+    *L.launches += 3;
+    return cudaGetLastError();
+}
+
+cudaError_t launch_reduce(const Launcher& L, const item_t* sorted, const MsgHeader* hdr, const uint32_t* ids,
+                          const uint32_t* seg_start, const Rec* rec, const double* gin_pos, float* table,
+                          float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
+                          ChunkItem* chunk_items, double* partials) {
+#define TENSAIR_RED(NV) \
+    return reduce_all<NV>(L, sorted, hdr, ids, seg_start, rec, gin_pos, table, delta, s, scale, long_counters, long_rows, \
+                          chunk_items, partials)
+    if (s.d4 <= 32) TENSAIR_RED(1);
+    if (s.d4 <= 64) TENSAIR_RED(2);
+    if (s.d4 <= 96) TENSAIR_RED(3);
+    if (s.d4 <= 128) TENSAIR_RED(4);
+    TENSAIR_RED(8);
+#undef TENSAIR_RED
+}
+
+}  // namespace tensair

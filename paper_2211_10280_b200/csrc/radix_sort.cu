@@ -1,0 +1,150 @@
+// Stable least-significant-digit radix sort of 64-bit items by (a bit range of) their 32-bit keys.
+//
+// Keys are row ids, dense in [0, 2V], so few digit passes are needed.  Every pass is three kernels:
+// per-tile digit histogram, exclusive scan of the digit-major histogram, stable scatter.  Stability
+// (equal keys keep their input order) is what makes the later per-row sums run in a fixed order.
+// The whole working set (two item buffers) stays in L2 at the sizes of interest.
+#include "kernels.h"
+
+namespace tensair {
+
+constexpr int kRadixBits = 8;
+constexpr int kBins = 1 << kRadixBits;
+constexpr int kSortThreads = 256;
+constexpr int kSortWarps = kSortThreads / 32;
+constexpr int kItemsPerThread = 16;
+constexpr int kTile = kSortThreads * kItemsPerThread;   // 4096 items per block
+constexpr int kWarpSpan = 32 * kItemsPerThread;         // consecutive items owned by one warp
+
+uint32_t sort_tiles(uint32_t n) { return (n + kTile - 1) / kTile; }
+uint32_t sort_hist_words(uint32_t n) { return sort_tiles(n) * kBins; }
+
+__global__ void __launch_bounds__(kSortThreads)
+k_radix_hist(const item_t* __restrict__ in, uint32_t n, uint32_t shift, uint32_t* __restrict__ hist, uint32_t tiles) {
+    __shared__ uint32_t h[kBins];
+    h[threadIdx.x] = 0;
+    __syncthreads();
+    const uint32_t base = blockIdx.x * kTile;
+#pragma unroll 4
+    for (int i = 0; i < kItemsPerThread; ++i) {
+        const uint32_t idx = base + i * kSortThreads + threadIdx.x;
+        if (idx < n) atomicAdd(&h[(item_key(in[idx]) >> shift) & (kBins - 1)], 1u);
+    }
+    __syncthreads();
+    hist[threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];   // digit-major
+}
+
+// Exclusive scan, in place, of `count` words by one block.
+__global__ void __launch_bounds__(1024) k_scan_exclusive(uint32_t* __restrict__ data, uint32_t count) {
+    __shared__ uint32_t warp_tot[32];
+    __shared__ uint32_t carry_s;
+    if (threadIdx.x == 0) carry_s = 0;
+    __syncthreads();
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (uint32_t base = 0; base < count; base += 1024) {
+        const uint32_t idx = base + threadIdx.x;
+        const uint32_t v = idx < count ? data[idx] : 0;
+        uint32_t incl = v;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= (uint32_t)o) incl += t;
+        }
+        if (lane == 31) warp_tot[wid] = incl;
+        __syncthreads();
+        if (wid == 0) {
+            const uint32_t t = warp_tot[lane];
+            uint32_t ti = t;
+#pragma unroll
+            for (int o = 1; o < 32; o <<= 1) {
+                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, ti, o);
+                if (lane >= (uint32_t)o) ti += u;
+            }
+            warp_tot[lane] = ti - t;   // exclusive over warps
+        }
+        __syncthreads();
+        const uint32_t carry = carry_s;
+        if (idx < count) data[idx] = carry + warp_tot[wid] + incl - v;
+        __syncthreads();
+        if (threadIdx.x == 1023) carry_s = carry + warp_tot[wid] + incl;
+        __syncthreads();
+    }
+}
+
+// Stable scatter.  Warp w of a block owns the consecutive items [w*512, (w+1)*512) of the tile and
+// walks them 32 at a time; lanes with the same digit are ranked by lane order within a round and
+// rounds are ranked by their order, so the rank of an item among equal digits follows input order.
+__global__ void __launch_bounds__(kSortThreads)
+k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_t n, uint32_t shift,
+                const uint32_t* __restrict__ hist, uint32_t tiles) {
+    __shared__ uint32_t cnt[kSortWarps][kBins];
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    for (int i = threadIdx.x; i < kSortWarps * kBins; i += kSortThreads) (&cnt[0][0])[i] = 0;
+    __syncthreads();
+    item_t item[kItemsPerThread];
+    uint32_t rank[kItemsPerThread];
+    const uint32_t wbase = blockIdx.x * kTile + wid * kWarpSpan;
+    const uint32_t lt_mask = (1u << lane) - 1;
+#pragma unroll
+    for (int r = 0; r < kItemsPerThread; ++r) {
+        const uint32_t idx = wbase + r * 32 + lane;
+        const bool valid = idx < n;
+        item[r] = valid ? in[idx] : 0;
+        const uint32_t live = __ballot_sync(0xFFFFFFFFu, valid);
+        rank[r] = 0;
+        if (valid) {
+            const uint32_t digit = (item_key(item[r]) >> shift) & (kBins - 1);
+            const uint32_t peers = __match_any_sync(live, digit);
+            const int leader = __ffs(peers) - 1;
+            uint32_t before = 0;
+            if ((int)lane == leader) {
+                before = cnt[wid][digit];
+                cnt[wid][digit] = before + __popc(peers);
+            }
+            before = __shfl_sync(peers, before, leader);
+            rank[r] = before + __popc(peers & lt_mask);
+        }
+        __syncwarp();
+    }
+    __syncthreads();
+    // per digit: global base of this tile, then exclusive prefix over the warps of the block
+    {
+        const uint32_t digit = threadIdx.x;
+        uint32_t run = hist[digit * tiles + blockIdx.x];
+#pragma unroll
+        for (int w = 0; w < kSortWarps; ++w) {
+            const uint32_t c = cnt[w][digit];
+            cnt[w][digit] = run;
+            run += c;
+        }
+    }
+    __syncthreads();
+#pragma unroll
+    for (int r = 0; r < kItemsPerThread; ++r) {
+        const uint32_t idx = wbase + r * 32 + lane;
+        if (idx < n) {
+            const uint32_t digit = (item_key(item[r]) >> shift) & (kBins - 1);
+            out[cnt[wid][digit] + rank[r]] = item[r];
+        }
+    }
+}
+
+cudaError_t launch_sort(const Launcher& L, item_t* a, item_t* b, uint32_t n, uint32_t key_bits, uint32_t* hist,
+                        item_t** sorted) {
+    *sorted = a;
+    if (n == 0) return cudaSuccess;
+    const uint32_t tiles = sort_tiles(n);
+    item_t* src = a;
+    item_t* dst = b;
+    for (uint32_t shift = 0; shift < key_bits; shift += kRadixBits) {
+        k_radix_hist<<<tiles, kSortThreads, 0, L.stream>>>(src, n, shift, hist, tiles);
+        k_scan_exclusive<<<1, 1024, 0, L.stream>>>(hist, tiles * kBins);
+        k_radix_scatter<<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles);
+        *L.launches += 3;
+        item_t* t = src; src = dst; dst = t;
+    }
+    *sorted = src;
+    return cudaGetLastError();
+}
+
+}  // namespace tensair

@@ -1,0 +1,156 @@
+// Negative sampler: alias table over count^0.75 (host build), token validation, and the kernel that
+// draws the negatives of a batch and emits the sort items of all its contributions.
+#include <cmath>
+#include <vector>
+
+#include "kernels.h"
+#include "philox.cuh"
+
+namespace tensair {
+
+// Walker/Vose alias table.  weight = (sqrt(sqrt(count)))^3 so that only correctly rounded operations
+// are involved; scaled probability p = weight * V / total with total summed in index order.  Entries
+// with p < 1 ("small") and p >= 1 ("large") are queued in index order; each small entry s is paired
+// with the large entry l at the head of its queue: thresh[s] = floor(p_s * 2^32) (saturated), alias[s]
+// = l, p_l = (p_l + p_s) - 1, and l joins the tail of the small queue once p_l < 1.  Entries never
+// paired accept always (thresh = 2^32-1, alias = self).
+void build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias) {
+    std::vector<double> prob(V);
+    double total = 0.0;
+    for (uint32_t i = 0; i < V; ++i) {
+        const double root4 = std::sqrt(std::sqrt(counts ? (double)counts[i] : 1.0));
+        prob[i] = root4 * root4 * root4;
+        total += prob[i];
+    }
+    // queues as arrays with a read cursor: at most V entries ever enter each
+    std::vector<uint32_t> q_small, q_large;
+    q_small.reserve(2 * (size_t)V);
+    q_large.reserve(V);
+    for (uint32_t i = 0; i < V; ++i) {
+        prob[i] = prob[i] * (double)V / total;
+        thresh[i] = 0xFFFFFFFFu;
+        alias[i] = i;
+        if (prob[i] < 1.0) q_small.push_back(i); else q_large.push_back(i);
+    }
+    size_t rs = 0, rl = 0;
+    while (rs < q_small.size() && rl < q_large.size()) {
+        const uint32_t s = q_small[rs++];
+        const uint32_t l = q_large[rl];
+        const double scaled = std::floor(prob[s] * 4294967296.0);
+        thresh[s] = scaled < 4294967295.0 ? (uint32_t)scaled : 0xFFFFFFFFu;
+        alias[s] = l;
+        prob[l] = (prob[l] + prob[s]) - 1.0;
+        if (prob[l] < 1.0) {
+            ++rl;
+            q_small.push_back(l);
+        }
+    }
+}
+
+__global__ void k_validate(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t* err) {
+    const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
+    if (i < n) {
+        const int32_t t = tok[i];
+        if (t < 0 || (uint32_t)t >= V) atomicOr(err, 1u);
+    }
+}
+
+cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, uint32_t V, uint32_t* err) {
+    if (n == 0) return cudaSuccess;
+    k_validate<<<(n + 255) / 256, 256, 0, L.stream>>>(tok, n, V, err);
+    ++*L.launches;
+    return cudaGetLastError();
+}
+
+__device__ inline uint32_t alias_pick(const uint2* __restrict__ tab, uint32_t V, uint32_t ra, uint32_t rb) {
+    const uint32_t slot = __umulhi(ra, V);
+    const uint2 e = __ldg(tab + slot);   // x = thresh, y = alias
+    return (e.x == 0xFFFFFFFFu || rb < e.x) ? slot : e.y;
+}
+
+// One thread per (centre position q, window slot s, draw pair jp).  Window slot s in [0, 2w) stands
+// for context position q + (s < w ? s - w : s - w + 1); slots outside the batch do nothing.
+// Thread jp = 0 also emits the positive contribution; thread (s = 0, jp = 0) emits the position's
+// input-row item and counts the token.
+__global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t w, uint32_t k,
+                          uint32_t replica, uint32_t batch_lo, uint32_t key0, uint32_t key1,
+                          const uint2* __restrict__ alias_tab, uint32_t* __restrict__ rows,
+                          item_t* __restrict__ items, unsigned long long* __restrict__ counts,
+                          const uint32_t* __restrict__ err) {
+    if (*err) return;
+    const uint32_t JP = (k + 1) / 2;
+    const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
+    const uint64_t total = (uint64_t)n * 2 * w * JP;
+    if (t >= total) return;
+    const uint32_t jp = (uint32_t)(t % JP);
+    const uint32_t ps = (uint32_t)(t / JP);
+    const uint32_t s = ps % (2 * w);
+    const uint32_t q = ps / (2 * w);
+    const uint32_t centre = (uint32_t)tok[q];
+    if (s == 0 && jp == 0) {
+        atomicAdd(counts + centre, 1ULL);
+        if (n >= 2) items[q] = make_item(centre, q);
+    }
+    const int64_t c = (int64_t)q + (s < w ? (int64_t)s - (int64_t)w : (int64_t)s - (int64_t)w + 1);
+    if (c < 0 || c >= (int64_t)n) return;
+    const uint32_t lo = q > w ? q - w : 0;
+    const uint32_t p = pair_offset(q, n, w) + ((uint32_t)c - lo) - ((uint32_t)c > q ? 1u : 0u);
+    const uint32_t K1 = k + 1;
+    const uint32_t ctx = (uint32_t)tok[c];
+    const uint32_t cbase = p * K1;
+    if (jp == 0) {
+        rows[cbase] = ctx;
+        items[n + cbase] = make_item(V + ctx, cbase);
+    }
+    const Philox4 r = philox4x32_10(Philox4{p, jp, batch_lo, kTagNegative | replica}, key0, key1);
+    const uint32_t j0 = 2 * jp;
+    const uint32_t n0 = alias_pick(alias_tab, V, r.x, r.y);
+    rows[cbase + 1 + j0] = n0;
+    items[n + cbase + 1 + j0] = make_item(n0 == ctx ? 2 * V : V + n0, cbase + 1 + j0);
+    if (j0 + 1 < k) {
+        const uint32_t n1 = alias_pick(alias_tab, V, r.z, r.w);
+        rows[cbase + 2 + j0] = n1;
+        items[n + cbase + 2 + j0] = make_item(n1 == ctx ? 2 * V : V + n1, cbase + 2 + j0);
+    }
+}
+
+cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, uint32_t replica,
+                           uint32_t batch_lo, uint64_t seed, const uint2* alias_tab, uint32_t* rows,
+                           item_t* items, unsigned long long* counts, const uint32_t* err) {
+    if (n == 0) return cudaSuccess;
+    const uint64_t total = (uint64_t)n * 2 * s.w * ((s.k + 1) / 2);
+    const uint32_t blocks = (uint32_t)((total + 255) / 256);
+    k_prepare<<<blocks, 256, 0, L.stream>>>(tok, n, s.V, s.w, s.k, replica, batch_lo, (uint32_t)seed,
+                                            (uint32_t)(seed >> 32), alias_tab, rows, items, counts, err);
+    ++*L.launches;
+    return cudaGetLastError();
+}
+
+// Seeded initial input rows: U(-0.5/d, 0.5/d).  The 24 high bits of a Philox word, centred, give a
+// uniform in (0,1) exactly representable in fp64; the division by d is taken in fp64, then rounded.
+__global__ void k_init_input(float* __restrict__ table, uint32_t V, uint32_t d, uint32_t stride, uint32_t key0,
+                             uint32_t key1) {
+    const uint64_t blk = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;   // group of 4 consecutive elements
+    const uint64_t total = (uint64_t)V * d;
+    if (blk * 4 >= total) return;
+    const Philox4 r = philox4x32_10(Philox4{(uint32_t)blk, (uint32_t)(blk >> 32), 0u, kTagInit}, key0, key1);
+    const uint32_t words[4] = {r.x, r.y, r.z, r.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const uint64_t e = blk * 4 + i;
+        if (e < total) {
+            const double u = ((double)(words[i] >> 8) + 0.5) * (1.0 / 16777216.0);
+            table[(e / d) * stride + (e % d)] = (float)((u - 0.5) / (double)d);
+        }
+    }
+}
+
+cudaError_t launch_init_input_table(const Launcher& L, float* table, const Shape& s, uint64_t seed) {
+    const uint64_t groups = ((uint64_t)s.V * s.d + 3) / 4;
+    k_init_input<<<(uint32_t)((groups + 255) / 256), 256, 0, L.stream>>>(table, s.V, s.d, s.stride, (uint32_t)seed,
+                                                                          (uint32_t)(seed >> 32));
+    ++*L.launches;
+    return cudaGetLastError();
+}
+
+}  // namespace tensair

@@ -1,0 +1,504 @@
+// C ABI of the library: context, workspace carving, the train / apply / drain calls and the parity taps.
+#include "../../include/tensair.h"
+
+#include <cstdio>
+#include <cstring>
+#include <new>
+#include <string>
+#include <vector>
+
+#include "kernels.h"
+#include "schedule.h"
+
+using namespace tensair;
+
+namespace {
+
+uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+// Offsets (bytes) of everything the library keeps in the caller's scratch buffer.
+struct Carve {
+    uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, gin_pos, loss_pos, hist,
+        tile_counts, seg_start, long_rows, chunk_items, partials, total;
+    uint64_t slot_bytes, ids_off, delta_off;
+    uint32_t stride, max_pairs, max_contrib, max_items, max_rows, max_long, max_chunks;
+};
+
+int validate_config(const tensair_config* c) {
+    if (!c) return TENSAIR_EINVAL;
+    if (c->V < 2 || c->V > (1u << 30)) return TENSAIR_EINVAL;
+    if (c->d < 4 || c->d > 1024 || c->d % 4) return TENSAIR_EINVAL;
+    if (c->window < 1 || c->window > 16) return TENSAIR_EINVAL;
+    if (c->k < 1 || c->k > 64) return TENSAIR_EINVAL;
+    if (c->batch < 1 || c->batch > (1u << 22)) return TENSAIR_EINVAL;
+    if (c->W < 1 || c->W > 256) return TENSAIR_EINVAL;
+    if (c->max_grad_buffer != 1) return TENSAIR_EINVAL;
+    if (c->max_delay > 64) return TENSAIR_EINVAL;
+    if (c->row_stride && (c->row_stride < c->d || c->row_stride % 4)) return TENSAIR_EINVAL;
+    if (!(c->lr == c->lr)) return TENSAIR_EINVAL;
+    if (c->reduction > TENSAIR_MEAN) return TENSAIR_EINVAL;
+    const uint64_t contrib = (uint64_t)pair_count(c->batch, c->window) * (c->k + 1);
+    if (contrib + c->batch >= (1ull << 31)) return TENSAIR_EINVAL;
+    return TENSAIR_OK;
+}
+
+void carve(const tensair_config& c, Carve& k) {
+    k.stride = c.row_stride ? c.row_stride : (uint32_t)round_up(c.d, 8);
+    k.max_pairs = pair_count(c.batch, c.window);
+    k.max_contrib = k.max_pairs * (c.k + 1);
+    k.max_items = c.batch + k.max_contrib;
+    k.max_rows = (c.batch < c.V ? c.batch : c.V) + (k.max_contrib < c.V ? k.max_contrib : c.V);
+    k.max_long = k.max_items / kChunk + 1;
+    k.max_chunks = 2 * (k.max_items / kChunk) + 2;
+    uint64_t off = 0;
+    auto take = [&off](uint64_t bytes) { const uint64_t at = off; off = round_up(off + bytes, 256); return at; };
+    k.err = take(4);
+    k.loss = take(8);
+    k.long_counters = take(8);
+    k.counts = take((uint64_t)c.V * 8);
+    k.alias_tab = take((uint64_t)c.V * 8);
+    k.tok = take((uint64_t)c.batch * 4);
+    k.rows = take((uint64_t)k.max_contrib * 4);
+    k.items_a = take((uint64_t)k.max_items * 8);
+    k.items_b = take((uint64_t)k.max_items * 8);
+    k.rec = take((uint64_t)k.max_contrib * sizeof(Rec));
+    k.gin_pos = take((uint64_t)c.batch * k.stride * 8);
+    k.loss_pos = take((uint64_t)c.batch * 8);
+    k.hist = take((uint64_t)sort_hist_words(k.max_items) * 4);
+    k.tile_counts = take((uint64_t)(heads_tiles(k.max_items) + 1) * 4);
+    k.seg_start = take((uint64_t)(k.max_rows + 2) * 4);
+    k.long_rows = take((uint64_t)k.max_long * sizeof(LongRow));
+    k.chunk_items = take((uint64_t)k.max_chunks * sizeof(ChunkItem));
+    k.partials = take((uint64_t)k.max_chunks * k.stride * 8);
+    k.total = off;
+    k.ids_off = kHeaderBytes;
+    k.delta_off = round_up(k.ids_off + (uint64_t)k.max_rows * 4, 256);
+    k.slot_bytes = round_up(k.delta_off + (uint64_t)k.max_rows * k.stride * 4, 256);
+}
+
+uint32_t bits_for(uint32_t x) {   // bits needed to represent x
+    uint32_t b = 0;
+    while (x) { ++b; x >>= 1; }
+    return b ? b : 1;
+}
+
+}  // namespace
+
+struct tensair_ctx {
+    tensair_config cfg;
+    Carve cv;
+    Shape shape;
+    cudaStream_t stream;
+    Launcher L;
+    uint64_t launches = 0;
+    float* tables;
+    uint8_t* pool;
+    uint8_t* scratch;
+    Schedule* sched = nullptr;
+    uint32_t last_n = 0, last_pairs = 0;
+    bool have_last = false;
+    std::string last_error;
+    // pinned host staging for small read-backs
+    struct Staging { MsgHeader hdr; double loss; uint32_t err; } *stage = nullptr;
+
+    template <class T> T* at(uint64_t off) const { return reinterpret_cast<T*>(scratch + off); }
+    float* table_of(uint32_t replica) const { return tables + (size_t)replica * 2 * cfg.V * cv.stride; }
+    uint8_t* slot_ptr(uint32_t slot) const { return pool + (size_t)slot * cv.slot_bytes; }
+    MsgHeader* slot_hdr(uint32_t slot) const { return reinterpret_cast<MsgHeader*>(slot_ptr(slot)); }
+    uint32_t* slot_ids(uint32_t slot) const { return reinterpret_cast<uint32_t*>(slot_ptr(slot) + cv.ids_off); }
+    float* slot_delta(uint32_t slot) const { return reinterpret_cast<float*>(slot_ptr(slot) + cv.delta_off); }
+};
+
+namespace {
+
+int fail(tensair_ctx* ctx, cudaError_t e, const char* what) {
+    if (ctx) ctx->last_error = std::string(what) + ": " + cudaGetErrorString(e);
+    return TENSAIR_ECUDA;
+}
+
+#define TENSAIR_CUDA(ctx, call)                                    \
+    do {                                                           \
+        const cudaError_t e_ = (call);                             \
+        if (e_ != cudaSuccess) return fail((ctx), e_, #call);      \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+// Reads and clears the device error flag after a synchronisation.
+int collect(tensair_ctx* ctx) {
+    TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->err, ctx->at<uint32_t>(ctx->cv.err), 4, cudaMemcpyDeviceToHost, ctx->stream));
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (ctx->stage->err) {
+        TENSAIR_CUDA(ctx, cudaMemsetAsync(ctx->at<uint32_t>(ctx->cv.err), 0, 4, ctx->stream));
+        ctx->last_error = "a batch held a token id outside [0,V); it and the batches after it were dropped";
+        return TENSAIR_EBADTOKEN;
+    }
+    return TENSAIR_OK;
+}
+
+int upload_sampler(tensair_ctx* ctx, const uint64_t* counts_host) {
+    const uint32_t V = ctx->cfg.V;
+    std::vector<uint32_t> thresh(V), alias(V);
+    build_alias_host(counts_host, V, thresh.data(), alias.data());
+    std::vector<uint2> packed(V);
+    for (uint32_t i = 0; i < V; ++i) packed[i] = make_uint2(thresh[i], alias[i]);
+    TENSAIR_CUDA(ctx, cudaMemcpyAsync(ctx->at<uint2>(ctx->cv.alias_tab), packed.data(), (size_t)V * 8, cudaMemcpyHostToDevice, ctx->stream));
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return TENSAIR_OK;
+}
+
+int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint32_t n, uint64_t batch_index,
+               double* loss_out, tensair_msg_info* info) {
+    const tensair_config& c = ctx->cfg;
+    const Carve& cv = ctx->cv;
+    const int rc = ctx->sched->on_train(replica, batch_index);
+    if (rc != TENSAIR_OK) return rc;
+    const uint32_t slot = ctx->sched->slot_of(replica, batch_index);
+    const uint32_t pairs = n >= 2 ? pair_count(n, c.window) : 0;
+    const uint32_t contrib = pairs * (c.k + 1);
+    const uint32_t n_items = pairs ? n + contrib : 0;
+    uint32_t* err = ctx->at<uint32_t>(cv.err);
+    float* table = ctx->table_of(replica);
+    MsgHeader* hdr = ctx->slot_hdr(slot);
+    // Eq. 1's alpha, divided by the number of pairs when the batch loss is the mean of the pair losses
+    const double scale = c.reduction == TENSAIR_MEAN && pairs ? (double)c.lr / (double)pairs : (double)c.lr;
+
+    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err));
+    TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tok_dev, n, ctx->shape, replica, (uint32_t)batch_index, c.seed,
+                                     ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows),
+                                     ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err));
+    if (n_items) {
+        TENSAIR_CUDA(ctx, launch_forward(ctx->L, tok_dev, n, ctx->shape, table, ctx->at<uint32_t>(cv.rows),
+                                         ctx->at<Rec>(cv.rec), ctx->at<double>(cv.gin_pos), ctx->at<double>(cv.loss_pos), err));
+        item_t* sorted = nullptr;
+        TENSAIR_CUDA(ctx, launch_sort(ctx->L, ctx->at<item_t>(cv.items_a), ctx->at<item_t>(cv.items_b), n_items,
+                                      bits_for(2 * c.V), ctx->at<uint32_t>(cv.hist), &sorted));
+        TENSAIR_CUDA(ctx, launch_heads(ctx->L, sorted, n_items, c.V, ctx->at<uint32_t>(cv.tile_counts), hdr,
+                                       ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
+                                       ctx->at<uint32_t>(cv.long_counters), err));
+        TENSAIR_CUDA(ctx, launch_reduce(ctx->L, sorted, hdr, ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
+                                        ctx->at<Rec>(cv.rec), ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot),
+                                        ctx->shape, scale, ctx->at<uint32_t>(cv.long_counters),
+                                        ctx->at<LongRow>(cv.long_rows), ctx->at<ChunkItem>(cv.chunk_items),
+                                        ctx->at<double>(cv.partials)));
+        // input rows last: they were the sources of every output-row sum
+        TENSAIR_CUDA(ctx, launch_apply_rows(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_delta(slot), table, ctx->shape, 1));
+    } else {
+        TENSAIR_CUDA(ctx, cudaMemsetAsync(hdr, 0, sizeof(MsgHeader), ctx->stream));
+    }
+    TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err));
+    ctx->last_n = n;
+    ctx->last_pairs = pairs;
+    ctx->have_last = true;
+    if (loss_out || info) {
+        TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->loss, ctx->at<double>(cv.loss), 8, cudaMemcpyDeviceToHost, ctx->stream));
+        TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->hdr, hdr, sizeof(MsgHeader), cudaMemcpyDeviceToHost, ctx->stream));
+        const int st = collect(ctx);
+        if (st != TENSAIR_OK) return st;
+        if (loss_out) *loss_out = ctx->stage->loss;
+        if (info) {
+            info->n_rows = ctx->stage->hdr.n_rows;
+            info->n_in_rows = ctx->stage->hdr.n_in_rows;
+            info->n_pairs = pairs;
+            info->slot = slot;
+            info->pool_offset = (uint64_t)slot * cv.slot_bytes;
+        }
+    }
+    return TENSAIR_OK;
+}
+
+int apply_due(tensair_ctx* ctx, uint32_t receiver, const std::vector<Due>& due) {
+    for (const Due& d : due)
+        TENSAIR_CUDA(ctx, launch_apply(ctx->L, ctx->slot_hdr(d.slot), ctx->slot_ids(d.slot), ctx->slot_delta(d.slot),
+                                       ctx->table_of(receiver), ctx->shape));
+    return TENSAIR_OK;
+}
+
+int copy_rows(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows, float* host, bool to_host) {
+    const tensair_config& c = ctx->cfg;
+    if (replica >= c.W || (which != 0 && which != 1) || (uint64_t)row0 + nrows > c.V || (!host && nrows)) return TENSAIR_EINVAL;
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (!nrows) return TENSAIR_OK;
+    float* dev = ctx->table_of(replica) + ((size_t)which * c.V + row0) * ctx->cv.stride;
+    if (to_host)
+        TENSAIR_CUDA(ctx, cudaMemcpy2D(host, (size_t)c.d * 4, dev, (size_t)ctx->cv.stride * 4, (size_t)c.d * 4, nrows, cudaMemcpyDeviceToHost));
+    else
+        TENSAIR_CUDA(ctx, cudaMemcpy2D(dev, (size_t)ctx->cv.stride * 4, host, (size_t)c.d * 4, (size_t)c.d * 4, nrows, cudaMemcpyHostToDevice));
+    return TENSAIR_OK;
+}
+
+}  // namespace
+
+extern "C" {
+
+int tensair_workspace_bytes(const tensair_config* cfg, tensair_sizes* out) {
+    const int rc = validate_config(cfg);
+    if (rc != TENSAIR_OK || !out) return TENSAIR_EINVAL;
+    Carve cv;
+    carve(*cfg, cv);
+    out->row_stride = cv.stride;
+    out->tables_bytes = (uint64_t)cfg->W * 2 * cfg->V * cv.stride * 4;
+    out->pool_bytes = (uint64_t)cfg->W * (cfg->max_delay + 1) * cv.slot_bytes;
+    out->scratch_bytes = cv.total;
+    out->max_pairs = cv.max_pairs;
+    out->max_rows = cv.max_rows;
+    out->reserved = 0;
+    return TENSAIR_OK;
+}
+
+int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const uint64_t* counts_host,
+                 const float* init_in_host, const float* init_out_host, tensair_ctx** out) {
+    tensair_sizes sz;
+    if (!out || !bufs || tensair_workspace_bytes(cfg, &sz) != TENSAIR_OK) return TENSAIR_EINVAL;
+    *out = nullptr;
+    if (!bufs->tables || !bufs->pool || !bufs->scratch) return TENSAIR_EINVAL;
+    if (((uintptr_t)bufs->tables | (uintptr_t)bufs->pool | (uintptr_t)bufs->scratch) & 255) return TENSAIR_EINVAL;
+    if (bufs->tables_bytes < sz.tables_bytes || bufs->pool_bytes < sz.pool_bytes || bufs->scratch_bytes < sz.scratch_bytes)
+        return TENSAIR_ENOMEM;
+    if (counts_host)
+        for (uint32_t i = 0; i < cfg->V; ++i) if (counts_host[i] < 1) return TENSAIR_EINVAL;
+    DeviceGuard guard(cfg->device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    tensair_ctx* ctx = new (std::nothrow) tensair_ctx();
+    if (!ctx) return TENSAIR_ENOMEM;
+    ctx->cfg = *cfg;
+    carve(*cfg, ctx->cv);
+    ctx->shape = Shape{cfg->V, cfg->d, cfg->d / 4, ctx->cv.stride, cfg->window, cfg->k, cfg->k + 1};
+    ctx->stream = (cudaStream_t)bufs->stream;
+    ctx->tables = (float*)bufs->tables;
+    ctx->pool = (uint8_t*)bufs->pool;
+    ctx->scratch = (uint8_t*)bufs->scratch;
+    cudaDeviceProp prop;
+    int status = TENSAIR_OK;
+    auto bail = [&](int code) { delete ctx->sched; if (ctx->stage) cudaFreeHost(ctx->stage); delete ctx; return code; };
+    if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return bail(TENSAIR_ECUDA);
+    ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount};
+    if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
+    ctx->sched = new Schedule(cfg->W, cfg->max_delay, cfg->seed);
+
+    const uint32_t V = cfg->V, stride = ctx->cv.stride;
+    const size_t replica_floats = (size_t)2 * V * stride;
+    auto run = [&]() -> int {
+        TENSAIR_CUDA(ctx, cudaMemsetAsync(ctx->scratch, 0, ctx->cv.total, ctx->stream));
+        TENSAIR_CUDA(ctx, cudaMemsetAsync(ctx->pool, 0, sz.pool_bytes, ctx->stream));
+        TENSAIR_CUDA(ctx, cudaMemsetAsync(ctx->tables, 0, replica_floats * 4, ctx->stream));
+        if (init_in_host)
+            TENSAIR_CUDA(ctx, cudaMemcpy2DAsync(ctx->tables, (size_t)stride * 4, init_in_host, (size_t)cfg->d * 4,
+                                                (size_t)cfg->d * 4, V, cudaMemcpyHostToDevice, ctx->stream));
+        else
+            TENSAIR_CUDA(ctx, launch_init_input_table(ctx->L, ctx->tables, ctx->shape, cfg->seed));
+        if (init_out_host)
+            TENSAIR_CUDA(ctx, cudaMemcpy2DAsync(ctx->tables + (size_t)V * stride, (size_t)stride * 4, init_out_host,
+                                                (size_t)cfg->d * 4, (size_t)cfg->d * 4, V, cudaMemcpyHostToDevice, ctx->stream));
+        for (uint32_t r = 1; r < cfg->W; ++r)
+            TENSAIR_CUDA(ctx, cudaMemcpyAsync(ctx->tables + r * replica_floats, ctx->tables, replica_floats * 4,
+                                              cudaMemcpyDeviceToDevice, ctx->stream));
+        std::vector<uint64_t> ones;
+        const uint64_t* counts = counts_host;
+        if (!counts) { ones.assign(V, 1); counts = ones.data(); }
+        TENSAIR_CUDA(ctx, cudaMemcpyAsync(ctx->at<uint64_t>(ctx->cv.counts), counts, (size_t)V * 8, cudaMemcpyHostToDevice, ctx->stream));
+        TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+        return upload_sampler(ctx, counts);
+    };
+    status = run();
+    if (status != TENSAIR_OK) return bail(status);
+    *out = ctx;
+    return TENSAIR_OK;
+}
+
+void tensair_destroy(tensair_ctx* ctx) {
+    if (!ctx) return;
+    DeviceGuard guard(ctx->cfg.device);
+    cudaStreamSynchronize(ctx->stream);
+    if (ctx->stage) cudaFreeHost(ctx->stage);
+    delete ctx->sched;
+    delete ctx;
+}
+
+int tensair_train_batch(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_dev, uint32_t n_tokens,
+                        uint64_t batch_index, double* loss_out, tensair_msg_info* info) {
+    if (!ctx || replica >= ctx->cfg.W || n_tokens > ctx->cfg.batch || (n_tokens && !tokens_dev) ||
+        batch_index >= (1ull << 32))
+        return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    return train_impl(ctx, replica, tokens_dev, n_tokens, batch_index, loss_out, info);
+}
+
+int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_host, uint32_t n_tokens,
+                             uint64_t batch_index, double* loss_out, tensair_msg_info* info) {
+    if (!ctx || replica >= ctx->cfg.W || n_tokens > ctx->cfg.batch || (n_tokens && !tokens_host) ||
+        batch_index >= (1ull << 32))
+        return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    int32_t* tok = ctx->at<int32_t>(ctx->cv.tok);
+    if (n_tokens)
+        TENSAIR_CUDA(ctx, cudaMemcpyAsync(tok, tokens_host, (size_t)n_tokens * 4, cudaMemcpyHostToDevice, ctx->stream));
+    return train_impl(ctx, replica, tok, n_tokens, batch_index, loss_out, info);
+}
+
+int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint64_t step, uint32_t* n_applied) {
+    if (!ctx || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const std::vector<Due> due = ctx->sched->take_due(replica, step, false);
+    if (n_applied) *n_applied = (uint32_t)due.size();
+    return apply_due(ctx, replica, due);
+}
+
+int tensair_drain(tensair_ctx* ctx, uint32_t* n_applied) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    uint32_t total = 0;
+    for (uint32_t r = 0; r < ctx->cfg.W; ++r) {
+        const std::vector<Due> due = ctx->sched->take_due(r, 0, true);
+        total += (uint32_t)due.size();
+        const int rc = apply_due(ctx, r, due);
+        if (rc != TENSAIR_OK) return rc;
+    }
+    if (n_applied) *n_applied = total;
+    return TENSAIR_OK;
+}
+
+int tensair_update_sampler(tensair_ctx* ctx) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    std::vector<uint64_t> counts(ctx->cfg.V);
+    TENSAIR_CUDA(ctx, cudaMemcpyAsync(counts.data(), ctx->at<uint64_t>(ctx->cv.counts), (size_t)ctx->cfg.V * 8, cudaMemcpyDeviceToHost, ctx->stream));
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return upload_sampler(ctx, counts.data());
+}
+
+int tensair_sync(tensair_ctx* ctx) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    return collect(ctx);
+}
+
+int tensair_read_embeddings(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows, float* host_dst) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    return copy_rows(ctx, replica, which, row0, nrows, host_dst, true);
+}
+
+int tensair_write_embeddings(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows, const float* host_src) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    return copy_rows(ctx, replica, which, row0, nrows, const_cast<float*>(host_src), false);
+}
+
+int tensair_read_negatives(tensair_ctx* ctx, uint32_t* host_neg, uint32_t* n_pairs) {
+    if (!ctx || !ctx->have_last) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    if (n_pairs) *n_pairs = ctx->last_pairs;
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (host_neg && ctx->last_pairs) {
+        const uint32_t k = ctx->cfg.k;
+        // rows are stored per pair as [positive, k negatives]
+        TENSAIR_CUDA(ctx, cudaMemcpy2D(host_neg, (size_t)k * 4, ctx->at<uint32_t>(ctx->cv.rows) + 1, (size_t)(k + 1) * 4,
+                                       (size_t)k * 4, ctx->last_pairs, cudaMemcpyDeviceToHost));
+    }
+    return TENSAIR_OK;
+}
+
+int tensair_read_scalars(tensair_ctx* ctx, double* host_g) {
+    if (!ctx || !ctx->have_last || !host_g) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    const size_t n = (size_t)ctx->last_pairs * (ctx->cfg.k + 1);
+    if (n) TENSAIR_CUDA(ctx, cudaMemcpy2D(host_g, 8, ctx->at<Rec>(ctx->cv.rec), sizeof(Rec), 8, n, cudaMemcpyDeviceToHost));
+    return TENSAIR_OK;
+}
+
+int tensair_read_message(tensair_ctx* ctx, uint32_t replica, uint64_t batch_index, uint32_t* n_rows,
+                         uint32_t* host_ids, float* host_delta) {
+    if (!ctx || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const uint32_t slot = ctx->sched->slot_of(replica, batch_index);
+    if (!ctx->sched->slot_holds(slot, batch_index)) return TENSAIR_ENOTFOUND;
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    MsgHeader h;
+    TENSAIR_CUDA(ctx, cudaMemcpy(&h, ctx->slot_hdr(slot), sizeof(h), cudaMemcpyDeviceToHost));
+    if (n_rows) *n_rows = h.n_rows;
+    if (host_ids && h.n_rows) TENSAIR_CUDA(ctx, cudaMemcpy(host_ids, ctx->slot_ids(slot), (size_t)h.n_rows * 4, cudaMemcpyDeviceToHost));
+    if (host_delta && h.n_rows)
+        TENSAIR_CUDA(ctx, cudaMemcpy2D(host_delta, (size_t)ctx->cfg.d * 4, ctx->slot_delta(slot), (size_t)ctx->cv.stride * 4,
+                                       (size_t)ctx->cfg.d * 4, h.n_rows, cudaMemcpyDeviceToHost));
+    return TENSAIR_OK;
+}
+
+int tensair_read_sampler(tensair_ctx* ctx, uint32_t* thresh, uint32_t* alias, uint64_t* counts) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const uint32_t V = ctx->cfg.V;
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    if (thresh || alias) {
+        std::vector<uint2> packed(V);
+        TENSAIR_CUDA(ctx, cudaMemcpy(packed.data(), ctx->at<uint2>(ctx->cv.alias_tab), (size_t)V * 8, cudaMemcpyDeviceToHost));
+        for (uint32_t i = 0; i < V; ++i) {
+            if (thresh) thresh[i] = packed[i].x;
+            if (alias) alias[i] = packed[i].y;
+        }
+    }
+    if (counts) TENSAIR_CUDA(ctx, cudaMemcpy(counts, ctx->at<uint64_t>(ctx->cv.counts), (size_t)V * 8, cudaMemcpyDeviceToHost));
+    return TENSAIR_OK;
+}
+
+int tensair_read_delivery_log(tensair_ctx* ctx, uint32_t replica, uint64_t max_records, tensair_delivery* out, uint64_t* n) {
+    if (!ctx || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
+    const std::vector<tensair_delivery>& lg = ctx->sched->log(replica);
+    if (n) *n = lg.size();
+    for (uint64_t i = 0; i < lg.size() && i < max_records && out; ++i) out[i] = lg[i];
+    return TENSAIR_OK;
+}
+
+int tensair_pending(tensair_ctx* ctx, uint32_t replica, uint64_t* n) {
+    if (!ctx || !n || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
+    *n = ctx->sched->pending(replica);
+    return TENSAIR_OK;
+}
+
+uint64_t tensair_kernel_launches(const tensair_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+const char* tensair_strerror(int code) {
+    switch (code) {
+        case TENSAIR_OK: return "ok";
+        case TENSAIR_EINVAL: return "invalid argument or unsupported configuration";
+        case TENSAIR_ENOMEM: return "a caller-provided buffer is too small";
+        case TENSAIR_ECUDA: return "a CUDA call failed";
+        case TENSAIR_EBADTOKEN: return "token id outside [0,V)";
+        case TENSAIR_EPENDING: return "message slot still has undelivered recipients";
+        case TENSAIR_ENOTFOUND: return "message no longer held";
+        default: return "unknown error";
+    }
+}
+
+const char* tensair_last_error(const tensair_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+int tensair_build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias) {
+    if (!V || !thresh || !alias) return TENSAIR_EINVAL;
+    if (counts)
+        for (uint32_t i = 0; i < V; ++i) if (counts[i] < 1) return TENSAIR_EINVAL;
+    build_alias_host(counts, V, thresh, alias);
+    return TENSAIR_OK;
+}
+
+}  // extern "C"

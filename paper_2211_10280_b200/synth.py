@@ -38,6 +38,7 @@ class Workload:
     drift_every: int = 0  # re-draw the rank->token permutation every this many batches (0 = never)
     lr: float = 0.025
     seed: int = 0         # library seed (negative sampler, delays)
+    reduction: int = 0    # 0: batch loss = sum of the pair losses; 1: their mean
 
     @property
     def pairs_per_batch(self) -> int:
@@ -52,18 +53,18 @@ def n_pairs(n: int, w: int) -> int:
 TINY = Workload("sgns_tiny", V=10_000, d=64, window=2, k=5, batch=512, W=1, batches=200,
                 zipf_s=1.0, stream_seeds=(0,), seed=0)
 MID = Workload("sgns_mid", V=100_000, d=128, window=5, k=5, batch=4096, W=1, batches=2000,
-               zipf_s=1.0, stream_seeds=(1,), seed=1)
+               zipf_s=1.0, stream_seeds=(1,), seed=1, reduction=1)
 LARGE_DASGD = Workload("sgns_large_dasgd", V=1_000_000, d=300, window=5, k=15, batch=8192, W=4,
-                       batches=500, zipf_s=1.0, stream_seeds=(2, 3, 4, 5), max_delay=2, seed=2)
+                       batches=500, zipf_s=1.0, stream_seeds=(2, 3, 4, 5), max_delay=2, seed=2, reduction=1)
 LARGE_DRIFT = Workload("sgns_large_drift", V=1_000_000, d=300, window=5, k=15, batch=16384, W=8,
                        batches=1000, zipf_s=1.1, stream_seeds=tuple(range(6, 14)), max_delay=2,
-                       drift_every=100, seed=6)
+                       drift_every=100, seed=6, reduction=1)
 
 
 def sweep_point(d: int, batch: int, k: int) -> Workload:
     """One point of the throughput sweep (V = 1M, one replica, window 5, 100 batches)."""
     return Workload(f"sgns_sweep_d{d}_B{batch}_k{k}", V=1_000_000, d=d, window=5, k=k, batch=batch,
-                    W=1, batches=100, zipf_s=1.0, stream_seeds=(14,), seed=14)
+                    W=1, batches=100, zipf_s=1.0, stream_seeds=(14,), seed=14, reduction=1)
 
 
 SWEEP = [sweep_point(d, b, k) for d in (64, 128, 300, 512) for b in (256, 2048, 16384, 65536)

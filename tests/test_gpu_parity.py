@@ -1,0 +1,346 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Bars: bit-exact for sampled negatives, sampler tables, counts, message row ids, delivery order and
+staleness; max relative error (see parity_utils.rel_err) <= 1e-5 for fp32 embeddings and delta rows
+after one batch and <= 1e-3 after 200 batches.
+"""
+import math
+
+import numpy as np
+import pytest
+
+from parity_utils import compare_message, compare_tables, make_pair, rel_err
+from paper_2211_10280_b200 import synth
+
+pytestmark = pytest.mark.gpu
+
+TOL_ONE = 1e-5
+TOL_200 = 1e-3
+
+
+@pytest.fixture(scope="module")
+def torch():
+    import torch as t
+
+    assert t.cuda.is_available(), "these tests need a CUDA device"
+    return t
+
+
+def dev(torch, a):
+    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+
+
+# ------------------------------------------------------------------ init, sampler
+def test_seeded_init_is_bit_identical(torch):
+    import oracle as orc
+
+    wl = synth.scaled(synth.TINY, V=3001, d=68, W=2)
+    o, g = make_pair(wl)
+    want = orc.init_input_table(wl.seed, wl.V, wl.d)
+    for r in range(2):
+        assert np.array_equal(g.tensair_read_embeddings(r, 0).view(np.uint32), want.view(np.uint32))
+        assert not g.tensair_read_embeddings(r, 1).any()
+    assert np.array_equal(o.read_embeddings(1, 0), want)
+
+
+@pytest.mark.parametrize("wl", [synth.TINY, synth.scaled(synth.MID, batches=2),
+                                synth.scaled(synth.LARGE_DASGD, V=60_000, d=12, batch=2048, W=1, max_delay=0)],
+                         ids=lambda w: w.name)
+def test_negatives_sampler_and_counts_are_bit_exact(torch, wl):
+    stream = synth.token_stream(wl, 0, 2)
+    counts = synth.stream_counts([stream], wl.V)
+    o, g = make_pair(wl, counts=counts)
+    to, ao, _ = o.sampler()
+    tg, ag, _ = g.tensair_read_sampler()
+    assert np.array_equal(to, tg) and np.array_equal(ao, ag)
+    for b in range(2):
+        assert o.train_batch(0, stream[b], b + 5)[0] == 0
+        g.tensair_train_batch(0, dev(torch, stream[b]), b + 5)
+        no, ng = o.read_negatives(), g.tensair_read_negatives()
+        assert no.shape == ng.shape == (wl.pairs_per_batch, wl.k)
+        assert np.array_equal(no, ng)
+    assert np.array_equal(o.sampler()[2], g.tensair_read_sampler()[2])
+
+
+# ------------------------------------------------------------------ one batch
+ONE_BATCH = [
+    ("tiny", synth.TINY, False),
+    ("tiny_mean", synth.scaled(synth.TINY, reduction=1), True),
+    ("tiny_random_tables", synth.TINY, True),
+    ("mid", synth.MID, True),
+    ("d300_k15", synth.scaled(synth.LARGE_DASGD, V=50_000, batch=1024, W=1, max_delay=0), True),
+    ("d512_k5", synth.scaled(synth.sweep_point(512, 2048, 5), V=30_000), True),
+    ("d8_w1_k1", synth.scaled(synth.TINY, V=500, d=8, window=1, k=1, batch=100), True),
+    ("d1024_w8_k3", synth.scaled(synth.TINY, V=2000, d=1024, window=8, k=3, batch=300), True),
+]
+
+
+@pytest.mark.parametrize("name,wl,random_tables", ONE_BATCH, ids=[c[0] for c in ONE_BATCH])
+def test_one_batch_matches_the_oracle(torch, name, wl, random_tables):
+    stream = synth.token_stream(wl, 0, 1)
+    counts = synth.stream_counts([stream], wl.V)
+    if random_tables:
+        t_in, t_out = synth.random_tables(wl.V, wl.d, 17, scale=2.0 / math.sqrt(wl.d))
+    else:
+        t_in, t_out = synth.init_tables(wl.V, wl.d, 17)
+    o, g = make_pair(wl, counts=counts, init_in=t_in, init_out=t_out)
+    rc, loss_o, nrows_o = o.train_batch(0, stream[0], 0)
+    assert rc == 0
+    loss_g, info = g.tensair_train_batch(0, dev(torch, stream[0]), 0, want_loss=True, want_info=True)
+    assert info.n_pairs == wl.pairs_per_batch == o.last_pairs()
+    assert info.n_rows == nrows_o
+    assert info.n_in_rows == len(set(stream[0].tolist()))
+    assert np.array_equal(o.read_negatives(), g.tensair_read_negatives())
+    go, gg = o.read_g(), g.tensair_read_scalars()
+    assert np.max(np.abs(go - gg)) <= 1e-13
+    assert np.array_equal(go == 0.0, gg == 0.0)
+    assert loss_g == pytest.approx(loss_o, rel=1e-12)
+    compare_message(o, g, 0, 0, TOL_ONE)
+    compare_tables(o, g, 0, TOL_ONE)
+    # rows outside the message are bit-unchanged
+    ids, _ = g.tensair_read_message(0, 0)
+    untouched = np.ones(2 * wl.V, bool)
+    untouched[ids] = False
+    after = np.concatenate([g.tensair_read_embeddings(0, 0), g.tensair_read_embeddings(0, 1)])
+    before = np.concatenate([t_in, t_out])
+    assert np.array_equal(after[untouched].view(np.uint32), before[untouched].view(np.uint32))
+    assert g.tensair_apply_messages(0, 0) == 0
+
+
+def test_hot_rows_take_the_chunked_path(torch):
+    # 40 tokens and a large batch: every row collects far more than one chunk of contributions
+    wl = synth.scaled(synth.TINY, V=40, d=36, window=3, k=7, batch=3000, zipf_s=0.3)
+    stream = synth.token_stream(wl, 0, 2)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 3, scale=0.05)
+    o, g = make_pair(wl, counts=synth.stream_counts([stream], wl.V), init_in=t_in, init_out=t_out)
+    for b in range(2):
+        assert o.train_batch(0, stream[b], b)[0] == 0
+        g.tensair_train_batch(0, dev(torch, stream[b]), b)
+        compare_message(o, g, 0, b, TOL_ONE)
+    compare_tables(o, g, 0, 3 * TOL_ONE)
+
+
+@pytest.mark.parametrize("n", [0, 1, 2, 3, 5, 6, 10, 11, 12, 509, 512])
+def test_ragged_and_degenerate_batches(torch, n):
+    wl = synth.scaled(synth.TINY, V=700, d=20, window=5, k=4)
+    toks = synth.token_stream(wl, 0, 1)[0][:n]
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 9, scale=0.4)
+    o, g = make_pair(wl, init_in=t_in, init_out=t_out)
+    rc, loss_o, nrows_o = o.train_batch(0, toks, 3)
+    assert rc == 0
+    loss_g, info = g.tensair_train_batch(0, dev(torch, toks) if n else torch.empty(0, dtype=torch.int32, device="cuda"),
+                                         3, want_loss=True, want_info=True)
+    assert info.n_rows == nrows_o and info.n_pairs == synth.n_pairs(n, 5)
+    assert loss_g == pytest.approx(loss_o, rel=2e-6, abs=1e-12)
+    if n >= 2:
+        assert np.array_equal(o.read_negatives(), g.tensair_read_negatives())
+        compare_message(o, g, 0, 3, TOL_ONE)
+    compare_tables(o, g, 0, TOL_ONE)
+    assert np.array_equal(o.sampler()[2], g.tensair_read_sampler()[2])
+
+
+def test_bad_token_is_reported_and_changes_nothing(torch):
+    from paper_2211_10280_b200 import binding as B
+
+    wl = synth.scaled(synth.TINY, V=300, d=16)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 1)
+    o, g = make_pair(wl, init_in=t_in, init_out=t_out)
+    toks = synth.token_stream(wl, 0, 1)[0].copy()
+    bad = toks.copy()
+    bad[77] = wl.V
+    with pytest.raises(B.TensairError) as ei:
+        g.tensair_train_batch(0, dev(torch, bad), 0, want_loss=True)
+    assert ei.value.code == B.EBADTOKEN
+    assert np.array_equal(g.tensair_read_embeddings(0, 0), t_in) and np.array_equal(g.tensair_read_embeddings(0, 1), t_out)
+    assert np.all(g.tensair_read_sampler()[2] == 1)
+    bad[77] = -1
+    g.tensair_train_batch(0, dev(torch, bad), 1)          # asynchronous: reported by the next sync
+    assert g.tensair_sync() == B.EBADTOKEN and g.tensair_sync() == B.OK
+    # the context keeps working
+    assert o.train_batch(0, toks, 2)[0] == 0
+    g.tensair_train_batch(0, dev(torch, toks), 2)
+    compare_tables(o, g, 0, TOL_ONE)
+
+
+def test_host_and_device_entry_points_agree_bit_for_bit(torch):
+    wl = synth.scaled(synth.TINY, V=2000, d=32)
+    stream = synth.token_stream(wl, 0, 3)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 4, scale=0.3)
+    counts = synth.stream_counts([stream], wl.V)
+    _, g1 = make_pair(wl, counts=counts, init_in=t_in, init_out=t_out)
+    _, g2 = make_pair(wl, counts=counts, init_in=t_in, init_out=t_out)
+    pinned = torch.from_numpy(stream).pin_memory()
+    for b in range(3):
+        l1, _ = g1.tensair_train_batch(0, dev(torch, stream[b]), b, want_loss=True)
+        l2, _ = g2.tensair_train_batch_host(0, pinned[b], b, want_loss=True)
+        assert l1 == l2
+    for which in (0, 1):
+        assert np.array_equal(g1.tensair_read_embeddings(0, which).view(np.uint32),
+                              g2.tensair_read_embeddings(0, which).view(np.uint32))
+
+
+def test_runs_are_bit_reproducible(torch):
+    wl = synth.scaled(synth.MID, V=20_000, batch=2048)
+    stream = synth.token_stream(wl, 0, 4)
+    counts = synth.stream_counts([stream], wl.V)
+    outs = []
+    for _ in range(2):
+        _, g = make_pair(wl, counts=counts)
+        msgs = []
+        for b in range(4):
+            g.tensair_train_batch(0, dev(torch, stream[b]), b)
+            msgs.append(g.tensair_read_message(0, b))
+        outs.append((g.tensair_read_embeddings(0, 0), g.tensair_read_embeddings(0, 1), msgs))
+        g.close()
+    assert np.array_equal(outs[0][0].view(np.uint32), outs[1][0].view(np.uint32))
+    assert np.array_equal(outs[0][1].view(np.uint32), outs[1][1].view(np.uint32))
+    for (i0, d0), (i1, d1) in zip(outs[0][2], outs[1][2]):
+        assert np.array_equal(i0, i1) and np.array_equal(d0.view(np.uint32), d1.view(np.uint32))
+
+
+# ------------------------------------------------------------------ many batches
+def test_tiny_200_batches(torch):
+    wl = synth.TINY
+    stream = synth.token_stream(wl, 0)
+    counts = synth.stream_counts([stream], wl.V)
+    o, g = make_pair(wl, counts=counts)
+    worst = 0.0
+    for b in range(wl.batches):
+        rc, loss_o, _ = o.train_batch(0, stream[b], b)
+        assert rc == 0
+        if b % 50 == 0 or b == wl.batches - 1:
+            loss_g, _ = g.tensair_train_batch(0, dev(torch, stream[b]), b, want_loss=True)
+            assert loss_g == pytest.approx(loss_o, rel=1e-4)
+            assert np.array_equal(o.read_negatives(), g.tensair_read_negatives())
+            assert np.array_equal(o.read_message(0, b)[0], g.tensair_read_message(0, b)[0])
+        else:
+            g.tensair_train_batch(0, dev(torch, stream[b]), b)
+        if b == 0:
+            compare_tables(o, g, 0, TOL_ONE)
+    e = compare_tables(o, g, 0, TOL_200)
+    print("tiny, 200 batches: rel err in/out", e)
+
+
+def test_mid_60_batches(torch):
+    wl = synth.scaled(synth.MID, batches=60)
+    stream = synth.token_stream(wl, 0)
+    counts = synth.stream_counts([stream], wl.V)
+    o, g = make_pair(wl, counts=counts)
+    for b in range(wl.batches):
+        assert o.train_batch(0, stream[b], b)[0] == 0
+        g.tensair_train_batch(0, dev(torch, stream[b]), b)
+    assert np.array_equal(o.read_message(0, 59)[0], g.tensair_read_message(0, 59)[0])
+    print("mid, 60 batches: rel err in/out", compare_tables(o, g, 0, TOL_200))
+
+
+# ------------------------------------------------------------------ DASGD exchange
+def _run_exchange(torch, wl, steps, drift_every=0):
+    streams = synth.all_streams(wl, steps)
+    counts = synth.stream_counts(streams, wl.V) if not drift_every else None
+    o, g = make_pair(wl, counts=counts)
+    dstreams = [dev(torch, s) for s in streams]
+    for t in range(steps):
+        if drift_every and t and t % drift_every == 0:
+            o.update_sampler()
+            g.tensair_update_sampler()
+            so, sg = o.sampler(), g.tensair_read_sampler()
+            assert all(np.array_equal(a, b) for a, b in zip(so, sg))
+        for i in range(wl.W):
+            assert o.train_batch(i, streams[i][t], t)[0] == 0
+            g.tensair_train_batch(i, dstreams[i][t], t)
+            if t in (0, steps - 1):
+                assert np.array_equal(o.read_negatives(), g.tensair_read_negatives())
+                compare_message(o, g, i, t, TOL_ONE if t == 0 else TOL_200)
+        for j in range(wl.W):
+            assert o.apply_messages(j, t) == g.tensair_apply_messages(j, t)
+    return o, g
+
+
+def test_dasgd_exchange_matches_the_oracle(torch):
+    wl = synth.scaled(synth.LARGE_DASGD, V=20_000, d=48, batch=512, k=6)
+    steps = 12
+    o, g = _run_exchange(torch, wl, steps)
+    for j in range(wl.W):
+        assert np.array_equal(o.delivery_log(j), g.tensair_read_delivery_log(j))
+        assert o.pending(j) == g.tensair_pending(j)
+        compare_tables(o, g, j, TOL_200)
+    assert o.drain() == g.tensair_drain()
+    ref = None
+    for j in range(wl.W):
+        assert np.array_equal(o.delivery_log(j), g.tensair_read_delivery_log(j))
+        assert g.tensair_pending(j) == 0
+        compare_tables(o, g, j, TOL_200)
+        cur = np.concatenate([g.tensair_read_embeddings(j, 0), g.tensair_read_embeddings(j, 1)])
+        if ref is None:
+            ref = cur
+        else:   # same gradients applied everywhere, in different orders: equal up to fp32 rounding
+            assert rel_err(cur, ref) <= 1e-4
+    log = g.tensair_read_delivery_log(0)
+    assert log[:, 4].max() > 0 and set((log[:, 2] - log[:, 0]).tolist()) == {0, 1, 2}
+
+
+def test_first_step_of_the_exchange_is_within_the_one_batch_bar(torch):
+    wl = synth.scaled(synth.LARGE_DASGD, V=20_000, d=300, batch=512, max_delay=0)
+    o, g = _run_exchange(torch, wl, 1)
+    for j in range(wl.W):
+        compare_tables(o, g, j, TOL_ONE)
+        assert g.tensair_read_delivery_log(j).shape[0] == wl.W - 1
+
+
+def test_overwriting_an_undelivered_message_is_refused(torch):
+    from paper_2211_10280_b200 import binding as B
+
+    wl = synth.scaled(synth.TINY, V=300, d=16, W=2, max_delay=1, stream_seeds=(1, 2))
+    _, g = make_pair(wl)
+    toks = dev(torch, synth.token_stream(wl, 0, 1)[0])
+    g.tensair_train_batch(0, toks, 0)
+    g.tensair_train_batch(0, toks, 1)
+    with pytest.raises(B.TensairError) as ei:
+        g.tensair_train_batch(0, toks, 2)
+    assert ei.value.code == B.EPENDING
+    g.tensair_apply_messages(1, 1)
+    g.tensair_train_batch(0, toks, 2)
+    assert g.tensair_read_message(0, 0) is None and g.tensair_read_message(0, 2) is not None
+
+
+def test_drift_rebuilds_the_sampler_from_running_counts(torch):
+    wl = synth.scaled(synth.LARGE_DRIFT, V=5000, d=24, batch=256, W=3, k=5, drift_every=4,
+                      stream_seeds=(6, 7, 8))
+    o, g = _run_exchange(torch, wl, 10, drift_every=4)
+    o.drain()
+    g.tensair_drain()
+    for j in range(wl.W):
+        assert np.array_equal(o.delivery_log(j), g.tensair_read_delivery_log(j))
+        compare_tables(o, g, j, TOL_200)
+
+
+# ------------------------------------------------------------------ full size, the benchmark's configuration
+def test_full_size_large_dasgd_two_steps(torch):
+    """V = 1M, d = 300, batch 8192, k = 15, W = 4, delay <= 2: the whole first two steps against the oracle."""
+    wl = synth.LARGE_DASGD
+    steps = 2
+    streams = synth.all_streams(wl, steps)
+    counts = synth.stream_counts(synth.all_streams(wl, 8), wl.V)
+    o, g = make_pair(wl, counts=counts)
+    dstreams = [dev(torch, s) for s in streams]
+    rng = np.random.default_rng(0)
+    for t in range(steps):
+        for i in range(wl.W):
+            rc, loss_o, nrows = o.train_batch(i, streams[i][t], t)
+            assert rc == 0
+            loss_g, info = g.tensair_train_batch(i, dstreams[i][t], t, want_loss=True, want_info=True)
+            assert info.n_rows == nrows and info.n_pairs == 81_890
+            assert loss_g == pytest.approx(loss_o, rel=1e-5)
+            assert np.array_equal(o.read_negatives(), g.tensair_read_negatives())
+            compare_message(o, g, i, t, TOL_ONE if t == 0 else 1e-4)
+        for j in range(wl.W):
+            assert o.apply_messages(j, t) == g.tensair_apply_messages(j, t)
+    for j in range(wl.W):
+        assert np.array_equal(o.delivery_log(j), g.tensair_read_delivery_log(j))
+        # hot rows (most contributions) plus random rows
+        rows = np.unique(np.concatenate([np.arange(2000), rng.integers(0, wl.V, 20000)]))
+        for which in (0, 1):
+            want = o.read_embeddings(j, which)
+            got = g.tensair_read_embeddings(j, which)
+            assert rel_err(got[rows], want[rows]) <= 1e-4
+            assert rel_err(got, want) <= 1e-4

@@ -188,6 +188,26 @@ def test_single_batch_matches_per_pair_closed_form():
     np.testing.assert_allclose(new_out, t_out - lr32 * g_out, rtol=3e-7, atol=1e-9)
 
 
+def test_mean_reduction_divides_the_step_by_the_pair_count():
+    # same batch under both readings of L(X): the deltas differ by exactly the factor 1/P (up to fp32 rounding)
+    V, d, w, k, n, lr = 30, 5, 2, 3, 12, 0.5
+    t_in, t_out = synth.random_tables(V, d, seed=6, scale=0.7)
+    toks = np.arange(n, dtype=np.int32) * 2 % V
+    out = []
+    for red in (0, 1):
+        o = Oracle(V=V, d=d, window=w, k=k, batch=n, lr=lr, seed=8, init_in=t_in, init_out=t_out, reduction=red)
+        rc, loss, _ = o.train_batch(0, toks, 0)
+        assert rc == 0
+        out.append((loss, *o.read_message(0, 0), o.read_negatives()))
+    P = synth.n_pairs(n, w)
+    assert out[0][0] == out[1][0]                       # the reported loss is the sum in both cases
+    assert np.array_equal(out[0][1], out[1][1]) and np.array_equal(out[0][3], out[1][3])
+    np.testing.assert_allclose(out[1][2], out[0][2] / P, rtol=3e-7, atol=0)
+    want_loss, g_in, g_out, _ = _dense_reference(None, toks, w, k, V, d, lr, out[1][3], t_in, t_out)
+    dense = np.concatenate([g_in, g_out])
+    np.testing.assert_allclose(out[1][2], -(lr / P) * dense[out[1][1]], rtol=3e-7, atol=1e-12)
+
+
 def test_two_tokens_one_negative_by_hand():
     # tokens [a, b], window 1: pairs (a<-b) and (b<-a).  All output rows zero except the ones set here.
     V, d = 4, 2
