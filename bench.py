@@ -1,0 +1,373 @@
+#!/usr/bin/env python
+"""Throughput of the SGNS step plus DASGD message application, in (centre, context) pairs per second.
+
+    python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference] [--workload NAME]
+
+A "step" is one pass of the whole hot path over one batch per replica: every replica trains its
+mini-batch (gradient calculation, message build, local application, send) and then every replica
+applies the messages that are due.  The default workload is the V = 1M, d = 300, W = 4 configuration.
+
+One JSON line is printed by rank 0.  `value` is measured with the batches already in device memory;
+`e2e` is the same metric through tensair_train_batch_host with the batches in pinned host memory and
+the loss and message header read back every call.  `roofline` describes the kernel with the largest
+share of device time, timed with CUDA events inside the library in a separate pass.  `cpu_baseline`
+is the CPU oracle timed on a bounded sample of the same workload on this host's cores.
+
+`--impl reference` times the CPU oracle alone (the only "reference" there is: the paper ships no code).
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import statistics
+import subprocess
+import sys
+import threading
+import time
+from pathlib import Path
+
+import numpy as np
+
+ROOT = Path(__file__).resolve().parent
+if str(ROOT) not in sys.path:
+    sys.path.insert(0, str(ROOT))
+
+from paper_2211_10280_b200 import synth  # noqa: E402
+
+METRIC = "SGNS (center,context) pairs/sec on 1 B200; achieved HBM GB/s vs peak"
+UNIT = "pairs/s"
+FALLBACK_HBM_GBS = 6650.0
+
+
+def hbm_peak():
+    p = ROOT / "MEASURED_PEAKS.json"
+    if p.exists():
+        try:
+            return float(json.loads(p.read_text())["hbm_gbs"]), "measured"
+        except Exception:
+            pass
+    return FALLBACK_HBM_GBS, "fallback"
+
+
+class ClockSampler:
+    """Samples SM clocks and throttle reasons with nvidia-smi while the timed region runs."""
+
+    QUERY = ("clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+             "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+             "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_id: str):
+        self.rows = []
+        self.proc = None
+        self.gpu_id = gpu_id
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", "-i", self.gpu_id, f"--query-gpu={self.QUERY}",
+                                          "--format=csv,noheader,nounits", "-lms", "100"],
+                                         stdout=subprocess.PIPE, stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.rows.append((time.time(), [x.strip() for x in line.split(",")]))
+
+    def stop(self):
+        if self.proc:
+            self.proc.terminate()
+            try:
+                self.proc.wait(timeout=5)
+            except Exception:
+                self.proc.kill()
+
+    def summary(self, t0: float, t1: float):
+        rows = [r for t, r in self.rows if t0 <= t <= t1 and len(r) >= 8] or [r for _, r in self.rows if len(r) >= 8]
+        if not rows:
+            return {"sm_mhz": None, "sm_max_mhz": None, "reasons": ["nvidia-smi unavailable"]}
+        sm = [float(r[0]) for r in rows if r[0].replace(".", "").isdigit()]
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        reasons = [n for i, n in enumerate(names) if any(r[4 + i].lower() == "active" for r in rows)]
+        return {"sm_mhz": statistics.median(sm) if sm else None, "sm_max_mhz": float(rows[0][1]), "samples": len(rows),
+                "power_w_max": max(float(r[2]) for r in rows), "reasons": reasons}
+
+
+def pick_workload(name: str, override: str = "") -> synth.Workload:
+    """A named workload, optionally with fields replaced (`--override V=250000,W=2`: reduced cases for profiling)."""
+    if name not in synth.WORKLOADS:
+        raise SystemExit(f"unknown workload {name!r}; one of {sorted(synth.WORKLOADS)}")
+    wl = synth.WORKLOADS[name]
+    if override:
+        kw = {}
+        for item in override.split(","):
+            key, val = item.split("=")
+            kw[key] = type(getattr(wl, key))(val)
+        if "W" in kw:
+            kw["stream_seeds"] = tuple(wl.stream_seeds[0] + i for i in range(kw["W"]))
+        wl = synth.scaled(wl, name=f"{wl.name}[{override}]", **kw)
+    return wl
+
+
+def rank_streams(wl: synth.Workload, rank: int, batches: int):
+    """Token batches [batches, W, B] of this rank and the unigram counts of its whole stream."""
+    wl_r = synth.scaled(wl, stream_seeds=tuple(s + 1000 * rank for s in wl.stream_seeds))
+    full = synth.all_streams(wl_r)                       # whole stream: its histogram feeds the sampler
+    counts = synth.stream_counts(full, wl.V)
+    reps = -(-batches // wl.batches)
+    toks = np.stack([np.concatenate([s] * reps)[:batches] for s in full], axis=1)
+    return np.ascontiguousarray(toks), counts
+
+
+# ------------------------------------------------------------------------------------------------
+def run_ours(args):
+    import torch
+    import torch.distributed as dist
+
+    from paper_2211_10280_b200 import binding as B
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SGNS path has no CPU implementation")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = pick_workload(args.workload, args.override)
+    K, Wm = args.steps, max(args.warmup, 3)
+    Kp = min(K, 8)                                          # steps of the per-kernel timing pass
+    total_steps = 2 * (Wm + K) + Kp
+    toks_np, counts = rank_streams(wl, rank, total_steps)
+    P = wl.pairs_per_batch
+
+    ctx = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=wl.W, lr=wl.lr,
+                    max_delay=wl.max_delay, seed=wl.seed + rank, counts=counts, device=local, reduction=wl.reduction)
+    toks_dev = torch.from_numpy(toks_np).cuda()
+    toks_pin = torch.from_numpy(toks_np).pin_memory()
+    n_rows = {}
+
+    def step(t, host=False, info=False):
+        for i in range(wl.W):
+            if host:
+                _, inf = ctx.tensair_train_batch_host(i, toks_pin[t, i], t, want_loss=True, want_info=True)
+            else:
+                _, inf = ctx.tensair_train_batch(i, toks_dev[t, i], t, want_info=info)
+            if inf is not None:
+                n_rows[(i, t)] = (inf.n_rows, inf.n_in_rows)
+        for j in range(wl.W):
+            ctx.tensair_apply_messages(j, t)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(first, host):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        wall0 = time.time()
+        ev0.record()
+        for t in range(first, first + K):
+            step(t, host=host)
+        ev1.record()
+        barrier()
+        wall1 = time.time()
+        ms = ev0.elapsed_time(ev1)
+        if world > 1:
+            x = torch.tensor([ms], device="cuda", dtype=torch.float64)
+            dist.all_reduce(x, op=dist.ReduceOp.MAX)
+            ms = float(x.item())
+        return ms, wall0, wall1
+
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    t = 0
+    for _ in range(Wm):
+        step(t)
+        t += 1
+    sampler.start()
+    time.sleep(0.3)
+    launches0 = ctx.tensair_kernel_launches()
+    ms_dev, wall0, wall1 = timed(t, host=False)
+    launches = ctx.tensair_kernel_launches() - launches0
+    sampler.stop()
+    t += K
+    for _ in range(Wm):
+        step(t, host=True)
+        t += 1
+    ms_e2e, _, _ = timed(t, host=True)
+    t += K
+
+    # per-kernel pass: CUDA events around every launch, on the library's stream
+    ctx.tensair_profile(True)
+    ctx.tensair_profile_read()
+    first_prof = t
+    for _ in range(Kp):
+        step(t, info=True)
+        t += 1
+    prof = ctx.tensair_profile_read()
+    ctx.tensair_profile(False)
+    if ctx.tensair_sync() != B.OK:
+        raise SystemExit("the device reported a bad token during the benchmark")
+
+    pairs_per_step = wl.W * P
+    value = world * pairs_per_step * K / (ms_dev * 1e-3)
+    e2e_value = world * pairs_per_step * K / (ms_e2e * 1e-3)
+
+    # algorithmic bytes (each distinct row moved once per pass), from the exact row counts
+    row = 4 * wl.d
+    msgs = [n_rows[(i, s)] for i in range(wl.W) for s in range(first_prof, first_prof + Kp)]
+    U = float(np.mean([m[0] for m in msgs]))
+    U_in = float(np.mean([m[1] for m in msgs]))
+    U_out = U - U_in
+    applied = []
+    for j in range(wl.W):
+        for origin, snd, due, at, _ in ctx.tensair_read_delivery_log(j).tolist():
+            if first_prof <= at < first_prof + Kp and (snd, origin) in n_rows:
+                applied.append(n_rows[(snd, origin)][0])
+    U_applied = float(np.mean(applied)) if applied else U
+    algo = {
+        "forward": (U_out + U_in) * row,                                   # every touched row gathered once
+        "reduce_rows": U * (row + 4) + U_out * 2 * row,                   # message write + read/write of output rows
+        "apply_message": U_applied * (row + 4 + 2 * row),                 # delta read + row read + row write
+    }
+    tot_ms = sum(v[1] for v in prof.values()) or 1.0
+    kernels = {}
+    for name, (cnt, ms) in prof.items():
+        if not cnt:
+            continue
+        avg = ms / cnt
+        rec = {"launches_per_step": cnt / Kp, "avg_ms": round(avg, 5), "share": round(ms / tot_ms, 4)}
+        if name in algo:
+            rec["algorithmic_bytes"] = int(algo[name])
+            rec["gbs"] = round(algo[name] / (avg * 1e-3) / 1e9, 1)
+        kernels[name] = rec
+    dom = max((n for n in kernels if n in algo), key=lambda n: kernels[n]["share"])
+    peak, peak_kind = hbm_peak()
+    achieved = kernels[dom]["gbs"]
+    roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_source": f"of {peak_kind}",
+                "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": None,
+                "avg_ms": kernels[dom]["avg_ms"], "share_of_device_time": kernels[dom]["share"]}
+    own = U * row + U * (row + 4) + U * (row + 4 + 2 * row)
+    remote = (wl.W - 1) * U * (row + 4 + 2 * row)
+    step_bytes = wl.W * (own + remote)
+    step_gbs = step_bytes / (ms_dev * 1e-3 / K) / 1e9
+
+    out = {
+        "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
+                   "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
+                   "pairs_per_batch": P, "storage": "f32", "l2": "inputs larger than L2 (tables %.1f GB)" %
+                   (ctx.sizes.tables_bytes / 1e9), "parallelism": f"{world} independent replica groups"},
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / K,
+                "h2d_bytes_per_step": wl.W * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4)},
+        "gpu_launches": int(launches),
+        "clocks": sampler.summary(wall0, wall1),
+        "roofline": roofline,
+        "step_hbm": {"algorithmic_bytes_per_step": int(step_bytes), "gbs": round(step_gbs, 1),
+                     "frac_of_peak": round(step_gbs / peak, 4), "rows_per_message": int(U)},
+        "kernels": kernels,
+    }
+    if rank == 0 and world == 1 and not args.no_cpu_baseline:
+        out["cpu_baseline"] = cpu_baseline(wl, toks_np, counts, steps=2)
+    ctx.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
+# ------------------------------------------------------------------------------------------------
+def make_oracle(wl, counts):
+    from oracle import Oracle
+
+    return Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=wl.W, lr=wl.lr,
+                  max_delay=wl.max_delay, seed=wl.seed, counts=counts, reduction=wl.reduction)
+
+
+def cpu_baseline(wl, toks_np, counts, steps):
+    """The oracle as it stands on a bounded sample: the first `steps` steps of all replicas."""
+    import oracle
+
+    o = make_oracle(wl, counts)
+    t0 = time.time()
+    for t in range(steps):
+        for i in range(wl.W):
+            rc, _, _ = o.train_batch(i, toks_np[t, i], t)
+            assert rc == 0
+        for j in range(wl.W):
+            o.apply_messages(j, t)
+    dt = time.time() - t0
+    o.close()
+    return {"value": wl.W * wl.pairs_per_batch * steps / dt, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle",
+            "sample": f"first {steps} steps of all {wl.W} replicas ({wl.W * steps} batches, {dt:.1f} s)"}
+
+
+def run_reference(args):
+    """The CPU oracle as the reference arm: every step trains one replica's batch (replicas in turn) and,
+    once all replicas have trained a step, applies what is due - a bounded sample of the workload."""
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    if rank != 0:
+        return
+    import oracle
+
+    wl = pick_workload(args.workload, args.override)
+    K, Wm = args.steps, args.warmup
+    total = Wm + K
+    toks_np, counts = rank_streams(wl, 0, -(-total // wl.W) + 1)
+    o = make_oracle(wl, counts)
+
+    def step(s):
+        t, i = divmod(s, wl.W)
+        rc, _, _ = o.train_batch(i, toks_np[t, i], t)
+        assert rc == 0
+        if i == wl.W - 1:
+            for j in range(wl.W):
+                o.apply_messages(j, t)
+
+    for s in range(Wm):
+        step(s)
+    t0 = time.time()
+    for s in range(Wm, total):
+        step(s)
+    dt = time.time() - t0
+    value = wl.pairs_per_batch * K / dt
+    sample = f"{K} steps of one replica-batch each (replicas in turn, messages applied after every {wl.W}th)"
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
+        "warmup": Wm, "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
+                   "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
+                   "pairs_per_batch": wl.pairs_per_batch},
+        "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
+        "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=60)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--workload", default=synth.LARGE_DASGD.name)
+    ap.add_argument("--override", default="", help="comma-separated field=value replacements of the workload")
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -213,6 +213,19 @@ TENSAIR_API int tensair_pending(tensair_ctx* ctx, uint32_t replica, uint64_t* n)
 /* Kernels launched by this context so far. */
 TENSAIR_API uint64_t tensair_kernel_launches(const tensair_ctx* ctx);
 
+/* Per-kernel timing.  While enabled, every kernel launch is bracketed by a pair of CUDA events on the
+ * context's stream (a few microseconds of overhead per launch, so do not time whole steps with it on).
+ * tensair_profile_read synchronises, writes one record per kernel kind (up to max_kinds; n_kinds =
+ * how many kinds exist) with the launches and summed device time since the previous read, and
+ * forgets them. */
+typedef struct tensair_kernel_time {
+    char name[32];
+    uint64_t launches;
+    double total_ms;
+} tensair_kernel_time;
+TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
+TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);
+
 TENSAIR_API const char* tensair_strerror(int code);
 TENSAIR_API const char* tensair_last_error(const tensair_ctx* ctx);
 

@@ -47,6 +47,10 @@ class Delivery(C.Structure):
                 ("applied_at", C.c_uint64), ("staleness", C.c_uint64)]
 
 
+class KernelTime(C.Structure):
+    _fields_ = [("name", C.c_char * 32), ("launches", C.c_uint64), ("total_ms", C.c_double)]
+
+
 class TensairError(RuntimeError):
     def __init__(self, code: int, what: str, detail: str = ""):
         self.code = code
@@ -75,6 +79,8 @@ SYMBOLS = {
     "tensair_read_delivery_log": (_int, [_vp, _u32, _u64, _vp, _P(_u64)]),
     "tensair_pending": (_int, [_vp, _u32, _P(_u64)]),
     "tensair_kernel_launches": (_u64, [_vp]),
+    "tensair_profile": (_int, [_vp, _int]),
+    "tensair_profile_read": (_int, [_vp, _u32, _vp, _P(_u32)]),
     "tensair_strerror": (C.c_char_p, [_int]),
     "tensair_last_error": (C.c_char_p, [_vp]),
     "tensair_build_alias_host": (_int, [_vp, _u32, _vp, _vp]),
@@ -331,3 +337,13 @@ class Context:
 
     def tensair_kernel_launches(self) -> int:
         return int(lib().tensair_kernel_launches(self._h))
+
+    def tensair_profile(self, enable: bool):
+        _check(lib().tensair_profile(self._h, int(enable)), "tensair_profile", self._h)
+
+    def tensair_profile_read(self) -> dict:
+        """{kernel name: (launches, total milliseconds)} since the previous read."""
+        n = C.c_uint32(0)
+        buf = (KernelTime * 64)()
+        _check(lib().tensair_profile_read(self._h, 64, buf, C.byref(n)), "tensair_profile_read", self._h)
+        return {buf[i].name.decode(): (int(buf[i].launches), float(buf[i].total_ms)) for i in range(min(64, n.value))}

@@ -45,6 +45,7 @@ cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uin
     const int blocks = L.sms * 8;
     const float4* d4p = reinterpret_cast<const float4*>(delta);
     float4* t4 = reinterpret_cast<float4*>(table);
+    Timed timed(L, input_rows_only ? K_APPLY_INPUT_ROWS : K_APPLY_MESSAGE);
 #define TENSAIR_APPLY(NV) k_apply<NV><<<blocks, 256, 0, L.stream>>>(hdr, ids, d4p, t4, s.d4, stride4, input_rows_only)
     if (s.d4 <= 32) TENSAIR_APPLY(1);
     else if (s.d4 <= 64) TENSAIR_APPLY(2);
@@ -52,7 +53,6 @@ cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uin
     else if (s.d4 <= 128) TENSAIR_APPLY(4);
     else TENSAIR_APPLY(8);
 #undef TENSAIR_APPLY
-    ++*L.launches;
     return cudaGetLastError();
 }
 

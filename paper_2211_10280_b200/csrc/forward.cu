@@ -138,6 +138,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     const size_t smem = ((size_t)warps * s.d + warps) * sizeof(double);
     const uint32_t stride4 = s.stride / 4;
     const float4* t4 = reinterpret_cast<const float4*>(table);
+    Timed timed(L, K_FORWARD);
 #define TENSAIR_FWD(NV, RIF) \
     k_forward<NV, RIF><<<n, warps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k, t4, rows, rec, gin_pos, loss_pos, err)
     if (s.d4 <= 32) TENSAIR_FWD(1, 4);
@@ -146,7 +147,6 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     else if (s.d4 <= 128) TENSAIR_FWD(4, 2);
     else TENSAIR_FWD(8, 1);
 #undef TENSAIR_FWD
-    ++*L.launches;
     return cudaGetLastError();
 }
 
@@ -167,8 +167,8 @@ k_loss_sum(const double* __restrict__ loss_pos, uint32_t n, double* __restrict__
 }
 
 cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err) {
+    Timed timed(L, K_LOSS_SUM);
     k_loss_sum<<<1, 1024, 0, L.stream>>>(loss_pos, n < 2 ? 0 : n, loss, err);
-    ++*L.launches;
     return cudaGetLastError();
 }
 

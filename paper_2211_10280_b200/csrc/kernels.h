@@ -1,13 +1,60 @@
 // Host-side launchers of the kernels; each enqueues on L.stream and returns the launch status.
 #pragma once
+#include <vector>
+
 #include "common.cuh"
 
 namespace tensair {
+
+enum KernelKind {
+    K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
+    K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_KINDS
+};
+inline const char* kernel_name(int kind) {
+    static const char* const names[K_KINDS] = {
+        "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
+        "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
+        "apply_message", "init_table"};
+    return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
+}
+
+// Optional per-launch timing: a pair of CUDA events around every kernel launch while `on` is set.
+struct Profiler {
+    struct Span { int kind; cudaEvent_t start, stop; };
+    bool on = false;
+    std::vector<Span> spans;
+    std::vector<cudaEvent_t> spare;
+    cudaEvent_t take() {
+        cudaEvent_t e = nullptr;
+        if (!spare.empty()) { e = spare.back(); spare.pop_back(); }
+        else cudaEventCreate(&e);
+        return e;
+    }
+};
 
 struct Launcher {
     cudaStream_t stream;
     uint64_t* launches;   // incremented once per kernel launch
     int sms;              // multiprocessors of the device
+    Profiler* prof;       // nullable
+};
+
+// Counts one kernel launch and, when profiling, brackets it with events: construct right before the
+// launch, let it go out of scope right after.
+struct Timed {
+    const Launcher& L;
+    cudaEvent_t stop = nullptr;
+    Timed(const Launcher& l, int kind) : L(l) {
+        ++*L.launches;
+        if (L.prof && L.prof->on) {
+            cudaEvent_t start = L.prof->take();
+            stop = L.prof->take();
+            cudaEventRecord(start, L.stream);
+            L.prof->spans.push_back(Profiler::Span{kind, start, stop});
+        }
+    }
+    ~Timed() { if (stop) cudaEventRecord(stop, L.stream); }
 };
 
 // sampler.cu

@@ -152,14 +152,16 @@ cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_ite
                          const uint32_t* err) {
     const uint32_t tiles = heads_tiles(n_items);
     if (tiles) {
+        Timed timed(L, K_HEADS_COUNT);
         k_heads_count<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, tile_counts, err);
-        ++*L.launches;
     }
-    k_heads_scan<<<1, 1024, 0, L.stream>>>(sorted, n_items, V, tile_counts, tiles, hdr, seg_start, long_counters, err);
-    ++*L.launches;
+    {
+        Timed timed(L, K_HEADS_SCAN);
+        k_heads_scan<<<1, 1024, 0, L.stream>>>(sorted, n_items, V, tile_counts, tiles, hdr, seg_start, long_counters, err);
+    }
     if (tiles) {
+        Timed timed(L, K_HEADS_WRITE);
         k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, err);
-        ++*L.launches;
     }
     return cudaGetLastError();
 }
@@ -359,13 +361,21 @@ static cudaError_t reduce_all(const Launcher& L, const item_t* sorted, const Msg
     const int blocks = L.sms * 8;
     float4* t4 = reinterpret_cast<float4*>(table);
     float4* d4p = reinterpret_cast<float4*>(delta);
+    {
+    Timed timed(L, K_REDUCE_ROWS);
     k_reduce_rows<NV><<<blocks, 256, 0, L.stream>>>(sorted, hdr, ids, seg_start, rec, gin_pos, t4, d4p, s.V, s.d4, stride4,
                                                     scale, long_counters, long_rows, chunk_items);
+    }
+    {
+    Timed timed(L, K_REDUCE_CHUNKS);
     k_reduce_chunks<NV><<<blocks, 256, 0, L.stream>>>(sorted, ids, seg_start, rec, gin_pos, t4, s.V, s.d4, stride4,
                                                       long_counters, chunk_items, partials);
+    }
+    {
+    Timed timed(L, K_REDUCE_LONG);
     k_reduce_long<NV><<<L.sms * 2, 256, 0, L.stream>>>(ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters,
                                                        long_rows);
-    *L.launches += 3;
+    }
     return cudaGetLastError();
 }
 

@@ -137,10 +137,18 @@ cudaError_t launch_sort(const Launcher& L, item_t* a, item_t* b, uint32_t n, uin
     item_t* src = a;
     item_t* dst = b;
     for (uint32_t shift = 0; shift < key_bits; shift += kRadixBits) {
-        k_radix_hist<<<tiles, kSortThreads, 0, L.stream>>>(src, n, shift, hist, tiles);
-        k_scan_exclusive<<<1, 1024, 0, L.stream>>>(hist, tiles * kBins);
-        k_radix_scatter<<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles);
-        *L.launches += 3;
+        {
+            Timed timed(L, K_SORT_HIST);
+            k_radix_hist<<<tiles, kSortThreads, 0, L.stream>>>(src, n, shift, hist, tiles);
+        }
+        {
+            Timed timed(L, K_SORT_SCAN);
+            k_scan_exclusive<<<1, 1024, 0, L.stream>>>(hist, tiles * kBins);
+        }
+        {
+            Timed timed(L, K_SORT_SCATTER);
+            k_radix_scatter<<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles);
+        }
         item_t* t = src; src = dst; dst = t;
     }
     *sorted = src;

@@ -57,8 +57,8 @@ __global__ void k_validate(const int32_t* __restrict__ tok, uint32_t n, uint32_t
 
 cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, uint32_t V, uint32_t* err) {
     if (n == 0) return cudaSuccess;
+    Timed timed(L, K_VALIDATE);
     k_validate<<<(n + 255) / 256, 256, 0, L.stream>>>(tok, n, V, err);
-    ++*L.launches;
     return cudaGetLastError();
 }
 
@@ -120,9 +120,9 @@ cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, co
     if (n == 0) return cudaSuccess;
     const uint64_t total = (uint64_t)n * 2 * s.w * ((s.k + 1) / 2);
     const uint32_t blocks = (uint32_t)((total + 255) / 256);
+    Timed timed(L, K_PREPARE);
     k_prepare<<<blocks, 256, 0, L.stream>>>(tok, n, s.V, s.w, s.k, replica, batch_lo, (uint32_t)seed,
                                             (uint32_t)(seed >> 32), alias_tab, rows, items, counts, err);
-    ++*L.launches;
     return cudaGetLastError();
 }
 
@@ -147,9 +147,9 @@ __global__ void k_init_input(float* __restrict__ table, uint32_t V, uint32_t d, 
 
 cudaError_t launch_init_input_table(const Launcher& L, float* table, const Shape& s, uint64_t seed) {
     const uint64_t groups = ((uint64_t)s.V * s.d + 3) / 4;
+    Timed timed(L, K_INIT_TABLE);
     k_init_input<<<(uint32_t)((groups + 255) / 256), 256, 0, L.stream>>>(table, s.V, s.d, s.stride, (uint32_t)seed,
                                                                           (uint32_t)(seed >> 32));
-    ++*L.launches;
     return cudaGetLastError();
 }
 

@@ -91,6 +91,7 @@ struct tensair_ctx {
     cudaStream_t stream;
     Launcher L;
     uint64_t launches = 0;
+    Profiler prof;
     float* tables;
     uint8_t* pool;
     uint8_t* scratch;
@@ -280,7 +281,7 @@ int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const u
     int status = TENSAIR_OK;
     auto bail = [&](int code) { delete ctx->sched; if (ctx->stage) cudaFreeHost(ctx->stage); delete ctx; return code; };
     if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return bail(TENSAIR_ECUDA);
-    ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount};
+    ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount, &ctx->prof};
     if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->sched = new Schedule(cfg->W, cfg->max_delay, cfg->seed);
 
@@ -318,6 +319,8 @@ void tensair_destroy(tensair_ctx* ctx) {
     if (!ctx) return;
     DeviceGuard guard(ctx->cfg.device);
     cudaStreamSynchronize(ctx->stream);
+    for (const Profiler::Span& sp : ctx->prof.spans) { cudaEventDestroy(sp.start); cudaEventDestroy(sp.stop); }
+    for (cudaEvent_t e : ctx->prof.spare) cudaEventDestroy(e);
     if (ctx->stage) cudaFreeHost(ctx->stage);
     delete ctx->sched;
     delete ctx;
@@ -477,6 +480,38 @@ int tensair_pending(tensair_ctx* ctx, uint32_t replica, uint64_t* n) {
 }
 
 uint64_t tensair_kernel_launches(const tensair_ctx* ctx) { return ctx ? ctx->launches : 0; }
+
+int tensair_profile(tensair_ctx* ctx, int enable) {
+    if (!ctx) return TENSAIR_EINVAL;
+    ctx->prof.on = enable != 0;
+    return TENSAIR_OK;
+}
+
+int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    double total[K_KINDS] = {0};
+    uint64_t count[K_KINDS] = {0};
+    for (const Profiler::Span& sp : ctx->prof.spans) {
+        float ms = 0.0f;
+        TENSAIR_CUDA(ctx, cudaEventElapsedTime(&ms, sp.start, sp.stop));
+        total[sp.kind] += ms;
+        ++count[sp.kind];
+        ctx->prof.spare.push_back(sp.start);
+        ctx->prof.spare.push_back(sp.stop);
+    }
+    ctx->prof.spans.clear();
+    if (n_kinds) *n_kinds = K_KINDS;
+    for (uint32_t i = 0; i < K_KINDS && i < max_kinds && out; ++i) {
+        std::memset(&out[i], 0, sizeof(out[i]));
+        std::snprintf(out[i].name, sizeof(out[i].name), "%s", kernel_name((int)i));
+        out[i].launches = count[i];
+        out[i].total_ms = total[i];
+    }
+    return TENSAIR_OK;
+}
 
 const char* tensair_strerror(int code) {
     switch (code) {
