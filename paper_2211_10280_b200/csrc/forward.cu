@@ -1,151 +1,247 @@
 // Gradient calculation at the snapshot: fused gather -> dot -> sigmoid -> gradient scalars, centre-stationary.
 // Rows are fp32 in memory; the dot products, the sigmoid and the partial sums are taken in fp64.
-//
-// One block per centre position q.  Each warp takes window slots of that position; for a slot it keeps
-// the centre row v_c in registers, gathers the 1 + k output rows of the pair (positive first), reduces
-// each dot product with warp shuffles, turns it into the gradient scalar g (sigma(x) - 1 for the
-// positive, sigma(x) for a negative, 0 for a negative equal to the positive), records g for the later
-// per-output-row sums and accumulates g * u into the centre's own gradient while the row is still in
-// registers - the output rows are read from memory exactly once per contribution.  The block then adds
-// its warps' partial sums in warp order and writes one partial centre gradient per position.
+// Each output row is fetched from memory once per contribution (by a bulk asynchronous copy into
+// shared memory) and serves both its dot product and the centre's gradient; the gradient scalar g
+// (sigma(x) - 1 for the positive, sigma(x) for a negative, 0 for a negative equal to the positive) is
+// recorded for the later per-output-row sums.
 #include "kernels.h"
 
 namespace tensair {
 
 
-// -log(sigmoid(-z)) = log(1 + e^z), without overflow
-__device__ inline double softplus(double z) { return fmax(z, 0.0) + log1p(exp(-fabs(z))); }
+// ---- asynchronous bulk copies (global -> shared) completed on an mbarrier -------------------------
+__device__ inline uint32_t smem_addr(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+__device__ inline void mbar_init(uint64_t* bar, uint32_t arrivals) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(smem_addr(bar)), "r"(arrivals) : "memory");
+    asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+}
+__device__ inline void mbar_arrive_expect_tx(uint64_t* bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(smem_addr(bar)), "r"(bytes) : "memory");
+}
+__device__ inline bool mbar_try_wait(uint64_t* bar, uint32_t parity) {
+    uint32_t done;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\tmbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\tselp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(done) : "r"(smem_addr(bar)), "r"(parity) : "memory");
+    return done != 0;
+}
+// Waits for a phase of the barrier, giving up after about a second.
+__device__ inline bool mbar_wait_bounded(uint64_t* bar, uint32_t parity) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    while (!mbar_try_wait(bar, parity))
+        if (clock64() - t0 > 2000000000LL) return false;
+    return true;
+}
+__device__ inline void bulk_copy_g2s(void* dst_smem, const void* src_global, uint32_t bytes, uint64_t* bar) {
+    asm volatile("cp.async.bulk.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1], %2, [%3];"
+                 ::"r"(smem_addr(dst_smem)), "l"(src_global), "r"(bytes), "r"(smem_addr(bar)) : "memory");
+}
+// Orders this thread's earlier shared-memory reads before later asynchronous writes to the same memory.
+__device__ inline void fence_generic_to_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-// NV: float4 slices per lane; RIF: output rows a warp loads before it starts reducing.
-template <int NV, int RIF>
-__global__ void __launch_bounds__(384)
+__device__ inline double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
+// -log(sigmoid(x)) without overflow
+__device__ inline double neg_log_sigmoid(double x) { return (x < 0.0 ? -x : 0.0) + log1p(exp(-fabs(x))); }
+
+constexpr int kChunkRows = 16;     // output rows a warp stages and reduces together
+constexpr int kFwdWarps = 2;       // warps per block
+
+// One warp per centre position (grid-stride), no block-level cooperation.  For every pair of the
+// position the warp stages the pair's 1 + k output rows into its own shared-memory buffer with one
+// bulk asynchronous copy per row (all in flight together, completion counted by an mbarrier), then
+//   1. takes the partial dot products of all staged rows with the centre row held in registers,
+//   2. reduces them with a transposing shuffle network that leaves row j's dot product in lanes 2j, 2j+1,
+//   3. evaluates sigmoid and loss for all rows at once (one row per lane pair instead of one per warp),
+//   4. re-reads the staged rows and adds g * u to the centre gradient kept in registers.
+// The centre gradient is written once per position; nothing is shared between warps.
+template <int NV>
+__global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, uint32_t stride4, uint32_t w,
-          uint32_t k, const float4* __restrict__ table, const uint32_t* __restrict__ rows, Rec* __restrict__ rec,
-          double* __restrict__ gin_pos, double* __restrict__ loss_pos, const uint32_t* __restrict__ err) {
+          uint32_t k, uint32_t chunk_rows, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
+          Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err) {
     if (*err) return;
-    extern __shared__ double smem[];          // [warps][4*d4] partial centre gradients, then [warps] losses
-    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5, nwarps = blockDim.x >> 5;
-    double* loss_s = smem + (size_t)nwarps * d4 * 4;
-    const uint32_t q = blockIdx.x;
-    const uint32_t centre = (uint32_t)tok[q];
+    extern __shared__ __align__(128) unsigned char smem_raw[];
+    const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
+    float4* stage = reinterpret_cast<float4*>(smem_raw) + (size_t)wib * chunk_rows * stride4;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)kFwdWarps * chunk_rows * stride4 * sizeof(float4)) + wib;
+    if (lane == 0) mbar_init(bar, 1);
+    __syncwarp();
+    uint32_t parity = 0;
+    bool failed = false;
     const uint32_t K1 = k + 1;
-    const float4* __restrict__ vin = table + (size_t)centre * stride4;
+    const uint32_t row_bytes = d4 * 16;
     const float4* __restrict__ tout = table + (size_t)V * stride4;
+    const uint32_t warp = blockIdx.x * kFwdWarps + wib, nwarps = gridDim.x * kFwdWarps;
 
-    // the centre row and this warp's partial gradient, both in fp64
-    double v[NV][4], acc[NV][4];
+    for (uint32_t q = warp; q < n && !failed; q += nwarps) {
+        const uint32_t centre = (uint32_t)tok[q];
+        const float4* __restrict__ vin = table + (size_t)centre * stride4;
+        double v[NV][4], acc[NV][4];
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-        const uint32_t e = lane + 32 * i;
-        const float4 f = e < d4 ? __ldg(vin + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-        v[i][0] = (double)f.x; v[i][1] = (double)f.y; v[i][2] = (double)f.z; v[i][3] = (double)f.w;
-        acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0;
-    }
-    double loss = 0.0;
-    const uint32_t lo = q > w ? q - w : 0;
-    const uint32_t pbase = pair_offset(q, n, w);
+        for (int i = 0; i < NV; ++i) {
+            const uint32_t e = lane + 32 * i;
+            const float4 f = e < d4 ? __ldg(vin + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+            v[i][0] = (double)f.x; v[i][1] = (double)f.y; v[i][2] = (double)f.z; v[i][3] = (double)f.w;
+            acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0;
+        }
+        double loss = 0.0;
+        const uint32_t lo = q > w ? q - w : 0;
+        const uint32_t hi = q + w < n ? q + w : n - 1;
+        uint32_t p = pair_offset(q, n, w);
+        for (uint32_t c = lo; c <= hi && !failed; ++c) {
+            if (c == q) continue;
+            const uint32_t ctx = (uint32_t)tok[c];
+            const uint32_t cbase = p * K1;
+            ++p;
+            for (uint32_t j0 = 0; j0 < K1 && !failed; j0 += chunk_rows) {
+                const uint32_t nr = K1 - j0 < chunk_rows ? K1 - j0 : chunk_rows;
+                const uint32_t rid = lane < nr ? __ldg(rows + cbase + j0 + lane) : 0u;
+                const bool mine = lane < nr && (j0 + lane == 0 || rid != ctx);
+                const uint32_t live = __ballot_sync(0xFFFFFFFFu, mine);
+                // stage the live rows: the buffer was last read by this warp, so order those reads first
+                fence_generic_to_async();
+                __syncwarp();
+                if (lane == 0) mbar_arrive_expect_tx(bar, __popc(live) * row_bytes);
+                __syncwarp();
+                if (mine) bulk_copy_g2s(stage + (size_t)lane * stride4, tout + (size_t)rid * stride4, row_bytes, bar);
+                if (__any_sync(0xFFFFFFFFu, !mbar_wait_bounded(bar, parity))) {
+                    failed = true;
+                    mbar_wait_bounded(bar, parity);   // give copies still in flight one more chance to land
+                    break;
+                }
+                parity ^= 1;
 
-    for (uint32_t s = wid; s < 2 * w; s += nwarps) {
-        const int64_t c = (int64_t)q + (s < w ? (int64_t)s - (int64_t)w : (int64_t)s - (int64_t)w + 1);
-        if (c < 0 || c >= (int64_t)n) continue;
-        const uint32_t p = pbase + ((uint32_t)c - lo) - ((uint32_t)c > q ? 1u : 0u);
-        const uint32_t cbase = p * K1;
-        const uint32_t ctx = (uint32_t)tok[c];
-        for (uint32_t j0 = 0; j0 < K1; j0 += RIF) {
-            uint32_t r[RIF];
-            bool live[RIF];
-            float4 u[RIF][NV];
+                // 1. partial dot products of the staged rows
+                double xp[kChunkRows];
 #pragma unroll
-            for (int t = 0; t < RIF; ++t) {
-                const uint32_t j = j0 + t;
-                r[t] = j < K1 ? __ldg(rows + cbase + j) : ctx;
-                live[t] = j < K1 && (j == 0 || r[t] != ctx);
-            }
+                for (int j = 0; j < kChunkRows; ++j) {
+                    xp[j] = 0.0;
+                    if ((live >> j) & 1u) {
+                        const float4* __restrict__ u = stage + (size_t)j * stride4;
 #pragma unroll
-            for (int t = 0; t < RIF; ++t) {
-                const float4* __restrict__ urow = tout + (size_t)r[t] * stride4;
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const uint32_t e = lane + 32 * i;
-                    u[t][i] = (live[t] && e < d4) ? __ldg(urow + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-                }
-            }
-#pragma unroll
-            for (int t = 0; t < RIF; ++t) {
-                const uint32_t j = j0 + t;
-                if (j >= K1) break;
-                double ud[NV][4];
-                double x = 0.0;
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    ud[i][0] = (double)u[t][i].x; ud[i][1] = (double)u[t][i].y;
-                    ud[i][2] = (double)u[t][i].z; ud[i][3] = (double)u[t][i].w;
-                    x = fma(ud[i][0], v[i][0], x);
-                    x = fma(ud[i][1], v[i][1], x);
-                    x = fma(ud[i][2], v[i][2], x);
-                    x = fma(ud[i][3], v[i][3], x);
-                }
-#pragma unroll
-                for (int o = 16; o > 0; o >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, o);
-                double g = 0.0;
-                if (live[t]) {
-                    const double sig = 1.0 / (1.0 + exp(-x));
-                    g = j == 0 ? sig - 1.0 : sig;
-                    loss += softplus(j == 0 ? -x : x);
-#pragma unroll
-                    for (int i = 0; i < NV; ++i) {
-                        acc[i][0] = fma(g, ud[i][0], acc[i][0]);
-                        acc[i][1] = fma(g, ud[i][1], acc[i][1]);
-                        acc[i][2] = fma(g, ud[i][2], acc[i][2]);
-                        acc[i][3] = fma(g, ud[i][3], acc[i][3]);
+                        for (int i = 0; i < NV; ++i) {
+                            const uint32_t e = lane + 32 * i;
+                            if (e < d4) {
+                                const float4 f = u[e];
+                                xp[j] = fma((double)f.x, v[i][0], xp[j]);
+                                xp[j] = fma((double)f.y, v[i][1], xp[j]);
+                                xp[j] = fma((double)f.z, v[i][2], xp[j]);
+                                xp[j] = fma((double)f.w, v[i][3], xp[j]);
+                            }
+                        }
                     }
                 }
-                if (lane == 0) rec[cbase + j] = Rec{g, centre, 0u};
+                // 2. transposing reduction: after it lanes 2j and 2j+1 hold the dot product of row j
+#pragma unroll
+                for (int i = 0; i < 8; ++i) {
+                    const bool up = lane & 16;
+                    const double keep = up ? xp[8 + i] : xp[i], give = up ? xp[i] : xp[8 + i];
+                    xp[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 16);
+                }
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const bool up = lane & 8;
+                    const double keep = up ? xp[4 + i] : xp[i], give = up ? xp[i] : xp[4 + i];
+                    xp[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 8);
+                }
+#pragma unroll
+                for (int i = 0; i < 2; ++i) {
+                    const bool up = lane & 4;
+                    const double keep = up ? xp[2 + i] : xp[i], give = up ? xp[i] : xp[2 + i];
+                    xp[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 4);
+                }
+                {
+                    const bool up = lane & 2;
+                    const double keep = up ? xp[1] : xp[0], give = up ? xp[0] : xp[1];
+                    xp[0] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 2);
+                }
+                const double x = xp[0] + __shfl_xor_sync(0xFFFFFFFFu, xp[0], 1);
+                // 3. gradient scalar and loss of row (lane / 2), all rows at once
+                const uint32_t jr = lane >> 1;
+                double g = 0.0;
+                if ((live >> jr) & 1u) {
+                    const bool positive = j0 + jr == 0;
+                    const double sig = sigmoid(x);
+                    g = positive ? sig - 1.0 : sig;
+                    if (!(lane & 1)) loss += neg_log_sigmoid(positive ? x : -x);
+                }
+                if (!(lane & 1) && jr < nr) rec[cbase + j0 + jr] = Rec{g, centre, 0u};
+                // 4. centre gradient: acc += g_j * u_j
+#pragma unroll
+                for (int j = 0; j < kChunkRows; ++j) {
+                    const double gj = __shfl_sync(0xFFFFFFFFu, g, 2 * j);
+                    if ((live >> j) & 1u) {
+                        const float4* __restrict__ u = stage + (size_t)j * stride4;
+#pragma unroll
+                        for (int i = 0; i < NV; ++i) {
+                            const uint32_t e = lane + 32 * i;
+                            if (e < d4) {
+                                const float4 f = u[e];
+                                acc[i][0] = fma(gj, (double)f.x, acc[i][0]);
+                                acc[i][1] = fma(gj, (double)f.y, acc[i][1]);
+                                acc[i][2] = fma(gj, (double)f.z, acc[i][2]);
+                                acc[i][3] = fma(gj, (double)f.w, acc[i][3]);
+                            }
+                        }
+                    }
+                }
             }
         }
-    }
+        if (failed) break;
+        double2* out = reinterpret_cast<double2*>(gin_pos + (size_t)q * stride4 * 4);
 #pragma unroll
-    for (int i = 0; i < NV; ++i) {
-        const uint32_t e = lane + 32 * i;
-        if (e < d4) {
-            double* dst = smem + ((size_t)wid * d4 + e) * 4;
-            dst[0] = acc[i][0]; dst[1] = acc[i][1]; dst[2] = acc[i][2]; dst[3] = acc[i][3];
+        for (int i = 0; i < NV; ++i) {
+            const uint32_t e = lane + 32 * i;
+            if (e < d4) {
+                out[2 * e] = make_double2(acc[i][0], acc[i][1]);
+                out[2 * e + 1] = make_double2(acc[i][2], acc[i][3]);
+            }
         }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xFFFFFFFFu, loss, o);
+        if (lane == 0) loss_pos[q] = loss;
     }
-    if (lane == 0) loss_s[wid] = loss;
-    __syncthreads();
-    const uint32_t dd = d4 * 4;
-    for (uint32_t e = threadIdx.x; e < dd; e += blockDim.x) {
-        double sum = smem[e];
-        for (uint32_t x = 1; x < nwarps; ++x) sum += smem[(size_t)x * dd + e];
-        gin_pos[(size_t)q * stride4 * 4 + e] = sum;
-    }
-    if (threadIdx.x == 0) {
-        double l = loss_s[0];
-        for (uint32_t x = 1; x < nwarps; ++x) l += loss_s[x];
-        loss_pos[q] = l;
-    }
+    if (failed && lane == 0) atomicOr(err, 2u);
+}
+
+// Rows per staging chunk and bytes of dynamic shared memory per block.
+static uint32_t forward_chunk_rows(const Shape& s, size_t* smem) {
+    const size_t budget = 200 * 1024 / 5;          // five blocks per multiprocessor
+    const size_t row = (size_t)s.stride * 4;
+    uint32_t r = s.K1 < (uint32_t)kChunkRows ? s.K1 : (uint32_t)kChunkRows;
+    while (r > 1 && (size_t)kFwdWarps * r * row + kFwdWarps * 8 > budget) --r;
+    *smem = (size_t)kFwdWarps * r * row + kFwdWarps * 8;
+    return r;
 }
 
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
-                           const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, const uint32_t* err) {
+                           const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err) {
     if (n < 2) return cudaSuccess;
-    uint32_t warps = 2 * s.w;
-    if (warps > 12) warps = 12;
-    const uint32_t fit = 49152 / (s.d * 8 + 8);   // partial sums and losses within 48 KB of shared memory
-    if (warps > fit) warps = fit;
-    if (warps < 1) warps = 1;
-    const size_t smem = ((size_t)warps * s.d + warps) * sizeof(double);
+    size_t smem = 0;
+    const uint32_t chunk_rows = forward_chunk_rows(s, &smem);
     const uint32_t stride4 = s.stride / 4;
     const float4* t4 = reinterpret_cast<const float4*>(table);
+    uint32_t blocks = (n + kFwdWarps - 1) / kFwdWarps;
+    const uint32_t resident = (uint32_t)L.sms * 5;
+    if (blocks > resident) blocks = resident;
     Timed timed(L, K_FORWARD);
-#define TENSAIR_FWD(NV, RIF) \
-    k_forward<NV, RIF><<<n, warps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k, t4, rows, rec, gin_pos, loss_pos, err)
-    if (s.d4 <= 32) TENSAIR_FWD(1, 4);
-    else if (s.d4 <= 64) TENSAIR_FWD(2, 4);
-    else if (s.d4 <= 96) TENSAIR_FWD(3, 4);
-    else if (s.d4 <= 128) TENSAIR_FWD(4, 2);
-    else TENSAIR_FWD(8, 1);
+#define TENSAIR_FWD(NV)                                                                                         \
+    do {                                                                                                        \
+        static bool attr_set = false;                                                                           \
+        if (!attr_set) {                                                                                        \
+            cudaFuncSetAttribute(k_forward<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);       \
+            cudaFuncSetAttribute(k_forward<NV>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);           \
+            attr_set = true;                                                                                    \
+        }                                                                                                       \
+        k_forward<NV><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k, chunk_rows, \
+                                                                  t4, rows, rec, gin_pos, loss_pos, err);       \
+    } while (0)
+    if (s.d4 <= 32) TENSAIR_FWD(1);
+    else if (s.d4 <= 64) TENSAIR_FWD(2);
+    else if (s.d4 <= 96) TENSAIR_FWD(3);
+    else if (s.d4 <= 128) TENSAIR_FWD(4);
+    else TENSAIR_FWD(8);
 #undef TENSAIR_FWD
     return cudaGetLastError();
 }

@@ -75,16 +75,16 @@ uint32_t sort_hist_words(uint32_t n);
 
 // forward.cu
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
-                           const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, const uint32_t* err);
+                           const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err);
 cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err);
 
 // message.cu
 uint32_t heads_tiles(uint32_t n_items);
 cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
                          MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
-                         const uint32_t* err);
-cudaError_t launch_reduce(const Launcher& L, const item_t* sorted, const MsgHeader* hdr, const uint32_t* ids,
-                          const uint32_t* seg_start, const Rec* rec, const double* gin_pos, float* table,
+                         const Rec* rec, Rec* terms, const uint32_t* err);
+cudaError_t launch_reduce(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
+                          const uint32_t* seg_start, const double* gin_pos, float* table,
                           float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
                           ChunkItem* chunk_items, double* partials);
 

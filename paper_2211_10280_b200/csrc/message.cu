@@ -3,6 +3,7 @@
 //
 // After the stable sort all contributions to one row are contiguous and in a fixed order.  "Heads"
 // (first item of each distinct key) give the message's ascending id list and the segment bounds.
+// The scalars of the contributions are gathered into that order once ("terms").
 // A warp then owns a row: it adds coefficient * source row over the segment (source = the centre's
 // input row and coefficient g for an output row; source = a position's partial centre gradient and
 // coefficient 1 for an input row), scales by -lr, writes the delta row into the message and, for an
@@ -114,8 +115,16 @@ k_heads_scan(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, ui
 __global__ void __launch_bounds__(kHeadThreads)
 k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, const uint32_t* __restrict__ tile_base,
               MsgHeader* __restrict__ hdr, uint32_t* __restrict__ ids, uint32_t* __restrict__ seg_start,
-              const uint32_t* __restrict__ err) {
+              const Rec* __restrict__ rec, Rec* __restrict__ terms, const uint32_t* __restrict__ err) {
     if (*err) return;
+    // terms[i] = scalar and centre token of the i-th sorted contribution (for an input-row item: the
+    // centre position), so that the row sums read their terms contiguously
+    for (uint32_t i = blockIdx.x * kHeadTile + threadIdx.x; i < n_items && i < (blockIdx.x + 1) * kHeadTile; i += kHeadThreads) {
+        const item_t it = sorted[i];
+        const uint32_t key = item_key(it);
+        if (key < V) terms[i] = Rec{1.0, item_payload(it), 0u};
+        else if (key < 2 * V) terms[i] = rec[item_payload(it)];
+    }
     __shared__ uint32_t warp_tot[kHeadThreads / 32];
     uint32_t keys[kHeadItems];
     const uint32_t first = blockIdx.x * kHeadTile + threadIdx.x * kHeadItems;
@@ -149,7 +158,7 @@ k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, c
 
 cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
                          MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
-                         const uint32_t* err) {
+                         const Rec* rec, Rec* terms, const uint32_t* err) {
     const uint32_t tiles = heads_tiles(n_items);
     if (tiles) {
         Timed timed(L, K_HEADS_COUNT);
@@ -161,7 +170,7 @@ cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_ite
     }
     if (tiles) {
         Timed timed(L, K_HEADS_WRITE);
-        k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, err);
+        k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, rec, terms, err);
     }
     return cudaGetLastError();
 }
@@ -170,6 +179,7 @@ cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_ite
 // per-row sums
 // ---------------------------------------------------------------------------------------------
 constexpr int kTermsInFlight = 4;
+constexpr int kReduceThreads = 128;
 
 // One lane's share of a row sum: fp64 accumulators for its NV float4 slices.
 template <int NV>
@@ -181,66 +191,89 @@ struct RowSum {
     }
 };
 
-// Adds coefficient * source over sorted[beg, end) in item order.  Sources and coefficients are fp32;
-// products and sums are taken in fp64, so the result does not feel the cancellation between the
-// positive and negative terms of a row.
+// Adds coefficient * source over terms[beg, end) in order.  A warp fetches up to 32 terms with one
+// coalesced load and hands them round by shuffle; the fp32 source rows of four terms are in flight
+// together.  Products and sums are taken in fp64, so the result does not feel the cancellation
+// between the positive and negative terms of a row.
 template <int NV>
-__device__ inline void accumulate_segment(const item_t* __restrict__ sorted, uint32_t beg, uint32_t end, bool input_row,
-                                          const Rec* __restrict__ rec, const double* __restrict__ gin_pos,
-                                          const float4* __restrict__ table, uint32_t d4, uint32_t stride4,
-                                          uint32_t lane, RowSum<NV>& sum) {
-    if (input_row) {
-        // sources are the fp64 partial centre gradients of the positions holding this token
-        for (uint32_t i = beg; i < end; ++i) {
-            const double2* src = reinterpret_cast<const double2*>(gin_pos + (size_t)item_payload(sorted[i]) * stride4 * 4);
+__device__ inline void accumulate_segment(const Rec* __restrict__ terms, uint32_t beg, uint32_t end, bool input_row,
+                                          const double* __restrict__ gin_pos, const float4* __restrict__ table,
+                                          uint32_t d4, uint32_t stride4, uint32_t lane, RowSum<NV>& sum,
+                                          bool have_first = false, Rec first = Rec{0.0, 0u, 0u}) {
+    for (uint32_t base = beg; base < end; base += 32) {
+        const uint32_t cnt = end - base < 32 ? end - base : 32;
+        Rec mine = Rec{0.0, 0u, 0u};
+        if (have_first && base == beg) mine = first;   // the caller fetched the first 32 terms ahead of time
+        else if (lane < cnt) mine = terms[base + lane];
+        if (input_row) {
+            // sources are the fp64 partial centre gradients of the positions holding this token
+            for (uint32_t t = 0; t < cnt; ++t) {
+                const uint32_t q = __shfl_sync(0xFFFFFFFFu, mine.centre, t);
+                const double2* src = reinterpret_cast<const double2*>(gin_pos + (size_t)q * stride4 * 4);
 #pragma unroll
-            for (int j = 0; j < NV; ++j) {
-                const uint32_t e = lane + 32 * j;
-                if (e < d4) {
-                    const double2 lo = src[2 * e], hi = src[2 * e + 1];
-                    sum.a[j][0] += lo.x; sum.a[j][1] += lo.y; sum.a[j][2] += hi.x; sum.a[j][3] += hi.y;
+                for (int j = 0; j < NV; ++j) {
+                    const uint32_t e = lane + 32 * j;
+                    if (e < d4) {
+                        const double2 lo = src[2 * e], hi = src[2 * e + 1];
+                        sum.a[j][0] += lo.x; sum.a[j][1] += lo.y; sum.a[j][2] += hi.x; sum.a[j][3] += hi.y;
+                    }
                 }
             }
+            continue;
         }
-        return;
-    }
-    for (uint32_t i0 = beg; i0 < end; i0 += kTermsInFlight) {
-        const float4* src[kTermsInFlight];
-        double coef[kTermsInFlight];
+        for (uint32_t t0 = 0; t0 < cnt; t0 += kTermsInFlight) {
+            const float4* src[kTermsInFlight];
+            double coef[kTermsInFlight];
 #pragma unroll
-        for (int t = 0; t < kTermsInFlight; ++t) {
-            coef[t] = 0.0;
-            src[t] = table;
-            if (i0 + t < end) {
-                const Rec r = rec[item_payload(sorted[i0 + t])];
-                coef[t] = r.g;
-                src[t] = table + (size_t)r.centre * stride4;
+            for (int t = 0; t < kTermsInFlight; ++t) {
+                const uint32_t from = (t0 + t) & 31;
+                const double g = __shfl_sync(0xFFFFFFFFu, mine.g, from);
+                const uint32_t centre = __shfl_sync(0xFFFFFFFFu, mine.centre, from);
+                const bool on = t0 + t < cnt;
+                coef[t] = on ? g : 0.0;
+                src[t] = table + (size_t)(on ? centre : 0u) * stride4;
             }
+            float4 x[kTermsInFlight][NV];
+#pragma unroll
+            for (int t = 0; t < kTermsInFlight; ++t)
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const uint32_t e = lane + 32 * i;
+                    x[t][i] = (t0 + t < cnt && e < d4) ? src[t][e] : make_float4(0.f, 0.f, 0.f, 0.f);
+                }
+#pragma unroll
+            for (int t = 0; t < kTermsInFlight; ++t)
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    sum.a[i][0] = fma(coef[t], (double)x[t][i].x, sum.a[i][0]);
+                    sum.a[i][1] = fma(coef[t], (double)x[t][i].y, sum.a[i][1]);
+                    sum.a[i][2] = fma(coef[t], (double)x[t][i].z, sum.a[i][2]);
+                    sum.a[i][3] = fma(coef[t], (double)x[t][i].w, sum.a[i][3]);
+                }
         }
-        float4 x[kTermsInFlight][NV];
-#pragma unroll
-        for (int t = 0; t < kTermsInFlight; ++t)
-#pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                const uint32_t e = lane + 32 * i;
-                x[t][i] = (i0 + t < end && e < d4) ? src[t][e] : make_float4(0.f, 0.f, 0.f, 0.f);
-            }
-#pragma unroll
-        for (int t = 0; t < kTermsInFlight; ++t)
-#pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                sum.a[i][0] = fma(coef[t], (double)x[t][i].x, sum.a[i][0]);
-                sum.a[i][1] = fma(coef[t], (double)x[t][i].y, sum.a[i][1]);
-                sum.a[i][2] = fma(coef[t], (double)x[t][i].z, sum.a[i][2]);
-                sum.a[i][3] = fma(coef[t], (double)x[t][i].w, sum.a[i][3]);
-            }
     }
 }
 
+// The table row of an output id, fetched before the sum starts so that its latency hides behind the sum.
+template <int NV>
+struct RowPrefetch {
+    float4 r[NV];
+    __device__ inline void load(const float4* __restrict__ table, uint32_t id, uint32_t V, uint32_t d4, uint32_t stride4,
+                                uint32_t lane) {
+        if (id >= V) {
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const uint32_t e = lane + 32 * i;
+                if (e < d4) r[i] = table[(size_t)id * stride4 + e];
+            }
+        }
+    }
+};
+
 // delta = fp32(-scale * sum); the delta row goes into the message and, for an output row, onto the table.
 template <int NV>
-__device__ inline void finish_row(const RowSum<NV>& sum, uint32_t m, uint32_t id, uint32_t V, double scale,
-                                  float4* __restrict__ table, float4* __restrict__ delta, uint32_t d4,
+__device__ inline void finish_row(const RowSum<NV>& sum, const RowPrefetch<NV>& old, uint32_t m, uint32_t id, uint32_t V,
+                                  double scale, float4* __restrict__ table, float4* __restrict__ delta, uint32_t d4,
                                   uint32_t stride4, uint32_t lane) {
     const double nlr = -scale;
 #pragma unroll
@@ -251,7 +284,7 @@ __device__ inline void finish_row(const RowSum<NV>& sum, uint32_t m, uint32_t id
                                           (float)(nlr * sum.a[i][2]), (float)(nlr * sum.a[i][3]));
             delta[(size_t)m * stride4 + e] = dl;
             if (id >= V) {
-                float4 t = table[(size_t)id * stride4 + e];
+                float4 t = old.r[i];
                 t.x += dl.x; t.y += dl.y; t.z += dl.z; t.w += dl.w;
                 table[(size_t)id * stride4 + e] = t;
             }
@@ -259,10 +292,13 @@ __device__ inline void finish_row(const RowSum<NV>& sum, uint32_t m, uint32_t id
     }
 }
 
+// One warp per message row, rows taken in a grid-stride loop that is software-pipelined over three
+// rows: while row i is summed, the terms and the old table row of row i+1 and the segment bounds of
+// row i+2 are already on their way, so only the gathers of the source rows are waited for.
 template <int NV>
-__global__ void __launch_bounds__(256)
-k_reduce_rows(const item_t* __restrict__ sorted, const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids,
-              const uint32_t* __restrict__ seg_start, const Rec* __restrict__ rec, const double* __restrict__ gin_pos,
+__global__ void __launch_bounds__(kReduceThreads)
+k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids,
+              const uint32_t* __restrict__ seg_start, const double* __restrict__ gin_pos,
               float4* __restrict__ table, float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4,
               double scale, uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows,
               ChunkItem* __restrict__ chunk_items) {
@@ -270,11 +306,31 @@ k_reduce_rows(const item_t* __restrict__ sorted, const MsgHeader* __restrict__ h
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const uint32_t n_rows = hdr->n_rows;
-    for (uint32_t m = warp; m < n_rows; m += nwarps) {
-        const uint32_t beg = seg_start[m], end = seg_start[m + 1];
-        const uint32_t id = ids[m];
-        if (end - beg > kChunk) {
-            const uint32_t nch = (end - beg + kChunk - 1) / kChunk;
+    struct Meta { uint32_t beg, end, id; };
+    auto load_meta = [&](uint32_t m) {
+        Meta x{0u, 0u, 0u};
+        if (m < n_rows) { x.beg = seg_start[m]; x.end = seg_start[m + 1]; x.id = ids[m]; }
+        return x;
+    };
+    auto load_terms = [&](const Meta& x) {
+        Rec r{0.0, 0u, 0u};
+        if (x.end - x.beg <= kChunk && x.beg + lane < x.end) r = terms[x.beg + lane];
+        return r;
+    };
+    uint32_t m = warp;
+    Meta cur = load_meta(m), nxt = load_meta(m + nwarps);
+    Rec cur_terms = load_terms(cur);
+    RowPrefetch<NV> cur_old;
+    if (m < n_rows && cur.end - cur.beg <= kChunk) cur_old.load(table, cur.id, V, d4, stride4, lane);
+    for (; m < n_rows; m += nwarps) {
+        // stage the next two rows
+        const Meta after = load_meta(m + 2 * nwarps);
+        const Rec nxt_terms = load_terms(nxt);
+        RowPrefetch<NV> nxt_old;
+        if (m + nwarps < n_rows && nxt.end - nxt.beg <= kChunk) nxt_old.load(table, nxt.id, V, d4, stride4, lane);
+
+        if (cur.end - cur.beg > kChunk) {
+            const uint32_t nch = (cur.end - cur.beg + kChunk - 1) / kChunk;
             uint32_t base = 0;
             if (lane == 0) {
                 const uint32_t slot = atomicAdd(long_counters, 1u);
@@ -283,20 +339,25 @@ k_reduce_rows(const item_t* __restrict__ sorted, const MsgHeader* __restrict__ h
             }
             base = __shfl_sync(0xFFFFFFFFu, base, 0);
             for (uint32_t c = lane; c < nch; c += 32) chunk_items[base + c] = ChunkItem{m, c};
-            continue;
+        } else {
+            RowSum<NV> sum;
+            sum.clear();
+            accumulate_segment<NV>(terms, cur.beg, cur.end, cur.id < V, gin_pos, table, d4, stride4, lane, sum, true,
+                                   cur_terms);
+            finish_row<NV>(sum, cur_old, m, cur.id, V, scale, table, delta, d4, stride4, lane);
         }
-        RowSum<NV> sum;
-        sum.clear();
-        accumulate_segment<NV>(sorted, beg, end, id < V, rec, gin_pos, table, d4, stride4, lane, sum);
-        finish_row<NV>(sum, m, id, V, scale, table, delta, d4, stride4, lane);
+        cur = nxt;
+        nxt = after;
+        cur_terms = nxt_terms;
+        cur_old = nxt_old;
     }
 }
 
 // Partial sums of the chunks of long rows, one warp per chunk; partials are kept in fp64.
 template <int NV>
-__global__ void __launch_bounds__(256)
-k_reduce_chunks(const item_t* __restrict__ sorted, const uint32_t* __restrict__ ids, const uint32_t* __restrict__ seg_start,
-                const Rec* __restrict__ rec, const double* __restrict__ gin_pos, const float4* __restrict__ table,
+__global__ void __launch_bounds__(kReduceThreads)
+k_reduce_chunks(const Rec* __restrict__ terms, const uint32_t* __restrict__ ids, const uint32_t* __restrict__ seg_start,
+                const double* __restrict__ gin_pos, const float4* __restrict__ table,
                 uint32_t V, uint32_t d4, uint32_t stride4, const uint32_t* __restrict__ long_counters,
                 const ChunkItem* __restrict__ chunk_items, double* __restrict__ partials) {
     const uint32_t lane = threadIdx.x & 31;
@@ -310,7 +371,7 @@ k_reduce_chunks(const item_t* __restrict__ sorted, const uint32_t* __restrict__ 
         const uint32_t end = beg + kChunk < seg_end ? beg + kChunk : seg_end;
         RowSum<NV> sum;
         sum.clear();
-        accumulate_segment<NV>(sorted, beg, end, ids[ci.m] < V, rec, gin_pos, table, d4, stride4, lane, sum);
+        accumulate_segment<NV>(terms, beg, end, ids[ci.m] < V, gin_pos, table, d4, stride4, lane, sum);
         double* out = partials + (size_t)x * stride4 * 4;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -325,7 +386,7 @@ k_reduce_chunks(const item_t* __restrict__ sorted, const uint32_t* __restrict__ 
 
 // Long rows: the chunk partials are added in chunk order, then the row is finished like a short one.
 template <int NV>
-__global__ void __launch_bounds__(256)
+__global__ void __launch_bounds__(kReduceThreads)
 k_reduce_long(const uint32_t* __restrict__ ids, const double* __restrict__ partials, float4* __restrict__ table,
               float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4, double scale,
               const uint32_t* __restrict__ long_counters, const LongRow* __restrict__ long_rows) {
@@ -335,6 +396,9 @@ k_reduce_long(const uint32_t* __restrict__ ids, const double* __restrict__ parti
     const uint32_t n_long = long_counters[0];
     for (uint32_t x = warp; x < n_long; x += nwarps) {
         const LongRow row = long_rows[x];
+        const uint32_t id = ids[row.m];
+        RowPrefetch<NV> old;
+        old.load(table, id, V, d4, stride4, lane);
         RowSum<NV> sum;
         sum.clear();
         for (uint32_t c = 0; c < row.nchunks; ++c) {
@@ -348,43 +412,43 @@ k_reduce_long(const uint32_t* __restrict__ ids, const double* __restrict__ parti
                 }
             }
         }
-        finish_row<NV>(sum, row.m, ids[row.m], V, scale, table, delta, d4, stride4, lane);
+        finish_row<NV>(sum, old, row.m, id, V, scale, table, delta, d4, stride4, lane);
     }
 }
 
 template <int NV>
-static cudaError_t reduce_all(const Launcher& L, const item_t* sorted, const MsgHeader* hdr, const uint32_t* ids,
-                              const uint32_t* seg_start, const Rec* rec, const double* gin_pos, float* table,
+static cudaError_t reduce_all(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
+                              const uint32_t* seg_start, const double* gin_pos, float* table,
                               float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
                               ChunkItem* chunk_items, double* partials) {
     const uint32_t stride4 = s.stride / 4;
-    const int blocks = L.sms * 8;
+    const int blocks = L.sms * 16;
     float4* t4 = reinterpret_cast<float4*>(table);
     float4* d4p = reinterpret_cast<float4*>(delta);
     {
     Timed timed(L, K_REDUCE_ROWS);
-    k_reduce_rows<NV><<<blocks, 256, 0, L.stream>>>(sorted, hdr, ids, seg_start, rec, gin_pos, t4, d4p, s.V, s.d4, stride4,
+    k_reduce_rows<NV><<<blocks, kReduceThreads, 0, L.stream>>>(terms, hdr, ids, seg_start, gin_pos, t4, d4p, s.V, s.d4, stride4,
                                                     scale, long_counters, long_rows, chunk_items);
     }
     {
     Timed timed(L, K_REDUCE_CHUNKS);
-    k_reduce_chunks<NV><<<blocks, 256, 0, L.stream>>>(sorted, ids, seg_start, rec, gin_pos, t4, s.V, s.d4, stride4,
+    k_reduce_chunks<NV><<<blocks, kReduceThreads, 0, L.stream>>>(terms, ids, seg_start, gin_pos, t4, s.V, s.d4, stride4,
                                                       long_counters, chunk_items, partials);
     }
     {
     Timed timed(L, K_REDUCE_LONG);
-    k_reduce_long<NV><<<L.sms * 2, 256, 0, L.stream>>>(ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters,
+    k_reduce_long<NV><<<L.sms * 4, kReduceThreads, 0, L.stream>>>(ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters,
                                                        long_rows);
     }
     return cudaGetLastError();
 }
 
-cudaError_t launch_reduce(const Launcher& L, const item_t* sorted, const MsgHeader* hdr, const uint32_t* ids,
-                          const uint32_t* seg_start, const Rec* rec, const double* gin_pos, float* table,
+cudaError_t launch_reduce(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
+                          const uint32_t* seg_start, const double* gin_pos, float* table,
                           float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
                           ChunkItem* chunk_items, double* partials) {
 #define TENSAIR_RED(NV) \
-    return reduce_all<NV>(L, sorted, hdr, ids, seg_start, rec, gin_pos, table, delta, s, scale, long_counters, long_rows, \
+    return reduce_all<NV>(L, terms, hdr, ids, seg_start, gin_pos, table, delta, s, scale, long_counters, long_rows, \
                           chunk_items, partials)
     if (s.d4 <= 32) TENSAIR_RED(1);
     if (s.d4 <= 64) TENSAIR_RED(2);

@@ -34,17 +34,24 @@ k_radix_hist(const item_t* __restrict__ in, uint32_t n, uint32_t shift, uint32_t
     hist[threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];   // digit-major
 }
 
-// Exclusive scan, in place, of `count` words by one block.
+// Exclusive scan, in place, of `count` words by one block; every thread takes 8 consecutive words per round.
+constexpr int kScanPerThread = 8;
 __global__ void __launch_bounds__(1024) k_scan_exclusive(uint32_t* __restrict__ data, uint32_t count) {
     __shared__ uint32_t warp_tot[32];
     __shared__ uint32_t carry_s;
     if (threadIdx.x == 0) carry_s = 0;
     __syncthreads();
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (uint32_t base = 0; base < count; base += 1024) {
-        const uint32_t idx = base + threadIdx.x;
-        const uint32_t v = idx < count ? data[idx] : 0;
-        uint32_t incl = v;
+    for (uint32_t base = 0; base < count; base += 1024 * kScanPerThread) {
+        const uint32_t first = base + threadIdx.x * kScanPerThread;
+        uint32_t v[kScanPerThread];
+        uint32_t sum = 0;
+#pragma unroll
+        for (int i = 0; i < kScanPerThread; ++i) {
+            v[i] = first + i < count ? data[first + i] : 0;
+            sum += v[i];
+        }
+        uint32_t incl = sum;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
@@ -64,9 +71,14 @@ __global__ void __launch_bounds__(1024) k_scan_exclusive(uint32_t* __restrict__ 
         }
         __syncthreads();
         const uint32_t carry = carry_s;
-        if (idx < count) data[idx] = carry + warp_tot[wid] + incl - v;
+        uint32_t run = carry + warp_tot[wid] + incl - sum;
+#pragma unroll
+        for (int i = 0; i < kScanPerThread; ++i) {
+            if (first + i < count) data[first + i] = run;
+            run += v[i];
+        }
         __syncthreads();
-        if (threadIdx.x == 1023) carry_s = carry + warp_tot[wid] + incl;
+        if (threadIdx.x == 1023) carry_s = run;
         __syncthreads();
     }
 }

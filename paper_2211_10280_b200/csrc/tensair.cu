@@ -18,7 +18,7 @@ uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 
 // Offsets (bytes) of everything the library keeps in the caller's scratch buffer.
 struct Carve {
-    uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, gin_pos, loss_pos, hist,
+    uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, terms, gin_pos, loss_pos, hist,
         tile_counts, seg_start, long_rows, chunk_items, partials, total;
     uint64_t slot_bytes, ids_off, delta_off;
     uint32_t stride, max_pairs, max_contrib, max_items, max_rows, max_long, max_chunks;
@@ -62,6 +62,7 @@ void carve(const tensair_config& c, Carve& k) {
     k.items_a = take((uint64_t)k.max_items * 8);
     k.items_b = take((uint64_t)k.max_items * 8);
     k.rec = take((uint64_t)k.max_contrib * sizeof(Rec));
+    k.terms = take((uint64_t)k.max_items * sizeof(Rec));
     k.gin_pos = take((uint64_t)c.batch * k.stride * 8);
     k.loss_pos = take((uint64_t)c.batch * 8);
     k.hist = take((uint64_t)sort_hist_words(k.max_items) * 4);
@@ -184,9 +185,10 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                                       bits_for(2 * c.V), ctx->at<uint32_t>(cv.hist), &sorted));
         TENSAIR_CUDA(ctx, launch_heads(ctx->L, sorted, n_items, c.V, ctx->at<uint32_t>(cv.tile_counts), hdr,
                                        ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
-                                       ctx->at<uint32_t>(cv.long_counters), err));
-        TENSAIR_CUDA(ctx, launch_reduce(ctx->L, sorted, hdr, ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
-                                        ctx->at<Rec>(cv.rec), ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot),
+                                       ctx->at<uint32_t>(cv.long_counters), ctx->at<Rec>(cv.rec),
+                                       ctx->at<Rec>(cv.terms), err));
+        TENSAIR_CUDA(ctx, launch_reduce(ctx->L, ctx->at<Rec>(cv.terms), hdr, ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
+                                        ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot),
                                         ctx->shape, scale, ctx->at<uint32_t>(cv.long_counters),
                                         ctx->at<LongRow>(cv.long_rows), ctx->at<ChunkItem>(cv.chunk_items),
                                         ctx->at<double>(cv.partials)));
