@@ -137,6 +137,8 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     wl = pick_workload(args.workload, args.override)
+    for item in filter(None, args.tune.split(",")):
+        B.tensair_tune(item.split("=")[0], int(item.split("=")[1]))
     K, Wm = args.steps, max(args.warmup, 3)
     Kp = min(K, 8)                                          # steps of the per-kernel timing pass
     total_steps = 2 * (Wm + K) + Kp
@@ -361,6 +363,7 @@ def main():
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--workload", default=synth.LARGE_DASGD.name)
     ap.add_argument("--override", default="", help="comma-separated field=value replacements of the workload")
+    ap.add_argument("--tune", default="", help="comma-separated knob=value pairs passed to tensair_tune (sweeps)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
     if args.impl == "reference":

@@ -80,6 +80,7 @@ SYMBOLS = {
     "tensair_pending": (_int, [_vp, _u32, _P(_u64)]),
     "tensair_kernel_launches": (_u64, [_vp]),
     "tensair_profile": (_int, [_vp, _int]),
+    "tensair_tune": (_int, [C.c_char_p, _int]),
     "tensair_profile_read": (_int, [_vp, _u32, _vp, _P(_u32)]),
     "tensair_strerror": (C.c_char_p, [_int]),
     "tensair_last_error": (C.c_char_p, [_vp]),
@@ -146,6 +147,10 @@ def tensair_philox4x32_10(counter, key):
     o = (C.c_uint32 * 4)()
     lib().tensair_philox4x32_10(c, k, o)
     return [int(x) for x in o]
+
+
+def tensair_tune(name: str, value: int):
+    _check(lib().tensair_tune(name.encode(), value), "tensair_tune")
 
 
 def tensair_delay(seed: int, max_delay: int, step: int, sender: int, receiver: int) -> int:

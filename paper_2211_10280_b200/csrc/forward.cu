@@ -44,7 +44,6 @@ __device__ inline double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
 // -log(sigmoid(x)) without overflow
 __device__ inline double neg_log_sigmoid(double x) { return (x < 0.0 ? -x : 0.0) + log1p(exp(-fabs(x))); }
 
-constexpr int kChunkRows = 16;     // output rows a warp stages and reduces together
 constexpr int kFwdWarps = 2;       // warps per block
 
 // One warp per centre position (grid-stride), no block-level cooperation.  For every pair of the
@@ -55,7 +54,8 @@ constexpr int kFwdWarps = 2;       // warps per block
 //   3. evaluates sigmoid and loss for all rows at once (one row per lane pair instead of one per warp),
 //   4. re-reads the staged rows and adds g * u to the centre gradient kept in registers.
 // The centre gradient is written once per position; nothing is shared between warps.
-template <int NV>
+// NV: float4 slices per lane.  CR: rows reduced together (16 or 8); 32 / CR lanes share a row's scalar.
+template <int NV, int CR>
 __global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, uint32_t stride4, uint32_t w,
           uint32_t k, uint32_t chunk_rows, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
@@ -113,9 +113,9 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                 parity ^= 1;
 
                 // 1. partial dot products of the staged rows
-                double xp[kChunkRows];
+                double xp[CR];
 #pragma unroll
-                for (int j = 0; j < kChunkRows; ++j) {
+                for (int j = 0; j < CR; ++j) {
                     xp[j] = 0.0;
                     if ((live >> j) & 1u) {
                         const float4* __restrict__ u = stage + (size_t)j * stride4;
@@ -132,45 +132,35 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                         }
                     }
                 }
-                // 2. transposing reduction: after it lanes 2j and 2j+1 hold the dot product of row j
+                // 2. transposing reduction: after it the 32 / CR lanes [j * LPR, (j + 1) * LPR) hold the dot product of row j
+                constexpr int LPR = 32 / CR;
 #pragma unroll
-                for (int i = 0; i < 8; ++i) {
-                    const bool up = lane & 16;
-                    const double keep = up ? xp[8 + i] : xp[i], give = up ? xp[i] : xp[8 + i];
-                    xp[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 16);
-                }
+                for (int h = CR / 2, off = 16; h >= 1; h >>= 1, off >>= 1) {
+                    const bool up = lane & off;
 #pragma unroll
-                for (int i = 0; i < 4; ++i) {
-                    const bool up = lane & 8;
-                    const double keep = up ? xp[4 + i] : xp[i], give = up ? xp[i] : xp[4 + i];
-                    xp[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 8);
+                    for (int i = 0; i < h; ++i) {
+                        const double keep = up ? xp[h + i] : xp[i], give = up ? xp[i] : xp[h + i];
+                        xp[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, off);
+                    }
                 }
+                double x = xp[0];
 #pragma unroll
-                for (int i = 0; i < 2; ++i) {
-                    const bool up = lane & 4;
-                    const double keep = up ? xp[2 + i] : xp[i], give = up ? xp[i] : xp[2 + i];
-                    xp[i] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 4);
-                }
-                {
-                    const bool up = lane & 2;
-                    const double keep = up ? xp[1] : xp[0], give = up ? xp[0] : xp[1];
-                    xp[0] = keep + __shfl_xor_sync(0xFFFFFFFFu, give, 2);
-                }
-                const double x = xp[0] + __shfl_xor_sync(0xFFFFFFFFu, xp[0], 1);
-                // 3. gradient scalar and loss of row (lane / 2), all rows at once
-                const uint32_t jr = lane >> 1;
+                for (int off = LPR / 2; off >= 1; off >>= 1) x += __shfl_xor_sync(0xFFFFFFFFu, x, off);
+                // 3. gradient scalar and loss of row (lane / LPR), all rows at once
+                const uint32_t jr = lane / LPR;
+                const bool writer = (lane % LPR) == 0;
                 double g = 0.0;
                 if ((live >> jr) & 1u) {
                     const bool positive = j0 + jr == 0;
                     const double sig = sigmoid(x);
                     g = positive ? sig - 1.0 : sig;
-                    if (!(lane & 1)) loss += neg_log_sigmoid(positive ? x : -x);
+                    if (writer) loss += neg_log_sigmoid(positive ? x : -x);
                 }
-                if (!(lane & 1) && jr < nr) rec[cbase + j0 + jr] = Rec{g, centre, 0u};
+                if (writer && jr < nr) rec[cbase + j0 + jr] = Rec{g, centre, 0u};
                 // 4. centre gradient: acc += g_j * u_j
 #pragma unroll
-                for (int j = 0; j < kChunkRows; ++j) {
-                    const double gj = __shfl_sync(0xFFFFFFFFu, g, 2 * j);
+                for (int j = 0; j < CR; ++j) {
+                    const double gj = __shfl_sync(0xFFFFFFFFu, g, LPR * j);
                     if ((live >> j) & 1u) {
                         const float4* __restrict__ u = stage + (size_t)j * stride4;
 #pragma unroll
@@ -205,43 +195,52 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
     if (failed && lane == 0) atomicOr(err, 2u);
 }
 
-// Rows per staging chunk and bytes of dynamic shared memory per block.
-static uint32_t forward_chunk_rows(const Shape& s, size_t* smem) {
-    const size_t budget = 200 * 1024 / 5;          // five blocks per multiprocessor
-    const size_t row = (size_t)s.stride * 4;
-    uint32_t r = s.K1 < (uint32_t)kChunkRows ? s.K1 : (uint32_t)kChunkRows;
-    while (r > 1 && (size_t)kFwdWarps * r * row + kFwdWarps * 8 > budget) --r;
-    *smem = (size_t)kFwdWarps * r * row + kFwdWarps * 8;
-    return r;
+// Launch shape of the forward kernel: rows reduced together (8 by default: less shared memory per warp, so
+// more resident warps; or 16) and blocks per multiprocessor; both can be overridden for sweeps.
+static int g_forward_rows = 0;     // 0 = choose
+static int g_forward_blocks = 0;   // 0 = choose
+void set_forward_shape(int rows, int blocks_per_sm) {
+    g_forward_rows = rows;
+    g_forward_blocks = blocks_per_sm;
 }
 
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err) {
     if (n < 2) return cudaSuccess;
-    size_t smem = 0;
-    const uint32_t chunk_rows = forward_chunk_rows(s, &smem);
+    const size_t row = (size_t)s.stride * 4;
+    const int cr = g_forward_rows == 8 || g_forward_rows == 16 ? g_forward_rows : 8;
+    int blocks_per_sm = g_forward_blocks > 0 ? g_forward_blocks : (cr == 16 ? 5 : 8);
+    // rows staged per chunk: as many of the cr as fit the shared memory share of one block
+    uint32_t chunk_rows = s.K1 < (uint32_t)cr ? s.K1 : (uint32_t)cr;
+    const size_t budget = (size_t)216 * 1024 / blocks_per_sm - 1024;
+    while (chunk_rows > 1 && (size_t)kFwdWarps * chunk_rows * row + kFwdWarps * 8 > budget) --chunk_rows;
+    const size_t smem = (size_t)kFwdWarps * chunk_rows * row + kFwdWarps * 8;
+    if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
     const uint32_t stride4 = s.stride / 4;
     const float4* t4 = reinterpret_cast<const float4*>(table);
     uint32_t blocks = (n + kFwdWarps - 1) / kFwdWarps;
-    const uint32_t resident = (uint32_t)L.sms * 5;
+    const uint32_t resident = (uint32_t)(L.sms * blocks_per_sm);
     if (blocks > resident) blocks = resident;
     Timed timed(L, K_FORWARD);
-#define TENSAIR_FWD(NV)                                                                                         \
+#define TENSAIR_FWD(NV, CR)                                                                                     \
     do {                                                                                                        \
         static bool attr_set = false;                                                                           \
         if (!attr_set) {                                                                                        \
-            cudaFuncSetAttribute(k_forward<NV>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);       \
-            cudaFuncSetAttribute(k_forward<NV>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);           \
+            cudaFuncSetAttribute(k_forward<NV, CR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);   \
+            cudaFuncSetAttribute(k_forward<NV, CR>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);       \
             attr_set = true;                                                                                    \
         }                                                                                                       \
-        k_forward<NV><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k, chunk_rows, \
-                                                                  t4, rows, rec, gin_pos, loss_pos, err);       \
+        k_forward<NV, CR><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,     \
+                                                                      chunk_rows, t4, rows, rec, gin_pos,      \
+                                                                      loss_pos, err);                           \
     } while (0)
-    if (s.d4 <= 32) TENSAIR_FWD(1);
-    else if (s.d4 <= 64) TENSAIR_FWD(2);
-    else if (s.d4 <= 96) TENSAIR_FWD(3);
-    else if (s.d4 <= 128) TENSAIR_FWD(4);
-    else TENSAIR_FWD(8);
+#define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else TENSAIR_FWD(NV, 8); } while (0)
+    if (s.d4 <= 32) TENSAIR_FWD_NV(1);
+    else if (s.d4 <= 64) TENSAIR_FWD_NV(2);
+    else if (s.d4 <= 96) TENSAIR_FWD_NV(3);
+    else if (s.d4 <= 128) TENSAIR_FWD_NV(4);
+    else TENSAIR_FWD_NV(8);
+#undef TENSAIR_FWD_NV
 #undef TENSAIR_FWD
     return cudaGetLastError();
 }

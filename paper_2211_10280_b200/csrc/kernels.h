@@ -76,6 +76,7 @@ uint32_t sort_hist_words(uint32_t n);
 // forward.cu
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err);
+void set_forward_shape(int rows, int blocks_per_sm);
 cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err);
 
 // message.cu

@@ -1,7 +1,7 @@
 // Stable least-significant-digit radix sort of 64-bit items by (a bit range of) their 32-bit keys.
 //
 // Keys are row ids, dense in [0, 2V], so few digit passes are needed.  Every pass is three kernels:
-// per-tile digit histogram, exclusive scan of the digit-major histogram, stable scatter.  Stability
+// per-tile digit histogram, per-digit scan over the tiles (one warp per digit), stable scatter.  Stability
 // (equal keys keep their input order) is what makes the later per-row sums run in a fixed order.
 // The whole working set (two item buffers) stays in L2 at the sizes of interest.
 #include "kernels.h"
@@ -17,7 +17,7 @@ constexpr int kTile = kSortThreads * kItemsPerThread;   // 4096 items per block
 constexpr int kWarpSpan = 32 * kItemsPerThread;         // consecutive items owned by one warp
 
 uint32_t sort_tiles(uint32_t n) { return (n + kTile - 1) / kTile; }
-uint32_t sort_hist_words(uint32_t n) { return sort_tiles(n) * kBins; }
+uint32_t sort_hist_words(uint32_t n) { return (sort_tiles(n) + 1) * kBins; }   // per-tile counts, then digit totals
 
 __global__ void __launch_bounds__(kSortThreads)
 k_radix_hist(const item_t* __restrict__ in, uint32_t n, uint32_t shift, uint32_t* __restrict__ hist, uint32_t tiles) {
@@ -34,53 +34,27 @@ k_radix_hist(const item_t* __restrict__ in, uint32_t n, uint32_t shift, uint32_t
     hist[threadIdx.x * tiles + blockIdx.x] = h[threadIdx.x];   // digit-major
 }
 
-// Exclusive scan, in place, of `count` words by one block; every thread takes 8 consecutive words per round.
-constexpr int kScanPerThread = 8;
-__global__ void __launch_bounds__(1024) k_scan_exclusive(uint32_t* __restrict__ data, uint32_t count) {
-    __shared__ uint32_t warp_tot[32];
-    __shared__ uint32_t carry_s;
-    if (threadIdx.x == 0) carry_s = 0;
-    __syncthreads();
-    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (uint32_t base = 0; base < count; base += 1024 * kScanPerThread) {
-        const uint32_t first = base + threadIdx.x * kScanPerThread;
-        uint32_t v[kScanPerThread];
-        uint32_t sum = 0;
-#pragma unroll
-        for (int i = 0; i < kScanPerThread; ++i) {
-            v[i] = first + i < count ? data[first + i] : 0;
-            sum += v[i];
-        }
-        uint32_t incl = sum;
+// Per digit: exclusive scan, in place, of its per-tile counts (one warp per digit), and the digit's total.
+constexpr int kScanWarps = 8;
+__global__ void __launch_bounds__(kScanWarps * 32)
+k_scan_digits(uint32_t* __restrict__ hist, uint32_t tiles, uint32_t* __restrict__ totals) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t digit = blockIdx.x * kScanWarps + (threadIdx.x >> 5);
+    uint32_t* row = hist + (size_t)digit * tiles;
+    uint32_t carry = 0;
+    for (uint32_t base = 0; base < tiles; base += 32) {
+        const uint32_t idx = base + lane;
+        const uint32_t v = idx < tiles ? row[idx] : 0;
+        uint32_t incl = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
             const uint32_t t = __shfl_up_sync(0xFFFFFFFFu, incl, o);
             if (lane >= (uint32_t)o) incl += t;
         }
-        if (lane == 31) warp_tot[wid] = incl;
-        __syncthreads();
-        if (wid == 0) {
-            const uint32_t t = warp_tot[lane];
-            uint32_t ti = t;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, ti, o);
-                if (lane >= (uint32_t)o) ti += u;
-            }
-            warp_tot[lane] = ti - t;   // exclusive over warps
-        }
-        __syncthreads();
-        const uint32_t carry = carry_s;
-        uint32_t run = carry + warp_tot[wid] + incl - sum;
-#pragma unroll
-        for (int i = 0; i < kScanPerThread; ++i) {
-            if (first + i < count) data[first + i] = run;
-            run += v[i];
-        }
-        __syncthreads();
-        if (threadIdx.x == 1023) carry_s = run;
-        __syncthreads();
+        if (idx < tiles) row[idx] = carry + incl - v;
+        carry += __shfl_sync(0xFFFFFFFFu, incl, 31);
     }
+    if (lane == 0) totals[digit] = carry;
 }
 
 // Stable scatter.  Warp w of a block owns the consecutive items [w*512, (w+1)*512) of the tile and
@@ -88,8 +62,10 @@ __global__ void __launch_bounds__(1024) k_scan_exclusive(uint32_t* __restrict__ 
 // rounds are ranked by their order, so the rank of an item among equal digits follows input order.
 __global__ void __launch_bounds__(kSortThreads)
 k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_t n, uint32_t shift,
-                const uint32_t* __restrict__ hist, uint32_t tiles) {
+                const uint32_t* __restrict__ hist, uint32_t tiles, const uint32_t* __restrict__ totals) {
     __shared__ uint32_t cnt[kSortWarps][kBins];
+    __shared__ uint32_t digit_base[kBins];
+    __shared__ uint32_t warp_tot[kSortWarps];
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     for (int i = threadIdx.x; i < kSortWarps * kBins; i += kSortThreads) (&cnt[0][0])[i] = 0;
     __syncthreads();
@@ -119,10 +95,25 @@ k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_
         __syncwarp();
     }
     __syncthreads();
-    // per digit: global base of this tile, then exclusive prefix over the warps of the block
+    // exclusive scan of the digit totals: where each digit's run starts in the output
+    {
+        const uint32_t t = totals[threadIdx.x];
+        uint32_t incl = t;
+#pragma unroll
+        for (int o = 1; o < 32; o <<= 1) {
+            const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, incl, o);
+            if (lane >= (uint32_t)o) incl += u;
+        }
+        if (lane == 31) warp_tot[wid] = incl;
+        __syncthreads();
+        uint32_t before = 0;
+        for (uint32_t x = 0; x < wid; ++x) before += warp_tot[x];
+        digit_base[threadIdx.x] = before + incl - t;
+    }
+    // per digit: start of the digit, this tile's offset in it, then exclusive prefix over the warps of the block
     {
         const uint32_t digit = threadIdx.x;
-        uint32_t run = hist[digit * tiles + blockIdx.x];
+        uint32_t run = digit_base[digit] + hist[digit * tiles + blockIdx.x];
 #pragma unroll
         for (int w = 0; w < kSortWarps; ++w) {
             const uint32_t c = cnt[w][digit];
@@ -155,11 +146,11 @@ cudaError_t launch_sort(const Launcher& L, item_t* a, item_t* b, uint32_t n, uin
         }
         {
             Timed timed(L, K_SORT_SCAN);
-            k_scan_exclusive<<<1, 1024, 0, L.stream>>>(hist, tiles * kBins);
+            k_scan_digits<<<kBins / kScanWarps, kScanWarps * 32, 0, L.stream>>>(hist, tiles, hist + (size_t)tiles * kBins);
         }
         {
             Timed timed(L, K_SORT_SCATTER);
-            k_radix_scatter<<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles);
+            k_radix_scatter<<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles, hist + (size_t)tiles * kBins);
         }
         item_t* t = src; src = dst; dst = t;
     }

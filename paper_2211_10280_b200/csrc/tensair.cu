@@ -483,6 +483,16 @@ int tensair_pending(tensair_ctx* ctx, uint32_t replica, uint64_t* n) {
 
 uint64_t tensair_kernel_launches(const tensair_ctx* ctx) { return ctx ? ctx->launches : 0; }
 
+int tensair_tune(const char* name, int value) {
+    if (!name) return TENSAIR_EINVAL;
+    static int rows = 0, blocks = 0;
+    if (!std::strcmp(name, "forward_rows")) rows = value;
+    else if (!std::strcmp(name, "forward_blocks_per_sm")) blocks = value;
+    else return TENSAIR_EINVAL;
+    set_forward_shape(rows, blocks);
+    return TENSAIR_OK;
+}
+
 int tensair_profile(tensair_ctx* ctx, int enable) {
     if (!ctx) return TENSAIR_EINVAL;
     ctx->prof.on = enable != 0;
