@@ -39,6 +39,24 @@ METRIC = "SGNS (center,context) pairs/sec on 1 B200; achieved HBM GB/s vs peak"
 UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0
 
+# DRAM bytes (read + write) per message row of the message-apply kernel, from the ncu capture summarised in
+# profiles/k_apply_small_case_V250k_W2.md (780.3 MB for a 224.6 K-row message; the kernel is a pure stream,
+# so traffic is proportional to the rows of the message).  Only valid for the source the capture ran.
+NCU_TRAFFIC = {"apply_message": {"bytes_per_row": 3474.0, "source": "paper_2211_10280_b200/csrc/apply.cu",
+                                 "sha256": "aed4fc3b02cdefba7ba9880789b118ad30969231c9c0bae3c29f1c8253db1cf7"}}
+
+
+def ncu_traffic(kernel: str, rows: float):
+    rec = NCU_TRAFFIC.get(kernel)
+    if not rec:
+        return None
+    import hashlib
+
+    src = ROOT / rec["source"]
+    if not src.exists() or hashlib.sha256(src.read_bytes()).hexdigest() != rec["sha256"]:
+        return None          # the kernel changed since the counters were taken
+    return int(rec["bytes_per_row"] * rows)
+
 
 def hbm_peak():
     p = ROOT / "MEASURED_PEAKS.json"
@@ -252,7 +270,9 @@ def run_ours(args):
     peak, peak_kind = hbm_peak()
     achieved = kernels[dom]["gbs"]
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_source": f"of {peak_kind}",
-                "unit": "GB/s", "frac": round(achieved / peak, 4), "traffic": None,
+                "unit": "GB/s", "frac": round(achieved / peak, 4),
+                "traffic": ncu_traffic(dom, U_applied if dom == "apply_message" else U),
+                "algorithmic_bytes": kernels[dom]["algorithmic_bytes"],
                 "avg_ms": kernels[dom]["avg_ms"], "share_of_device_time": kernels[dom]["share"]}
     own = U * row + U * (row + 4) + U * (row + 4 + 2 * row)
     remote = (wl.W - 1) * U * (row + 4 + 2 * row)
