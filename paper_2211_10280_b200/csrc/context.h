@@ -1,0 +1,80 @@
+// The context behind the C ABI and the helpers every entry point shares.
+#pragma once
+#include <stdint.h>
+
+#include <string>
+
+#include "../../include/tensair.h"
+#include "kernels.h"
+#include "schedule.h"
+
+namespace tensair {
+
+inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
+
+// Offsets (bytes) of everything the library keeps in the caller's scratch buffer.
+struct Carve {
+    uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, terms, gin_pos, loss_pos, hist,
+        tile_counts, seg_start, long_rows, chunk_items, partials, total;
+    uint64_t slot_bytes, ids_off, delta_off;
+    uint32_t stride, max_pairs, max_contrib, max_items, max_rows, max_long, max_chunks;
+};
+
+inline uint32_t bits_for(uint32_t x) {   // bits needed to represent x
+    uint32_t b = 0;
+    while (x) { ++b; x >>= 1; }
+    return b ? b : 1;
+}
+
+}  // namespace tensair
+
+struct tensair_ctx {
+    tensair_config cfg;
+    tensair::Carve cv;
+    tensair::Shape shape;
+    cudaStream_t stream;
+    tensair::Launcher L;
+    uint64_t launches = 0;
+    tensair::Profiler prof;
+    float* tables;
+    uint8_t* pool;
+    uint8_t* scratch;
+    tensair::Schedule* sched = nullptr;
+    uint32_t last_n = 0, last_pairs = 0;
+    bool have_last = false;
+    std::string last_error;
+    // pinned host staging for small read-backs
+    struct Staging { tensair::MsgHeader hdr; double loss; uint32_t err; } *stage = nullptr;
+
+    template <class T> T* at(uint64_t off) const { return reinterpret_cast<T*>(scratch + off); }
+    float* table_of(uint32_t replica) const { return tables + (size_t)replica * 2 * cfg.V * cv.stride; }
+    uint8_t* slot_ptr(uint32_t slot) const { return pool + (size_t)slot * cv.slot_bytes; }
+    tensair::MsgHeader* slot_hdr(uint32_t slot) const { return reinterpret_cast<tensair::MsgHeader*>(slot_ptr(slot)); }
+    uint32_t* slot_ids(uint32_t slot) const { return reinterpret_cast<uint32_t*>(slot_ptr(slot) + cv.ids_off); }
+    float* slot_delta(uint32_t slot) const { return reinterpret_cast<float*>(slot_ptr(slot) + cv.delta_off); }
+};
+
+namespace tensair {
+
+// Records the CUDA error text on the context and returns TENSAIR_ECUDA.
+int fail(tensair_ctx* ctx, cudaError_t e, const char* what);
+// Waits for the stream, then reads and clears the device error flag.
+int collect(tensair_ctx* ctx);
+
+#define TENSAIR_CUDA(ctx, call)                                    \
+    do {                                                           \
+        const cudaError_t e_ = (call);                             \
+        if (e_ != cudaSuccess) return tensair::fail((ctx), e_, #call);      \
+    } while (0)
+
+struct DeviceGuard {
+    int prev = -1;
+    bool ok = true;
+    explicit DeviceGuard(int dev) {
+        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
+        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
+    }
+    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
+};
+
+}  // namespace tensair

@@ -7,22 +7,11 @@
 #include <string>
 #include <vector>
 
-#include "kernels.h"
-#include "schedule.h"
+#include "context.h"
 
 using namespace tensair;
 
 namespace {
-
-uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
-
-// Offsets (bytes) of everything the library keeps in the caller's scratch buffer.
-struct Carve {
-    uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, terms, gin_pos, loss_pos, hist,
-        tile_counts, seg_start, long_rows, chunk_items, partials, total;
-    uint64_t slot_bytes, ids_off, delta_off;
-    uint32_t stride, max_pairs, max_contrib, max_items, max_rows, max_long, max_chunks;
-};
 
 int validate_config(const tensair_config* c) {
     if (!c) return TENSAIR_EINVAL;
@@ -77,62 +66,14 @@ void carve(const tensair_config& c, Carve& k) {
     k.slot_bytes = round_up(k.delta_off + (uint64_t)k.max_rows * k.stride * 4, 256);
 }
 
-uint32_t bits_for(uint32_t x) {   // bits needed to represent x
-    uint32_t b = 0;
-    while (x) { ++b; x >>= 1; }
-    return b ? b : 1;
-}
-
 }  // namespace
 
-struct tensair_ctx {
-    tensair_config cfg;
-    Carve cv;
-    Shape shape;
-    cudaStream_t stream;
-    Launcher L;
-    uint64_t launches = 0;
-    Profiler prof;
-    float* tables;
-    uint8_t* pool;
-    uint8_t* scratch;
-    Schedule* sched = nullptr;
-    uint32_t last_n = 0, last_pairs = 0;
-    bool have_last = false;
-    std::string last_error;
-    // pinned host staging for small read-backs
-    struct Staging { MsgHeader hdr; double loss; uint32_t err; } *stage = nullptr;
-
-    template <class T> T* at(uint64_t off) const { return reinterpret_cast<T*>(scratch + off); }
-    float* table_of(uint32_t replica) const { return tables + (size_t)replica * 2 * cfg.V * cv.stride; }
-    uint8_t* slot_ptr(uint32_t slot) const { return pool + (size_t)slot * cv.slot_bytes; }
-    MsgHeader* slot_hdr(uint32_t slot) const { return reinterpret_cast<MsgHeader*>(slot_ptr(slot)); }
-    uint32_t* slot_ids(uint32_t slot) const { return reinterpret_cast<uint32_t*>(slot_ptr(slot) + cv.ids_off); }
-    float* slot_delta(uint32_t slot) const { return reinterpret_cast<float*>(slot_ptr(slot) + cv.delta_off); }
-};
-
-namespace {
+namespace tensair {
 
 int fail(tensair_ctx* ctx, cudaError_t e, const char* what) {
     if (ctx) ctx->last_error = std::string(what) + ": " + cudaGetErrorString(e);
     return TENSAIR_ECUDA;
 }
-
-#define TENSAIR_CUDA(ctx, call)                                    \
-    do {                                                           \
-        const cudaError_t e_ = (call);                             \
-        if (e_ != cudaSuccess) return fail((ctx), e_, #call);      \
-    } while (0)
-
-struct DeviceGuard {
-    int prev = -1;
-    bool ok = true;
-    explicit DeviceGuard(int dev) {
-        if (cudaGetDevice(&prev) != cudaSuccess) { ok = false; return; }
-        if (prev != dev && cudaSetDevice(dev) != cudaSuccess) ok = false;
-    }
-    ~DeviceGuard() { if (prev >= 0) cudaSetDevice(prev); }
-};
 
 // Reads and clears the device error flag after a synchronisation.
 int collect(tensair_ctx* ctx) {
@@ -145,6 +86,10 @@ int collect(tensair_ctx* ctx) {
     }
     return TENSAIR_OK;
 }
+
+}  // namespace tensair
+
+namespace {
 
 int upload_sampler(tensair_ctx* ctx, const uint64_t* counts_host) {
     const uint32_t V = ctx->cfg.V;
