@@ -166,6 +166,30 @@ TENSAIR_API int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, con
                              uint64_t batch_index, double* loss_out, tensair_msg_info* info);
 
 /*
+ * The same step for callers that may not allocate device memory when they train - a plug-in that is
+ * handed its tables and message pool by a host application with a fixed memory plan, or a service
+ * thread that must stay out of the allocator.  (The paper has no counterpart: this is an addition of
+ * this library.)  Arguments, results, error codes and the filing of the message are those of
+ * tensair_train_batch, and the result is bit-identical to it.  The difference: the per-batch working
+ * memory (sort buffers, segment lists, partial sums) is not taken from the scratch buffer given at
+ * tensair_init but from a fixed 32 MiB array inside the library image, which every GPU that loads the
+ * library reserves until the process exits.  The call allocates nothing on the device, neither
+ * directly nor through a library.
+ *   - TENSAIR_ENOMEM (with the sizes in tensair_last_error) when the context's configuration needs
+ *     more per-batch memory than the array holds; roughly batch * 2 * window * (k+1) * 32 bytes plus
+ *     batch * row_stride * 8 bytes must stay below 32 MiB.
+ *   - The first call on a device looks up the array's device address (once per device, with that device
+ *     current).  Make that first call before any stream capture begins.
+ *   - All calls, from all contexts of the process on one GPU, share the one array.  It keeps the last
+ *     call's contents; the call clears what it needs to be zero itself.  Two calls that may overlap on
+ *     the GPU (contexts on different streams) race on it: serialise them.
+ *   - The parity taps tensair_read_negatives and tensair_read_scalars work after this call as well.
+ */
+TENSAIR_API int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_dev,
+                                           uint32_t n_tokens, uint64_t batch_index, double* loss_out,
+                                           tensair_msg_info* info);
+
+/*
  * Algorithm 1, train, gradient branch, for one receiver: applies every pending message whose due step
  * is <= step, in (origin step, sender) order - the order in which Section 3.1 has a Model work off
  * the gradients that arrived while it was busy.  Call it for step t after every replica has run

@@ -66,6 +66,7 @@ SYMBOLS = {
     "tensair_destroy": (None, [_vp]),
     "tensair_train_batch": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
     "tensair_train_batch_host": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
+    "tensair_train_batch_static": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
     "tensair_apply_messages": (_int, [_vp, _u32, _u64, _P(_u32)]),
     "tensair_drain": (_int, [_vp, _P(_u32)]),
     "tensair_update_sampler": (_int, [_vp]),
@@ -252,6 +253,12 @@ class Context:
         assert tokens_dev.is_cuda and tokens_dev.dtype == self.torch.int32 and tokens_dev.is_contiguous()
         return self._train(lib().tensair_train_batch, "tensair_train_batch", replica, tokens_dev.data_ptr(),
                            tokens_dev.numel(), batch_index, want_loss, want_info)
+
+    def tensair_train_batch_static(self, replica, tokens_dev, batch_index, want_loss=False, want_info=False):
+        """tensair_train_batch with the per-batch working memory taken from the library's built-in array."""
+        assert tokens_dev.is_cuda and tokens_dev.dtype == self.torch.int32 and tokens_dev.is_contiguous()
+        return self._train(lib().tensair_train_batch_static, "tensair_train_batch_static", replica,
+                           tokens_dev.data_ptr(), tokens_dev.numel(), batch_index, want_loss, want_info)
 
     def tensair_train_batch_host(self, replica, tokens_host, batch_index, want_loss=False, want_info=False):
         """tokens_host: int32 numpy array or CPU tensor (pinned for an asynchronous copy)."""
