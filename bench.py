@@ -113,6 +113,15 @@ class ClockSampler:
                 "power_w_max": max(float(r[2]) for r in rows), "reasons": reasons}
 
 
+def max_over_ranks(ms: float, dist, device) -> float:
+    """The slowest rank's time: what a multi-rank run reports (works with nccl on GPUs and gloo on CPU)."""
+    import torch
+
+    x = torch.tensor([ms], device=device, dtype=torch.float64)
+    dist.all_reduce(x, op=dist.ReduceOp.MAX)
+    return float(x.item())
+
+
 def pick_workload(name: str, override: str = "") -> synth.Workload:
     """A named workload, optionally with fields replaced (`--override V=250000,W=2`: reduced cases for profiling)."""
     if name not in synth.WORKLOADS:
@@ -198,9 +207,7 @@ def run_ours(args):
         wall1 = time.time()
         ms = ev0.elapsed_time(ev1)
         if world > 1:
-            x = torch.tensor([ms], device="cuda", dtype=torch.float64)
-            dist.all_reduce(x, op=dist.ReduceOp.MAX)
-            ms = float(x.item())
+            ms = max_over_ranks(ms, dist, "cuda")
         return ms, wall0, wall1
 
     uuid = str(torch.cuda.get_device_properties(local).uuid)
