@@ -7,7 +7,7 @@
 // A warp then owns a row: it adds coefficient * source row over the segment (source = the centre's
 // input row and coefficient g for an output row; source = a position's partial centre gradient and
 // coefficient 1 for an input row), scales by -lr, writes the delta row into the message and, for an
-// output row, adds it to the table in the same pass.  Input rows are NOT updated here: they are the
+// output row, adds it to the table in the same pass (as a bulk asynchronous add performed at the memory side).  Input rows are NOT updated here: they are the
 // sources of every output-row sum and must keep their snapshot values until all sums are done.
 // Rows with more than kChunk contributions are split into chunks that run on separate warps; their
 // partial sums are combined in chunk order, so every sum has a fixed association.  All sums are
@@ -292,9 +292,34 @@ __device__ inline void finish_row(const RowSum<NV>& sum, const RowPrefetch<NV>& 
     }
 }
 
-// One warp per message row, rows taken in a grid-stride loop that is software-pipelined over three
-// rows: while row i is summed, the terms and the old table row of row i+1 and the segment bounds of
-// row i+2 are already on their way, so only the gathers of the source rows are waited for.
+// ---- bulk asynchronous copies out of shared memory -------------------------------------------------
+__device__ inline uint32_t smem_addr32(const void* p) { return (uint32_t)__cvta_generic_to_shared(p); }
+// Makes this thread's earlier shared-memory writes visible to the asynchronous copy engine.
+__device__ inline void fence_smem_writes_for_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+// global[dst .. dst+bytes) = shared[src .. src+bytes)
+__device__ inline void bulk_store_s2g(void* dst_global, const void* src_smem, uint32_t bytes) {
+    asm volatile("cp.async.bulk.global.shared::cta.bulk_group [%0], [%1], %2;"
+                 ::"l"(dst_global), "r"(smem_addr32(src_smem)), "r"(bytes) : "memory");
+}
+// global[dst + i] += shared[src + i] for every fp32 element: the read-modify-write is done at the memory
+// side (one IEEE addition per element, rounded to nearest even; each destination row has one writer here).
+__device__ inline void bulk_add_f32_s2g(void* dst_global, const void* src_smem, uint32_t bytes) {
+    asm volatile("cp.reduce.async.bulk.global.shared::cta.bulk_group.add.f32 [%0], [%1], %2;"
+                 ::"l"(dst_global), "r"(smem_addr32(src_smem)), "r"(bytes) : "memory");
+}
+__device__ inline void bulk_commit() { asm volatile("cp.async.bulk.commit_group;" ::: "memory"); }
+// Waits until all but the newest `keep` groups of this thread have finished READING their shared-memory source.
+template <int keep>
+__device__ inline void bulk_wait_read() { asm volatile("cp.async.bulk.wait_group.read %0;" ::"n"(keep) : "memory"); }
+__device__ inline void bulk_wait_all() { asm volatile("cp.async.bulk.wait_group 0;" ::: "memory"); }
+
+constexpr int kOutBuffers = 2;   // delta rows a warp may have on their way out
+
+// One warp per message row, rows taken in a grid-stride loop that is software-pipelined: while row i is
+// summed, the terms of row i+1 and the segment bounds of row i+2 are already on their way.  The finished
+// delta row is placed in shared memory and leaves by two bulk asynchronous operations: a store into the
+// message and, for an output row, an add onto the table row.  The table row is never read into the
+// multiprocessor, so nothing here waits on DRAM.
 template <int NV>
 __global__ void __launch_bounds__(kReduceThreads)
 k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids,
@@ -302,10 +327,14 @@ k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, 
               float4* __restrict__ table, float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4,
               double scale, uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows,
               ChunkItem* __restrict__ chunk_items) {
+    extern __shared__ __align__(128) float4 out_rows[];   // [warps in block][kOutBuffers][stride4]
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    float4* my_out = out_rows + (size_t)(threadIdx.x >> 5) * kOutBuffers * stride4;
     const uint32_t n_rows = hdr->n_rows;
+    const uint32_t row_bytes = d4 * 16;
+    const double nscale = -scale;
     struct Meta { uint32_t beg, end, id; };
     auto load_meta = [&](uint32_t m) {
         Meta x{0u, 0u, 0u};
@@ -320,15 +349,10 @@ k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, 
     uint32_t m = warp;
     Meta cur = load_meta(m), nxt = load_meta(m + nwarps);
     Rec cur_terms = load_terms(cur);
-    RowPrefetch<NV> cur_old;
-    if (m < n_rows && cur.end - cur.beg <= kChunk) cur_old.load(table, cur.id, V, d4, stride4, lane);
+    uint32_t buf = 0;
     for (; m < n_rows; m += nwarps) {
-        // stage the next two rows
         const Meta after = load_meta(m + 2 * nwarps);
         const Rec nxt_terms = load_terms(nxt);
-        RowPrefetch<NV> nxt_old;
-        if (m + nwarps < n_rows && nxt.end - nxt.beg <= kChunk) nxt_old.load(table, nxt.id, V, d4, stride4, lane);
-
         if (cur.end - cur.beg > kChunk) {
             const uint32_t nch = (cur.end - cur.beg + kChunk - 1) / kChunk;
             uint32_t base = 0;
@@ -344,13 +368,31 @@ k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, 
             sum.clear();
             accumulate_segment<NV>(terms, cur.beg, cur.end, cur.id < V, gin_pos, table, d4, stride4, lane, sum, true,
                                    cur_terms);
-            finish_row<NV>(sum, cur_old, m, cur.id, V, scale, table, delta, d4, stride4, lane);
+            // the buffer about to be refilled must have been read by the copies issued from it
+            if (lane == 0) bulk_wait_read<kOutBuffers - 1>();
+            __syncwarp();
+            float4* out = my_out + (size_t)buf * stride4;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const uint32_t e = lane + 32 * i;
+                if (e < d4)
+                    out[e] = make_float4((float)(nscale * sum.a[i][0]), (float)(nscale * sum.a[i][1]),
+                                         (float)(nscale * sum.a[i][2]), (float)(nscale * sum.a[i][3]));
+            }
+            fence_smem_writes_for_async();
+            __syncwarp();
+            if (lane == 0) {
+                bulk_store_s2g(delta + (size_t)m * stride4, out, row_bytes);
+                if (cur.id >= V) bulk_add_f32_s2g(table + (size_t)cur.id * stride4, out, row_bytes);
+                bulk_commit();
+            }
+            buf = (buf + 1) % kOutBuffers;
         }
         cur = nxt;
         nxt = after;
         cur_terms = nxt_terms;
-        cur_old = nxt_old;
     }
+    if (lane == 0) bulk_wait_all();
 }
 
 // Partial sums of the chunks of long rows, one warp per chunk; partials are kept in fp64.
@@ -427,7 +469,7 @@ static cudaError_t reduce_all(const Launcher& L, const Rec* terms, const MsgHead
     float4* d4p = reinterpret_cast<float4*>(delta);
     {
     Timed timed(L, K_REDUCE_ROWS);
-    k_reduce_rows<NV><<<blocks, kReduceThreads, 0, L.stream>>>(terms, hdr, ids, seg_start, gin_pos, t4, d4p, s.V, s.d4, stride4,
+    k_reduce_rows<NV><<<blocks, kReduceThreads, (size_t)(kReduceThreads / 32) * kOutBuffers * s.stride * 4, L.stream>>>(terms, hdr, ids, seg_start, gin_pos, t4, d4p, s.V, s.d4, stride4,
                                                     scale, long_counters, long_rows, chunk_items);
     }
     {
