@@ -250,7 +250,8 @@ typedef struct tensair_kernel_time {
 TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
 /* Launch-shape knobs for sweeps (process-wide; results do not depend on them): "forward_rows" = 8 or 16
  * output rows reduced together by a warp of the forward kernel (0 = default), "forward_blocks_per_sm"
- * = resident blocks per multiprocessor the forward grid is sized for (0 = default). */
+ * = resident blocks per multiprocessor the forward grid is sized for (0 = default),
+ * "reduce_blocks_per_sm" / "apply_blocks_per_sm" = blocks per multiprocessor of the row-sum / message-apply grids. */
 TENSAIR_API int tensair_tune(const char* name, int value);
 TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);
 

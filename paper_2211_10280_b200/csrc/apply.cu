@@ -7,6 +7,11 @@
 
 namespace tensair {
 
+GridShape& grid_shape() {
+    static GridShape shape;
+    return shape;
+}
+
 template <int NV>
 __global__ void __launch_bounds__(256)
 k_apply(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids, const float4* __restrict__ delta,
@@ -42,11 +47,12 @@ k_apply(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids, con
 cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
                               float* table, const Shape& s, int input_rows_only) {
     const uint32_t stride4 = s.stride / 4;
-    const int blocks = L.sms * 8;
     const float4* d4p = reinterpret_cast<const float4*>(delta);
     float4* t4 = reinterpret_cast<float4*>(table);
     Timed timed(L, input_rows_only ? K_APPLY_INPUT_ROWS : K_APPLY_MESSAGE);
-#define TENSAIR_APPLY(NV) k_apply<NV><<<blocks, 256, 0, L.stream>>>(hdr, ids, d4p, t4, s.d4, stride4, input_rows_only)
+#define TENSAIR_APPLY(NV)                                                                 \
+    k_apply<NV><<<L.sms * grid_shape().apply_blocks_per_sm, 256, 0, L.stream>>>(hdr, ids, d4p, t4, s.d4, stride4, \
+                                                                               input_rows_only)
     if (s.d4 <= 32) TENSAIR_APPLY(1);
     else if (s.d4 <= 64) TENSAIR_APPLY(2);
     else if (s.d4 <= 96) TENSAIR_APPLY(3);

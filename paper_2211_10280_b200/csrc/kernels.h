@@ -40,6 +40,14 @@ struct Launcher {
     Profiler* prof;       // nullable
 };
 
+// Blocks per multiprocessor of the grid-stride kernels (row sums, message apply).  More blocks than
+// are resident at once let the hardware scheduler even out rows of unequal cost.
+struct GridShape {
+    int reduce_blocks_per_sm = 64;
+    int apply_blocks_per_sm = 64;
+};
+GridShape& grid_shape();
+
 // Counts one kernel launch and, when profiling, brackets it with events: construct right before the
 // launch, let it go out of scope right after.
 struct Timed {

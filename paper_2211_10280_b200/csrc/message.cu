@@ -464,17 +464,17 @@ static cudaError_t reduce_all(const Launcher& L, const Rec* terms, const MsgHead
                               float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
                               ChunkItem* chunk_items, double* partials) {
     const uint32_t stride4 = s.stride / 4;
-    const int blocks = L.sms * 16;
+    const size_t out_smem = (size_t)(kReduceThreads / 32) * kOutBuffers * s.stride * 4;
     float4* t4 = reinterpret_cast<float4*>(table);
     float4* d4p = reinterpret_cast<float4*>(delta);
     {
     Timed timed(L, K_REDUCE_ROWS);
-    k_reduce_rows<NV><<<blocks, kReduceThreads, (size_t)(kReduceThreads / 32) * kOutBuffers * s.stride * 4, L.stream>>>(terms, hdr, ids, seg_start, gin_pos, t4, d4p, s.V, s.d4, stride4,
+    k_reduce_rows<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, out_smem, L.stream>>>(terms, hdr, ids, seg_start, gin_pos, t4, d4p, s.V, s.d4, stride4,
                                                     scale, long_counters, long_rows, chunk_items);
     }
     {
     Timed timed(L, K_REDUCE_CHUNKS);
-    k_reduce_chunks<NV><<<blocks, kReduceThreads, 0, L.stream>>>(terms, ids, seg_start, gin_pos, t4, s.V, s.d4, stride4,
+    k_reduce_chunks<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, 0, L.stream>>>(terms, ids, seg_start, gin_pos, t4, s.V, s.d4, stride4,
                                                       long_counters, chunk_items, partials);
     }
     {

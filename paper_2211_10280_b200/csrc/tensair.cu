@@ -433,6 +433,8 @@ int tensair_tune(const char* name, int value) {
     static int rows = 0, blocks = 0;
     if (!std::strcmp(name, "forward_rows")) rows = value;
     else if (!std::strcmp(name, "forward_blocks_per_sm")) blocks = value;
+    else if (!std::strcmp(name, "reduce_blocks_per_sm") && value > 0) { grid_shape().reduce_blocks_per_sm = value; return TENSAIR_OK; }
+    else if (!std::strcmp(name, "apply_blocks_per_sm") && value > 0) { grid_shape().apply_blocks_per_sm = value; return TENSAIR_OK; }
     else return TENSAIR_EINVAL;
     set_forward_shape(rows, blocks);
     return TENSAIR_OK;
