@@ -41,7 +41,7 @@ struct ChunkItem {
     uint32_t m;
     uint32_t chunk;
 };
-constexpr uint32_t kChunk = 128;   // contributions per chunk; rows with more than this go the long way
+constexpr uint32_t kChunk = 64;    // contributions per chunk; rows with more than this go the long way
 
 // Sum over i < x of min(i, w): how many left (or, mirrored, right) neighbours the first x positions have.
 __host__ __device__ inline uint64_t neighbours_before(uint64_t x, uint64_t w) {

@@ -426,35 +426,74 @@ k_reduce_chunks(const Rec* __restrict__ terms, const uint32_t* __restrict__ ids,
     }
 }
 
-// Long rows: the chunk partials are added in chunk order, then the row is finished like a short one.
+// Long rows: one block per row.  Warp w adds a contiguous run of the row's chunk partials in chunk order
+// (four fetched together), the runs are then added in warp order by warp 0, and the row is finished like a
+// short one - a fixed association for every launch shape.
+constexpr int kLongWarps = 8;
 template <int NV>
-__global__ void __launch_bounds__(kReduceThreads)
+__global__ void __launch_bounds__(kLongWarps * 32)
 k_reduce_long(const uint32_t* __restrict__ ids, const double* __restrict__ partials, float4* __restrict__ table,
               float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4, double scale,
-              const uint32_t* __restrict__ long_counters, const LongRow* __restrict__ long_rows) {
-    const uint32_t lane = threadIdx.x & 31;
-    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
-    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+              const uint32_t* __restrict__ long_counters, const LongRow* __restrict__ long_rows, uint32_t warps) {
+    extern __shared__ __align__(16) double runs[];   // [warps][4 * d4]
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t n_long = long_counters[0];
-    for (uint32_t x = warp; x < n_long; x += nwarps) {
+    for (uint32_t x = blockIdx.x; x < n_long; x += gridDim.x) {
         const LongRow row = long_rows[x];
         const uint32_t id = ids[row.m];
-        RowPrefetch<NV> old;
-        old.load(table, id, V, d4, stride4, lane);
+        const uint32_t per = (row.nchunks + warps - 1) / warps;
+        const uint32_t c_beg = wid * per < row.nchunks ? wid * per : row.nchunks;
+        const uint32_t c_end = c_beg + per < row.nchunks ? c_beg + per : row.nchunks;
         RowSum<NV> sum;
         sum.clear();
-        for (uint32_t c = 0; c < row.nchunks; ++c) {
-            const double2* in = reinterpret_cast<const double2*>(partials + (size_t)(row.base + c) * stride4 * 4);
+        for (uint32_t c0 = c_beg; c0 < c_end; c0 += 4) {
+            double2 part[4][NV][2];
 #pragma unroll
-            for (int i = 0; i < NV; ++i) {
-                const uint32_t e = lane + 32 * i;
-                if (e < d4) {
-                    const double2 lo = in[2 * e], hi = in[2 * e + 1];
-                    sum.a[i][0] += lo.x; sum.a[i][1] += lo.y; sum.a[i][2] += hi.x; sum.a[i][3] += hi.y;
+            for (int t = 0; t < 4; ++t) {
+                const double2* in = reinterpret_cast<const double2*>(partials + (size_t)(row.base + c0 + t) * stride4 * 4);
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const uint32_t e = lane + 32 * i;
+                    const bool on = c0 + t < c_end && e < d4;
+                    part[t][i][0] = on ? in[2 * e] : make_double2(0.0, 0.0);
+                    part[t][i][1] = on ? in[2 * e + 1] : make_double2(0.0, 0.0);
                 }
             }
+#pragma unroll
+            for (int t = 0; t < 4; ++t)
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    sum.a[i][0] += part[t][i][0].x; sum.a[i][1] += part[t][i][0].y;
+                    sum.a[i][2] += part[t][i][1].x; sum.a[i][3] += part[t][i][1].y;
+                }
         }
-        finish_row<NV>(sum, old, row.m, id, V, scale, table, delta, d4, stride4, lane);
+        double2* mine = reinterpret_cast<double2*>(runs + (size_t)wid * d4 * 4);
+#pragma unroll
+        for (int i = 0; i < NV; ++i) {
+            const uint32_t e = lane + 32 * i;
+            if (e < d4) {
+                mine[2 * e] = make_double2(sum.a[i][0], sum.a[i][1]);
+                mine[2 * e + 1] = make_double2(sum.a[i][2], sum.a[i][3]);
+            }
+        }
+        __syncthreads();
+        if (wid == 0) {
+            RowPrefetch<NV> old;
+            old.load(table, id, V, d4, stride4, lane);
+            for (uint32_t w = 1; w < warps; ++w) {
+                const double2* other = reinterpret_cast<const double2*>(runs + (size_t)w * d4 * 4);
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const uint32_t e = lane + 32 * i;
+                    if (e < d4) {
+                        const double2 lo = other[2 * e], hi = other[2 * e + 1];
+                        sum.a[i][0] += lo.x; sum.a[i][1] += lo.y; sum.a[i][2] += hi.x; sum.a[i][3] += hi.y;
+                    }
+                }
+            }
+            finish_row<NV>(sum, old, row.m, id, V, scale, table, delta, d4, stride4, lane);
+        }
+        __syncthreads();
     }
 }
 
@@ -479,8 +518,11 @@ static cudaError_t reduce_all(const Launcher& L, const Rec* terms, const MsgHead
     }
     {
     Timed timed(L, K_REDUCE_LONG);
-    k_reduce_long<NV><<<L.sms * 4, kReduceThreads, 0, L.stream>>>(ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters,
-                                                       long_rows);
+    uint32_t long_warps = 49152 / (s.d * 8);          // run sums of one block within 48 KB of shared memory
+    if (long_warps > (uint32_t)kLongWarps) long_warps = kLongWarps;
+    if (long_warps < 1) long_warps = 1;
+    k_reduce_long<NV><<<L.sms * 2, long_warps * 32, (size_t)long_warps * s.d * 8, L.stream>>>(
+        ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters, long_rows, long_warps);
     }
     return cudaGetLastError();
 }
