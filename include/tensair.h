@@ -17,7 +17,9 @@
  *     this boundary.  tensair_strerror() names a code, tensair_last_error() gives detail.
  *   - "device pointer" means memory of the GPU named in tensair_config.device; "host pointer" means
  *     ordinary process memory (pinned or pageable).
- *   - All GPU work is enqueued on the stream given at tensair_init, in call order.  Calls are
+ *   - All GPU work is enqueued on the stream given at tensair_init, in call order (inside one call the
+ *     library may fork part of the work onto an internal stream and join it again before the call's
+ *     last kernel; to the caller's stream the call is one ordered piece of work).  Calls are
  *     asynchronous unless stated; a context must be used from one thread at a time.
  *   - The library allocates no device memory: tables, message pool and scratch are caller-owned and
  *     must stay valid until tensair_destroy.
@@ -251,7 +253,8 @@ TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
 /* Launch-shape knobs for sweeps (process-wide; results do not depend on them): "forward_rows" = 8 or 16
  * output rows reduced together by a warp of the forward kernel (0 = default), "forward_blocks_per_sm"
  * = resident blocks per multiprocessor the forward grid is sized for (0 = default),
- * "reduce_blocks_per_sm" / "apply_blocks_per_sm" = blocks per multiprocessor of the row-sum / message-apply grids. */
+ * "reduce_blocks_per_sm" / "apply_blocks_per_sm" = blocks per multiprocessor of the row-sum / message-apply grids,
+ * "overlap_sort" = 0 keeps the sort of a batch on the caller's stream instead of an internal second stream. */
 TENSAIR_API int tensair_tune(const char* name, int value);
 TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);
 

@@ -33,6 +33,10 @@ struct tensair_ctx {
     tensair::Carve cv;
     tensair::Shape shape;
     cudaStream_t stream;
+    // internal second stream: the sort of a batch's contributions runs there, beside the forward kernel
+    cudaStream_t side = nullptr;
+    cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
+    tensair::Launcher L_side;
     tensair::Launcher L;
     uint64_t launches = 0;
     tensair::Profiler prof;

@@ -43,6 +43,7 @@ struct Launcher {
 // Blocks per multiprocessor of the grid-stride kernels (row sums, message apply).  More blocks than
 // are resident at once let the hardware scheduler even out rows of unequal cost.
 struct GridShape {
+    int overlap_sort = 1;            // run the radix sort on a second stream while the forward kernel runs
     int reduce_blocks_per_sm = 64;
     int apply_blocks_per_sm = 64;
 };

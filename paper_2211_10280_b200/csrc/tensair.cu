@@ -123,11 +123,22 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows),
                                      ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err));
     if (n_items) {
+        // The sort needs only the items written by the prepare kernel and the forward kernel does not
+        // touch them: the two run side by side (the sort is latency-bound and leaves the machine idle).
+        const bool fork = ctx->side && grid_shape().overlap_sort;
+        if (fork) {
+            TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
+            TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+        }
+        item_t* sorted = nullptr;
+        TENSAIR_CUDA(ctx, launch_sort(fork ? ctx->L_side : ctx->L, ctx->at<item_t>(cv.items_a), ctx->at<item_t>(cv.items_b),
+                                      n_items, bits_for(2 * c.V), ctx->at<uint32_t>(cv.hist), &sorted));
         TENSAIR_CUDA(ctx, launch_forward(ctx->L, tok_dev, n, ctx->shape, table, ctx->at<uint32_t>(cv.rows),
                                          ctx->at<Rec>(cv.rec), ctx->at<double>(cv.gin_pos), ctx->at<double>(cv.loss_pos), err));
-        item_t* sorted = nullptr;
-        TENSAIR_CUDA(ctx, launch_sort(ctx->L, ctx->at<item_t>(cv.items_a), ctx->at<item_t>(cv.items_b), n_items,
-                                      bits_for(2 * c.V), ctx->at<uint32_t>(cv.hist), &sorted));
+        if (fork) {
+            TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+            TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0));
+        }
         TENSAIR_CUDA(ctx, launch_heads(ctx->L, sorted, n_items, c.V, ctx->at<uint32_t>(cv.tile_counts), hdr,
                                        ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
                                        ctx->at<uint32_t>(cv.long_counters), ctx->at<Rec>(cv.rec),
@@ -226,11 +237,25 @@ int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const u
     ctx->scratch = (uint8_t*)bufs->scratch;
     cudaDeviceProp prop;
     int status = TENSAIR_OK;
-    auto bail = [&](int code) { delete ctx->sched; if (ctx->stage) cudaFreeHost(ctx->stage); delete ctx; return code; };
+    auto bail = [&](int code) {
+        delete ctx->sched;
+        if (ctx->stage) cudaFreeHost(ctx->stage);
+        if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
+        if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
+        if (ctx->side) cudaStreamDestroy(ctx->side);
+        delete ctx;
+        return code;
+    };
     if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount, &ctx->prof};
     if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->sched = new Schedule(cfg->W, cfg->max_delay, cfg->seed);
+    if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess)
+        return bail(TENSAIR_ECUDA);
+    ctx->L_side = ctx->L;
+    ctx->L_side.stream = ctx->side;
 
     const uint32_t V = cfg->V, stride = ctx->cv.stride;
     const size_t replica_floats = (size_t)2 * V * stride;
@@ -269,6 +294,12 @@ void tensair_destroy(tensair_ctx* ctx) {
     for (const Profiler::Span& sp : ctx->prof.spans) { cudaEventDestroy(sp.start); cudaEventDestroy(sp.stop); }
     for (cudaEvent_t e : ctx->prof.spare) cudaEventDestroy(e);
     if (ctx->stage) cudaFreeHost(ctx->stage);
+    if (ctx->side) {
+        cudaStreamSynchronize(ctx->side);
+        cudaEventDestroy(ctx->ev_fork);
+        cudaEventDestroy(ctx->ev_join);
+        cudaStreamDestroy(ctx->side);
+    }
     delete ctx->sched;
     delete ctx;
 }
@@ -433,6 +464,7 @@ int tensair_tune(const char* name, int value) {
     static int rows = 0, blocks = 0;
     if (!std::strcmp(name, "forward_rows")) rows = value;
     else if (!std::strcmp(name, "forward_blocks_per_sm")) blocks = value;
+    else if (!std::strcmp(name, "overlap_sort")) { grid_shape().overlap_sort = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "reduce_blocks_per_sm") && value > 0) { grid_shape().reduce_blocks_per_sm = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "apply_blocks_per_sm") && value > 0) { grid_shape().apply_blocks_per_sm = value; return TENSAIR_OK; }
     else return TENSAIR_EINVAL;
