@@ -262,6 +262,7 @@ def run_ours(args):
         "reduce_rows": U * (row + 4) + U_out * 2 * row,                   # message write + read/write of output rows
         "apply_message": U_applied * (row + 4 + 2 * row),                 # delta read + row read + row write
     }
+    algo["apply_fused"] = algo["apply_message"] * (len(applied) / max(1, prof.get("apply_fused", (0, 0))[0]))
     tot_ms = sum(v[1] for v in prof.values()) or 1.0
     kernels = {}
     for name, (cnt, ms) in prof.items():

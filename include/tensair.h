@@ -254,7 +254,8 @@ TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
  * output rows reduced together by a warp of the forward kernel (0 = default), "forward_blocks_per_sm"
  * = resident blocks per multiprocessor the forward grid is sized for (0 = default),
  * "reduce_blocks_per_sm" / "apply_blocks_per_sm" = blocks per multiprocessor of the row-sum / message-apply grids,
- * "overlap_sort" = 0 keeps the sort of a batch on the caller's stream instead of an internal second stream. */
+ * "fuse_apply" = 0 applies the messages due for a receiver one launch each instead of in one pass,
+ * "fused_blocks_per_sm" = blocks per multiprocessor of that pass, "overlap_sort" = 0 keeps the sort of a batch on the caller's stream instead of an internal second stream. */
 TENSAIR_API int tensair_tune(const char* name, int value);
 TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);
 

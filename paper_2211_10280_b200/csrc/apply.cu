@@ -62,6 +62,88 @@ cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uin
     return cudaGetLastError();
 }
 
+// One thread per bucket boundary: lower bound of b << kBucketShift in the ascending id list.
+__global__ void __launch_bounds__(256)
+k_bucket_index(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids, uint32_t* __restrict__ bucket_start,
+               uint32_t n_buckets) {
+    const uint32_t b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b > n_buckets) return;
+    const uint32_t n_rows = hdr->n_rows;
+    const uint64_t key = (uint64_t)b << kBucketShift;
+    uint32_t lo = 0, hi = n_rows;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if ((uint64_t)__ldg(ids + mid) < key) lo = mid + 1; else hi = mid;
+    }
+    bucket_start[b] = lo;
+}
+
+cudaError_t launch_bucket_index(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
+                                uint32_t V) {
+    const uint32_t nb = bucket_count(V);
+    Timed timed(L, K_BUCKET_INDEX);
+    k_bucket_index<<<(nb + 1 + 255) / 256, 256, 0, L.stream>>>(hdr, ids, bucket_start, nb);
+    return cudaGetLastError();
+}
+
+// Several messages, one pass.  A block owns an id range (a few buckets in a grid-stride loop); for each
+// message in order its warps take the message's rows in that range; a block-wide barrier separates the
+// messages, so a row touched by two of them gets its additions in message order.  Table rows are read
+// with L1 bypassed (another warp of the block may just have written them).
+constexpr int kFusedThreads = 128;
+template <int NV>
+__global__ void __launch_bounds__(kFusedThreads)
+k_apply_fused(FusedMessages f, float4* __restrict__ table, uint32_t d4, uint32_t stride4, uint32_t n_buckets) {
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    constexpr uint32_t kWarps = kFusedThreads / 32;
+    for (uint32_t b = blockIdx.x; b < n_buckets; b += gridDim.x) {
+        for (uint32_t k = 0; k < f.count; ++k) {
+            const uint32_t beg = __ldg(f.buckets[k] + b), end = __ldg(f.buckets[k] + b + 1);
+            const float4* __restrict__ delta = reinterpret_cast<const float4*>(f.delta[k]);
+            for (uint32_t m = beg + wid; m < end; m += kWarps) {
+                const uint32_t id = __ldg(f.ids[k] + m);
+                const float4* __restrict__ src = delta + (size_t)m * stride4;
+                float4* dst = table + (size_t)id * stride4;
+                float4 a[NV], r[NV];
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const uint32_t e = lane + 32 * i;
+                    if (e < d4) {
+                        a[i] = __ldg(src + e);
+                        r[i] = __ldcg(dst + e);
+                    }
+                }
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const uint32_t e = lane + 32 * i;
+                    if (e < d4) {
+                        r[i].x += a[i].x; r[i].y += a[i].y; r[i].z += a[i].z; r[i].w += a[i].w;
+                        dst[e] = r[i];
+                    }
+                }
+            }
+            __syncthreads();
+        }
+    }
+}
+
+cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float* table, const Shape& s) {
+    const uint32_t stride4 = s.stride / 4;
+    float4* t4 = reinterpret_cast<float4*>(table);
+    const uint32_t nb = bucket_count(s.V);
+    uint32_t blocks = (uint32_t)(L.sms * grid_shape().fused_blocks_per_sm);
+    if (blocks > nb) blocks = nb;
+    Timed timed(L, K_APPLY_FUSED);
+#define TENSAIR_FUSED(NV) k_apply_fused<NV><<<blocks, kFusedThreads, 0, L.stream>>>(f, t4, s.d4, stride4, nb)
+    if (s.d4 <= 32) TENSAIR_FUSED(1);
+    else if (s.d4 <= 64) TENSAIR_FUSED(2);
+    else if (s.d4 <= 96) TENSAIR_FUSED(3);
+    else if (s.d4 <= 128) TENSAIR_FUSED(4);
+    else TENSAIR_FUSED(8);
+#undef TENSAIR_FUSED
+    return cudaGetLastError();
+}
+
 cudaError_t launch_apply(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
                          float* table, const Shape& s) {
     return launch_apply_rows(L, hdr, ids, delta, table, s, 0);

@@ -16,7 +16,7 @@ inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 struct Carve {
     uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, terms, gin_pos, loss_pos, hist,
         tile_counts, seg_start, long_rows, chunk_items, partials, total;
-    uint64_t slot_bytes, ids_off, delta_off;
+    uint64_t slot_bytes, bucket_off, ids_off, delta_off;
     uint32_t stride, max_pairs, max_contrib, max_items, max_rows, max_long, max_chunks;
 };
 
@@ -54,6 +54,7 @@ struct tensair_ctx {
     float* table_of(uint32_t replica) const { return tables + (size_t)replica * 2 * cfg.V * cv.stride; }
     uint8_t* slot_ptr(uint32_t slot) const { return pool + (size_t)slot * cv.slot_bytes; }
     tensair::MsgHeader* slot_hdr(uint32_t slot) const { return reinterpret_cast<tensair::MsgHeader*>(slot_ptr(slot)); }
+    uint32_t* slot_buckets(uint32_t slot) const { return reinterpret_cast<uint32_t*>(slot_ptr(slot) + cv.bucket_off); }
     uint32_t* slot_ids(uint32_t slot) const { return reinterpret_cast<uint32_t*>(slot_ptr(slot) + cv.ids_off); }
     float* slot_delta(uint32_t slot) const { return reinterpret_cast<float*>(slot_ptr(slot) + cv.delta_off); }
 };

@@ -9,13 +9,13 @@ namespace tensair {
 enum KernelKind {
     K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
     K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
-    K_APPLY_MESSAGE, K_INIT_TABLE, K_KINDS
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_KINDS
 };
 inline const char* kernel_name(int kind) {
     static const char* const names[K_KINDS] = {
         "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
         "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
-        "apply_message", "init_table"};
+        "apply_message", "init_table", "bucket_index", "apply_fused"};
     return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
 }
 
@@ -43,9 +43,11 @@ struct Launcher {
 // Blocks per multiprocessor of the grid-stride kernels (row sums, message apply).  More blocks than
 // are resident at once let the hardware scheduler even out rows of unequal cost.
 struct GridShape {
+    int fuse_apply = 1;              // apply the messages due for a receiver in one pass over its table
     int overlap_sort = 1;            // run the radix sort on a second stream while the forward kernel runs
     int reduce_blocks_per_sm = 64;
     int apply_blocks_per_sm = 64;
+    int fused_blocks_per_sm = 64;
 };
 GridShape& grid_shape();
 
@@ -101,6 +103,19 @@ cudaError_t launch_reduce(const Launcher& L, const Rec* terms, const MsgHeader* 
 // apply.cu
 cudaError_t launch_apply(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
                          float* table, const Shape& s);
+// Several messages for one receiver in one pass: applied id range by id range, message after message within
+// a range, so every table row sees its deltas in message order and is fetched from memory once.
+constexpr int kMaxFused = 8;
+struct FusedMessages {
+    uint32_t count;
+    const uint32_t* ids[kMaxFused];
+    const float* delta[kMaxFused];
+    const uint32_t* buckets[kMaxFused];
+};
+cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float* table, const Shape& s);
+// bucket_start[b] = first row of the message with id >= b << kBucketShift, for b in [0, bucket_count(V)].
+cudaError_t launch_bucket_index(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
+                                uint32_t V);
 // Same, restricted to the message's input rows when input_rows_only != 0.
 cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
                               float* table, const Shape& s, int input_rows_only);

@@ -127,6 +127,7 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
     } else {
         TENSAIR_CUDA(ctx, cudaMemsetAsync(hdr, 0, sizeof(MsgHeader), ctx->stream));
     }
+    TENSAIR_CUDA(ctx, launch_bucket_index(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
     TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, loss_pos, n_tokens, ctx->at<double>(cv.loss), err));
     ctx->last_n = n_tokens;
     ctx->last_pairs = pairs;

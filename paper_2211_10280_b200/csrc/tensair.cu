@@ -2,6 +2,7 @@
 #include "../../include/tensair.h"
 
 #include <cstdio>
+#include <algorithm>
 #include <cstring>
 #include <new>
 #include <string>
@@ -61,7 +62,8 @@ void carve(const tensair_config& c, Carve& k) {
     k.chunk_items = take((uint64_t)k.max_chunks * sizeof(ChunkItem));
     k.partials = take((uint64_t)k.max_chunks * k.stride * 8);
     k.total = off;
-    k.ids_off = kHeaderBytes;
+    k.bucket_off = kHeaderBytes;
+    k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
     k.delta_off = round_up(k.ids_off + (uint64_t)k.max_rows * 4, 256);
     k.slot_bytes = round_up(k.delta_off + (uint64_t)k.max_rows * k.stride * 4, 256);
 }
@@ -153,6 +155,7 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
     } else {
         TENSAIR_CUDA(ctx, cudaMemsetAsync(hdr, 0, sizeof(MsgHeader), ctx->stream));
     }
+    TENSAIR_CUDA(ctx, launch_bucket_index(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
     TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err));
     ctx->last_n = n;
     ctx->last_pairs = pairs;
@@ -175,9 +178,27 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
 }
 
 int apply_due(tensair_ctx* ctx, uint32_t receiver, const std::vector<Due>& due) {
-    for (const Due& d : due)
-        TENSAIR_CUDA(ctx, launch_apply(ctx->L, ctx->slot_hdr(d.slot), ctx->slot_ids(d.slot), ctx->slot_delta(d.slot),
-                                       ctx->table_of(receiver), ctx->shape));
+    // Messages are applied in the order given; up to kMaxFused of them share one pass over the table.
+    size_t at = 0;
+    while (at < due.size()) {
+        const size_t k = grid_shape().fuse_apply ? std::min(due.size() - at, (size_t)kMaxFused) : 1;
+        if (k == 1) {
+            const Due& d = due[at];
+            TENSAIR_CUDA(ctx, launch_apply(ctx->L, ctx->slot_hdr(d.slot), ctx->slot_ids(d.slot), ctx->slot_delta(d.slot),
+                                           ctx->table_of(receiver), ctx->shape));
+        } else {
+            FusedMessages f;
+            f.count = (uint32_t)k;
+            for (size_t i = 0; i < k; ++i) {
+                const uint32_t slot = due[at + i].slot;
+                f.ids[i] = ctx->slot_ids(slot);
+                f.delta[i] = ctx->slot_delta(slot);
+                f.buckets[i] = ctx->slot_buckets(slot);
+            }
+            TENSAIR_CUDA(ctx, launch_apply_fused(ctx->L, f, ctx->table_of(receiver), ctx->shape));
+        }
+        at += k;
+    }
     return TENSAIR_OK;
 }
 
@@ -464,6 +485,8 @@ int tensair_tune(const char* name, int value) {
     static int rows = 0, blocks = 0;
     if (!std::strcmp(name, "forward_rows")) rows = value;
     else if (!std::strcmp(name, "forward_blocks_per_sm")) blocks = value;
+    else if (!std::strcmp(name, "fused_blocks_per_sm") && value > 0) { grid_shape().fused_blocks_per_sm = value; return TENSAIR_OK; }
+    else if (!std::strcmp(name, "fuse_apply")) { grid_shape().fuse_apply = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "overlap_sort")) { grid_shape().overlap_sort = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "reduce_blocks_per_sm") && value > 0) { grid_shape().reduce_blocks_per_sm = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "apply_blocks_per_sm") && value > 0) { grid_shape().apply_blocks_per_sm = value; return TENSAIR_OK; }
