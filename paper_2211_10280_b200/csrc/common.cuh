@@ -33,7 +33,7 @@ constexpr uint32_t kHeaderBytes = 256;
 // Every message carries an index of its rows by id range ("bucket" b = ids in [b << kBucketShift, (b+1) << kBucketShift)):
 // bucket_start[b] = first row whose id is not below the bucket.  It lets one pass apply several messages
 // id range by id range, so that a table row touched by more than one of them is fetched from memory once.
-constexpr uint32_t kBucketShift = 6;
+constexpr uint32_t kBucketShift = 4;
 __host__ __device__ inline uint32_t bucket_count(uint32_t V) { return ((2 * V - 1) >> kBucketShift) + 1; }
 
 // A long row (more contributions than one warp takes in one go) and its chunk partials.

@@ -47,7 +47,7 @@ struct GridShape {
     int overlap_sort = 1;            // run the radix sort on a second stream while the forward kernel runs
     int reduce_blocks_per_sm = 64;
     int apply_blocks_per_sm = 64;
-    int fused_blocks_per_sm = 64;
+    int fused_blocks_per_sm = 256;
 };
 GridShape& grid_shape();
 
