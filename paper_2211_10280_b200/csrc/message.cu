@@ -178,7 +178,8 @@ cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_ite
 // ---------------------------------------------------------------------------------------------
 // per-row sums
 // ---------------------------------------------------------------------------------------------
-constexpr int kTermsInFlight = 4;
+constexpr int kTermsInFlightRows = 1;     // source rows a warp of the row kernel gathers at once (few: more warps fit)
+constexpr int kTermsInFlightChunks = 4;   // the same for the chunk kernel, whose segments are long
 constexpr int kReduceThreads = 128;
 
 // One lane's share of a row sum: fp64 accumulators for its NV float4 slices.
@@ -195,7 +196,7 @@ struct RowSum {
 // coalesced load and hands them round by shuffle; the fp32 source rows of four terms are in flight
 // together.  Products and sums are taken in fp64, so the result does not feel the cancellation
 // between the positive and negative terms of a row.
-template <int NV>
+template <int NV, int kTermsInFlight>
 __device__ inline void accumulate_segment(const Rec* __restrict__ terms, uint32_t beg, uint32_t end, bool input_row,
                                           const double* __restrict__ gin_pos, const float4* __restrict__ table,
                                           uint32_t d4, uint32_t stride4, uint32_t lane, RowSum<NV>& sum,
@@ -366,7 +367,7 @@ k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, 
         } else {
             RowSum<NV> sum;
             sum.clear();
-            accumulate_segment<NV>(terms, cur.beg, cur.end, cur.id < V, gin_pos, table, d4, stride4, lane, sum, true,
+            accumulate_segment<NV, kTermsInFlightRows>(terms, cur.beg, cur.end, cur.id < V, gin_pos, table, d4, stride4, lane, sum, true,
                                    cur_terms);
             // the buffer about to be refilled must have been read by the copies issued from it
             if (lane == 0) bulk_wait_read<kOutBuffers - 1>();
@@ -413,7 +414,7 @@ k_reduce_chunks(const Rec* __restrict__ terms, const uint32_t* __restrict__ ids,
         const uint32_t end = beg + kChunk < seg_end ? beg + kChunk : seg_end;
         RowSum<NV> sum;
         sum.clear();
-        accumulate_segment<NV>(terms, beg, end, ids[ci.m] < V, gin_pos, table, d4, stride4, lane, sum);
+        accumulate_segment<NV, kTermsInFlightChunks>(terms, beg, end, ids[ci.m] < V, gin_pos, table, d4, stride4, lane, sum);
         double* out = partials + (size_t)x * stride4 * 4;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
