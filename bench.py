@@ -383,6 +383,48 @@ def run_reference(args):
     }))
 
 
+def run_sweep(args):
+    """The throughput sweep (V = 1M, one replica): one JSON line per (d, batch, k) point with pairs/s and
+    the algorithmic HBM GB/s of the step (gather + message write + local application, each touched row once per pass)."""
+    import torch
+
+    from paper_2211_10280_b200 import binding as B
+
+    peak, peak_kind = hbm_peak()
+    steps = min(args.steps, 100)
+    for wl in synth.SWEEP:
+        nb = steps + 6
+        stream = synth.token_stream(wl, 0, nb)
+        counts = synth.stream_counts([synth.token_stream(wl, 0, min(wl.batches, 100))], wl.V)
+        ctx = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=1, lr=wl.lr, seed=wl.seed,
+                        counts=counts, reduction=wl.reduction)
+        toks = torch.from_numpy(stream).cuda()
+        rows = []
+        for t in range(3):
+            _, info = ctx.tensair_train_batch(0, toks[t], t, want_info=True)
+            rows.append(info.n_rows)
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        torch.cuda.synchronize()
+        ev0.record()
+        for t in range(3, 3 + steps):
+            ctx.tensair_train_batch(0, toks[t], t)
+        ev1.record()
+        torch.cuda.synchronize()
+        ms = ev0.elapsed_time(ev1) / steps
+        _, info = ctx.tensair_train_batch(0, toks[3 + steps], 3 + steps, want_info=True)
+        U = float(np.mean(rows + [info.n_rows]))
+        row = 4 * wl.d
+        own = U * row + U * (row + 4) + U * (row + 4 + 2 * row)
+        print(json.dumps({"workload": wl.name, "d": wl.d, "batch": wl.batch, "k": wl.k, "pairs_per_batch": wl.pairs_per_batch,
+                          "rows_per_message": int(U), "ms_per_batch": round(ms, 4),
+                          "pairs_per_s": wl.pairs_per_batch / (ms * 1e-3), "algorithmic_gbs": round(own / (ms * 1e-3) / 1e9, 1),
+                          "frac_of_peak": round(own / (ms * 1e-3) / 1e9 / peak, 4), "peak": f"{peak} GB/s of {peak_kind}"}),
+              flush=True)
+        ctx.close()
+        del ctx, toks
+        torch.cuda.empty_cache()
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -392,9 +434,12 @@ def main():
     ap.add_argument("--workload", default=synth.LARGE_DASGD.name)
     ap.add_argument("--override", default="", help="comma-separated field=value replacements of the workload")
     ap.add_argument("--tune", default="", help="comma-separated knob=value pairs passed to tensair_tune (sweeps)")
+    ap.add_argument("--sweep", action="store_true", help="run the 32-point throughput sweep instead (one line per point)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.sweep:
+        run_sweep(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)

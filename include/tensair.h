@@ -219,6 +219,19 @@ TENSAIR_API int tensair_read_embeddings(tensair_ctx* ctx, uint32_t replica, int 
 TENSAIR_API int tensair_write_embeddings(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows,
                              const float* host_src);
 
+/*
+ * Drift metric of Section 4.3 (Table 1): how far an embedding row has moved between two points of the
+ * stream, as the cosine difference 1 - cos(a, b) of the row now (a) and in an earlier snapshot (b).
+ *   tensair_snapshot_rows      copies rows [row0, row0+nrows) of a table into snap_dev, device float[nrows*d] dense.
+ *   tensair_cosine_difference  writes 1 - (a.b) / (|a| |b|) per row into out_dev, device float[nrows]; dot and
+ *                              norms in fp64; two zero rows give 0, one zero row gives 1.
+ * Both are asynchronous on the context's stream; the buffers are the caller's.
+ */
+TENSAIR_API int tensair_snapshot_rows(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows,
+                                      float* snap_dev);
+TENSAIR_API int tensair_cosine_difference(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows,
+                                          const float* snap_dev, float* out_dev);
+
 /* ---- parity taps (synchronous; for tests and diagnostics) ---- */
 
 /* Raw negative draws of the last train_batch call: host uint32[n_pairs*k] (nullable); n_pairs nullable. */

@@ -64,6 +64,7 @@ def lib():
             "orc_book_compute": (u64, [vp, u32]),
             "orc_book_apply": (u32, [vp, u32, u64]),
             "orc_book_size": (u32, [vp, u32]),
+            "orc_cosine_difference": (None, [vp, vp, u32, u32, vp]),
             "orc_threads": (C.c_int, []),
         }
         for name, (res, args) in sig.items():
@@ -101,6 +102,16 @@ def negative(seed, replica, batch_index, p, j, thresh, alias):
 def init_input_table(seed, V, d):
     out = np.empty((V, d), dtype=np.float32)
     lib().orc_init_input_table(seed, V, d, _ptr(out))
+    return out
+
+
+def cosine_difference(a, b):
+    """1 - cos(a_r, b_r) per row of two float32 arrays [n, d]."""
+    a = np.ascontiguousarray(a, dtype=np.float32)
+    b = np.ascontiguousarray(b, dtype=np.float32)
+    assert a.shape == b.shape and a.ndim == 2
+    out = np.empty(a.shape[0], dtype=np.float32)
+    lib().orc_cosine_difference(_ptr(a), _ptr(b), a.shape[0], a.shape[1], _ptr(out))
     return out
 
 

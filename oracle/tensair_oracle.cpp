@@ -459,6 +459,23 @@ uint32_t orc_book_apply(Book* b, uint32_t model, uint64_t grad) {
 }
 uint32_t orc_book_size(Book* b, uint32_t model) { return (uint32_t)b->G[model].size(); }
 
+// Cosine difference 1 - cos(a_r, b_r) per row (the drift metric of Section 4.3, Table 1), fp64 arithmetic;
+// two zero rows give 0, one zero row gives 1.
+void orc_cosine_difference(const float* a, const float* b, uint32_t nrows, uint32_t d, float* out) {
+    for (uint32_t r = 0; r < nrows; ++r) {
+        double ab = 0.0, aa = 0.0, bb = 0.0;
+        for (uint32_t e = 0; e < d; ++e) {
+            const double x = a[(size_t)r * d + e], y = b[(size_t)r * d + e];
+            ab += x * y; aa += x * x; bb += y * y;
+        }
+        double diff;
+        if (aa == 0.0 && bb == 0.0) diff = 0.0;
+        else if (aa == 0.0 || bb == 0.0) diff = 1.0;
+        else diff = 1.0 - ab / (std::sqrt(aa) * std::sqrt(bb));
+        out[r] = (float)diff;
+    }
+}
+
 int orc_threads() {
 #ifdef _OPENMP
     return omp_get_max_threads();

@@ -73,6 +73,8 @@ SYMBOLS = {
     "tensair_sync": (_int, [_vp]),
     "tensair_read_embeddings": (_int, [_vp, _u32, _int, _u32, _u32, _vp]),
     "tensair_write_embeddings": (_int, [_vp, _u32, _int, _u32, _u32, _vp]),
+    "tensair_snapshot_rows": (_int, [_vp, _u32, _int, _u32, _u32, _vp]),
+    "tensair_cosine_difference": (_int, [_vp, _u32, _int, _u32, _u32, _vp, _vp]),
     "tensair_read_negatives": (_int, [_vp, _vp, _P(_u32)]),
     "tensair_read_scalars": (_int, [_vp, _vp]),
     "tensair_read_message": (_int, [_vp, _u32, _u64, _P(_u32), _vp, _vp]),
@@ -299,6 +301,22 @@ class Context:
         rows = np.ascontiguousarray(rows, dtype=np.float32)
         _check(lib().tensair_write_embeddings(self._h, replica, which, row0, rows.shape[0], _np_ptr(rows)),
                "tensair_write_embeddings", self._h)
+
+    def tensair_snapshot_rows(self, replica, which, row0=0, nrows=None):
+        """A dense float32 CUDA tensor [nrows, d] holding the rows as they are now."""
+        nrows = self.cfg.V - row0 if nrows is None else nrows
+        snap = self.torch.empty((nrows, self.cfg.d), dtype=self.torch.float32, device=self.device)
+        _check(lib().tensair_snapshot_rows(self._h, replica, which, row0, nrows, snap.data_ptr()),
+               "tensair_snapshot_rows", self._h)
+        return snap
+
+    def tensair_cosine_difference(self, replica, which, snap, row0=0):
+        """float32 CUDA tensor [nrows]: 1 - cos(row now, row in `snap`)."""
+        assert snap.is_cuda and snap.dtype == self.torch.float32 and snap.is_contiguous() and snap.shape[1] == self.cfg.d
+        out = self.torch.empty(snap.shape[0], dtype=self.torch.float32, device=self.device)
+        _check(lib().tensair_cosine_difference(self._h, replica, which, row0, snap.shape[0], snap.data_ptr(),
+                                               out.data_ptr()), "tensair_cosine_difference", self._h)
+        return out
 
     def tensair_read_negatives(self) -> np.ndarray:
         n = C.c_uint32(0)

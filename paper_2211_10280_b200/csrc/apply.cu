@@ -144,6 +144,49 @@ cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float*
     return cudaGetLastError();
 }
 
+// One warp per row: dot product and both squared norms in fp64, combined by shuffles.
+__global__ void __launch_bounds__(256)
+k_cosine_difference(const float* __restrict__ rows, const float* __restrict__ snap, float* __restrict__ out,
+                    uint32_t nrows, uint32_t d, uint32_t stride) {
+    const uint32_t lane = threadIdx.x & 31;
+    const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
+    const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
+    for (uint32_t r = warp; r < nrows; r += nwarps) {
+        const float* a = rows + (size_t)r * stride;
+        const float* b = snap + (size_t)r * d;
+        double ab = 0.0, aa = 0.0, bb = 0.0;
+        for (uint32_t e = lane; e < d; e += 32) {
+            const double x = (double)a[e], y = (double)b[e];
+            ab = fma(x, y, ab);
+            aa = fma(x, x, aa);
+            bb = fma(y, y, bb);
+        }
+#pragma unroll
+        for (int o = 16; o > 0; o >>= 1) {
+            ab += __shfl_xor_sync(0xFFFFFFFFu, ab, o);
+            aa += __shfl_xor_sync(0xFFFFFFFFu, aa, o);
+            bb += __shfl_xor_sync(0xFFFFFFFFu, bb, o);
+        }
+        if (lane == 0) {
+            double diff;
+            if (aa == 0.0 && bb == 0.0) diff = 0.0;
+            else if (aa == 0.0 || bb == 0.0) diff = 1.0;
+            else diff = 1.0 - ab / (sqrt(aa) * sqrt(bb));
+            out[r] = (float)diff;
+        }
+    }
+}
+
+cudaError_t launch_cosine_difference(const Launcher& L, const float* rows, const float* snap, float* out, uint32_t nrows,
+                                     const Shape& s) {
+    if (!nrows) return cudaSuccess;
+    uint32_t blocks = (nrows + 7) / 8;
+    if (blocks > (uint32_t)L.sms * 32) blocks = (uint32_t)L.sms * 32;
+    Timed timed(L, K_COSINE);
+    k_cosine_difference<<<blocks, 256, 0, L.stream>>>(rows, snap, out, nrows, s.d, s.stride);
+    return cudaGetLastError();
+}
+
 cudaError_t launch_apply(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
                          float* table, const Shape& s) {
     return launch_apply_rows(L, hdr, ids, delta, table, s, 0);

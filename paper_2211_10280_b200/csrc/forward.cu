@@ -208,8 +208,8 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err) {
     if (n < 2) return cudaSuccess;
     const size_t row = (size_t)s.stride * 4;
-    const int cr = g_forward_rows == 8 || g_forward_rows == 16 ? g_forward_rows : 8;
-    int blocks_per_sm = g_forward_blocks > 0 ? g_forward_blocks : (cr == 16 ? 5 : 8);
+    const int cr = g_forward_rows == 4 || g_forward_rows == 8 || g_forward_rows == 16 ? g_forward_rows : 8;
+    int blocks_per_sm = g_forward_blocks > 0 ? g_forward_blocks : (cr == 16 ? 5 : cr == 8 ? 8 : 10);
     // rows staged per chunk: as many of the cr as fit the shared memory share of one block
     uint32_t chunk_rows = s.K1 < (uint32_t)cr ? s.K1 : (uint32_t)cr;
     const size_t budget = (size_t)216 * 1024 / blocks_per_sm - 1024;
@@ -234,7 +234,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
                                                                       chunk_rows, t4, rows, rec, gin_pos,      \
                                                                       loss_pos, err);                           \
     } while (0)
-#define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else TENSAIR_FWD(NV, 8); } while (0)
+#define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)
     if (s.d4 <= 32) TENSAIR_FWD_NV(1);
     else if (s.d4 <= 64) TENSAIR_FWD_NV(2);
     else if (s.d4 <= 96) TENSAIR_FWD_NV(3);

@@ -403,6 +403,33 @@ int tensair_write_embeddings(tensair_ctx* ctx, uint32_t replica, int which, uint
     return copy_rows(ctx, replica, which, row0, nrows, const_cast<float*>(host_src), false);
 }
 
+int tensair_snapshot_rows(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows, float* snap_dev) {
+    if (!ctx || replica >= ctx->cfg.W || (which != 0 && which != 1) || (uint64_t)row0 + nrows > ctx->cfg.V ||
+        (!snap_dev && nrows))
+        return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    if (!nrows) return TENSAIR_OK;
+    const tensair_config& c = ctx->cfg;
+    const float* src = ctx->table_of(replica) + ((size_t)which * c.V + row0) * ctx->cv.stride;
+    TENSAIR_CUDA(ctx, cudaMemcpy2DAsync(snap_dev, (size_t)c.d * 4, src, (size_t)ctx->cv.stride * 4, (size_t)c.d * 4, nrows,
+                                        cudaMemcpyDeviceToDevice, ctx->stream));
+    return TENSAIR_OK;
+}
+
+int tensair_cosine_difference(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows,
+                              const float* snap_dev, float* out_dev) {
+    if (!ctx || replica >= ctx->cfg.W || (which != 0 && which != 1) || (uint64_t)row0 + nrows > ctx->cfg.V ||
+        ((!snap_dev || !out_dev) && nrows))
+        return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const tensair_config& c = ctx->cfg;
+    const float* rows = ctx->table_of(replica) + ((size_t)which * c.V + row0) * ctx->cv.stride;
+    TENSAIR_CUDA(ctx, launch_cosine_difference(ctx->L, rows, snap_dev, out_dev, nrows, ctx->shape));
+    return TENSAIR_OK;
+}
+
 int tensair_read_negatives(tensair_ctx* ctx, uint32_t* host_neg, uint32_t* n_pairs) {
     if (!ctx || !ctx->have_last) return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);

@@ -344,3 +344,82 @@ def test_full_size_large_dasgd_two_steps(torch):
             got = g.tensair_read_embeddings(j, which)
             assert rel_err(got[rows], want[rows]) <= 1e-4
             assert rel_err(got, want) <= 1e-4
+
+
+# ------------------------------------------------------------------ drift metric
+def test_cosine_difference_of_a_snapshot_matches_the_oracle(torch):
+    import oracle as orc
+
+    wl = synth.scaled(synth.TINY, V=60_000, d=300, batches=6)
+    stream = synth.token_stream(wl, 0)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 12, scale=0.1)
+    _, g = make_pair(wl, counts=synth.stream_counts([stream], wl.V), init_in=t_in, init_out=t_out)
+    snaps = [g.tensair_snapshot_rows(0, which) for which in (0, 1)]
+    assert np.array_equal(snaps[0].cpu().numpy(), t_in) and np.array_equal(snaps[1].cpu().numpy(), t_out)
+    for b in range(6):
+        g.tensair_train_batch(0, dev(torch, stream[b]), b)
+    for which, before in ((0, t_in), (1, t_out)):
+        got = g.tensair_cosine_difference(0, which, snaps[which]).cpu().numpy()
+        want = orc.cosine_difference(g.tensair_read_embeddings(0, which), before)
+        np.testing.assert_allclose(got, want, rtol=0, atol=2e-7)
+        assert got.max() > 1e-4 and (np.abs(got) < 1e-15).sum() > 0          # touched rows moved, untouched rows did not
+    part = g.tensair_snapshot_rows(0, 1, row0=100, nrows=50)
+    assert np.array_equal(part.cpu().numpy(), g.tensair_read_embeddings(0, 1, 100, 50))
+    assert np.abs(g.tensair_cosine_difference(0, 1, part, row0=100).cpu().numpy()).max() < 1e-15
+
+
+# ------------------------------------------------------------------ launch variants give the same bits
+def test_fused_and_one_by_one_application_are_bit_identical(torch):
+    from paper_2211_10280_b200 import binding as B
+
+    wl = synth.scaled(synth.LARGE_DRIFT, V=30_000, d=40, batch=1024, W=5, k=6, drift_every=0,
+                      stream_seeds=(6, 7, 8, 9, 10))
+    streams = synth.all_streams(wl, 7)
+    counts = synth.stream_counts(streams, wl.V)
+    outs = []
+    try:
+        for fuse in (1, 0):
+            B.tensair_tune("fuse_apply", fuse)
+            _, g = make_pair(wl, counts=counts)
+            for t in range(7):
+                for i in range(wl.W):
+                    g.tensair_train_batch(i, dev(torch, streams[i][t]), t)
+                for j in range(wl.W):
+                    g.tensair_apply_messages(j, t)
+            g.tensair_drain()
+            outs.append([g.tensair_read_embeddings(j, which) for j in range(wl.W) for which in (0, 1)])
+            g.close()
+    finally:
+        B.tensair_tune("fuse_apply", 1)
+    for a, b in zip(*outs):
+        assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
+
+
+def test_full_size_drift_workload_with_sampler_rebuild(torch):
+    """V = 1M, d = 300, batch 16384, k = 15, W = 8, delay <= 2, Zipf 1.1 with a permuted vocabulary: two steps,
+    the sampler rebuilt from the running counts in between, everything against the oracle."""
+    wl = synth.scaled(synth.LARGE_DRIFT, drift_every=1)
+    steps = 2
+    streams = synth.all_streams(wl, steps)
+    o, g = make_pair(wl)
+    dstreams = [dev(torch, s) for s in streams]
+    for t in range(steps):
+        if t:
+            o.update_sampler()
+            g.tensair_update_sampler()
+            assert all(np.array_equal(a, b) for a, b in zip(o.sampler(), g.tensair_read_sampler()))
+        for i in range(wl.W):
+            rc, loss_o, nrows = o.train_batch(i, streams[i][t], t)
+            assert rc == 0
+            loss_g, info = g.tensair_train_batch(i, dstreams[i][t], t, want_loss=True, want_info=True)
+            assert info.n_rows == nrows and info.n_pairs == 163_810
+            assert loss_g == pytest.approx(loss_o, rel=1e-5)
+            if i in (0, wl.W - 1):
+                assert np.array_equal(o.read_negatives(), g.tensair_read_negatives())
+                compare_message(o, g, i, t, TOL_ONE if t == 0 else 1e-4)
+        for j in range(wl.W):
+            assert o.apply_messages(j, t) == g.tensair_apply_messages(j, t)
+    for j in (0, 3, wl.W - 1):
+        assert np.array_equal(o.delivery_log(j), g.tensair_read_delivery_log(j))
+        for which in (0, 1):
+            assert rel_err(g.tensair_read_embeddings(j, which), o.read_embeddings(j, which)) <= 1e-4

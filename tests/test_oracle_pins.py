@@ -539,3 +539,21 @@ def test_result_does_not_depend_on_thread_count(tmp_path):
         subprocess.check_call([sys.executable, "-c", code, str(f)], env=env)
         outs.append(np.load(f))
     assert np.array_equal(outs[0].view(np.uint64), outs[1].view(np.uint64))
+
+
+# ------------------------------------------------------------------ drift metric
+def test_cosine_difference_special_cases_and_library_formula():
+    rng = np.random.default_rng(3)
+    a = rng.standard_normal((50, 7)).astype(np.float32)
+    b = rng.standard_normal((50, 7)).astype(np.float32)
+    got = oracle.cosine_difference(a, b)
+    a64, b64 = a.astype(np.float64), b.astype(np.float64)
+    want = 1.0 - np.einsum("ij,ij->i", a64, b64) / (np.linalg.norm(a64, axis=1) * np.linalg.norm(b64, axis=1))
+    np.testing.assert_allclose(got, want, rtol=0, atol=1e-7)
+    assert np.all(oracle.cosine_difference(a, 3.5 * a) < 1e-7)                    # same direction, any length
+    np.testing.assert_allclose(oracle.cosine_difference(a, -a), 2.0, atol=1e-7)   # opposite
+    e = np.eye(4, dtype=np.float32)
+    np.testing.assert_allclose(oracle.cosine_difference(e, np.roll(e, 1, axis=0)), 1.0, atol=0)   # orthogonal
+    z = np.zeros((2, 4), np.float32)
+    assert oracle.cosine_difference(z, z).tolist() == [0.0, 0.0]
+    assert oracle.cosine_difference(z, e[:2]).tolist() == [1.0, 1.0]
