@@ -39,14 +39,14 @@ METRIC = "SGNS (center,context) pairs/sec on 1 B200; achieved HBM GB/s vs peak"
 UNIT = "pairs/s"
 FALLBACK_HBM_GBS = 6650.0
 
-# DRAM bytes (read + write) per message row of the message-apply kernel, from the ncu capture summarised in
-# profiles/k_apply_small_case_V250k_W2.md (780.3 MB for a 224.6 K-row message; the kernel is a pure stream,
-# so traffic is proportional to the rows of the message).  Only valid for the source the capture ran.
-NCU_TRAFFIC = {"apply_message": {"bytes_per_row": 3474.0, "source": "paper_2211_10280_b200/csrc/apply.cu",
-                                 "sha256": "aed4fc3b02cdefba7ba9880789b118ad30969231c9c0bae3c29f1c8253db1cf7"}}
+# DRAM traffic (dram__bytes_read.sum + dram__bytes_write.sum) of a kernel relative to its algorithmic bytes, from
+# the ncu captures summarised under profiles/ on a reduced case; the apply kernels are pure streams over the rows
+# of their messages, so traffic grows in proportion to the algorithmic bytes of a launch.  Only valid for the
+# source file the capture ran (checked by its SHA-256), null otherwise.
+NCU_TRAFFIC = {}
 
 
-def ncu_traffic(kernel: str, rows: float):
+def ncu_traffic(kernel: str, algorithmic_bytes: float):
     rec = NCU_TRAFFIC.get(kernel)
     if not rec:
         return None
@@ -55,7 +55,7 @@ def ncu_traffic(kernel: str, rows: float):
     src = ROOT / rec["source"]
     if not src.exists() or hashlib.sha256(src.read_bytes()).hexdigest() != rec["sha256"]:
         return None          # the kernel changed since the counters were taken
-    return int(rec["bytes_per_row"] * rows)
+    return int(rec["traffic_per_algorithmic_byte"] * algorithmic_bytes)
 
 
 def hbm_peak():
@@ -168,7 +168,7 @@ def run_ours(args):
         B.tensair_tune(item.split("=")[0], int(item.split("=")[1]))
     K, Wm = args.steps, max(args.warmup, 3)
     Kp = min(K, 8)                                          # steps of the per-kernel timing pass
-    total_steps = 2 * (Wm + K) + Kp
+    total_steps = 2 * (Wm + K) + Kp + wl.max_delay
     toks_np, counts = rank_streams(wl, rank, total_steps)
     P = wl.pairs_per_batch
 
@@ -178,6 +178,8 @@ def run_ours(args):
     toks_pin = torch.from_numpy(toks_np).pin_memory()
     n_rows = {}
 
+    msg_ids = {}
+
     def step(t, host=False, info=False):
         for i in range(wl.W):
             if host:
@@ -186,6 +188,8 @@ def run_ours(args):
                 _, inf = ctx.tensair_train_batch(i, toks_dev[t, i], t, want_info=info)
             if inf is not None:
                 n_rows[(i, t)] = (inf.n_rows, inf.n_in_rows)
+            if info:
+                msg_ids[(i, t)] = ctx.tensair_read_message_ids(i, t)
         for j in range(wl.W):
             ctx.tensair_apply_messages(j, t)
 
@@ -230,6 +234,9 @@ def run_ours(args):
     t += K
 
     # per-kernel pass: CUDA events around every launch, on the library's stream
+    for _ in range(wl.max_delay):                            # so that every message applied below has its ids on record
+        step(t, info=True)
+        t += 1
     ctx.tensair_profile(True)
     ctx.tensair_profile_read()
     first_prof = t
@@ -251,18 +258,27 @@ def run_ours(args):
     U = float(np.mean([m[0] for m in msgs]))
     U_in = float(np.mean([m[1] for m in msgs]))
     U_out = U - U_in
-    applied = []
+    applied, groups = [], {}
     for j in range(wl.W):
         for origin, snd, due, at, _ in ctx.tensair_read_delivery_log(j).tolist():
             if first_prof <= at < first_prof + Kp and (snd, origin) in n_rows:
                 applied.append(n_rows[(snd, origin)][0])
+                groups.setdefault((j, at), []).append((snd, origin))
     U_applied = float(np.mean(applied)) if applied else U
+    # one pass over the receiver's table for all messages due: every delta row read once, every row of the
+    # union of their id sets read and written once
+    fused_bytes = []
+    for members in groups.values():
+        if len(members) >= 2 and all(m in msg_ids and msg_ids[m] is not None for m in members):
+            union = np.unique(np.concatenate([msg_ids[m] for m in members])).size
+            fused_bytes.append(sum(msg_ids[m].size for m in members) * (row + 4) + union * 2 * row)
     algo = {
         "forward": (U_out + U_in) * row,                                   # every touched row gathered once
         "reduce_rows": U * (row + 4) + U_out * 2 * row,                   # message write + read/write of output rows
         "apply_message": U_applied * (row + 4 + 2 * row),                 # delta read + row read + row write
     }
-    algo["apply_fused"] = algo["apply_message"] * (len(applied) / max(1, prof.get("apply_fused", (0, 0))[0]))
+    if fused_bytes:
+        algo["apply_fused"] = float(np.mean(fused_bytes))
     tot_ms = sum(v[1] for v in prof.values()) or 1.0
     kernels = {}
     for name, (cnt, ms) in prof.items():
@@ -279,7 +295,7 @@ def run_ours(args):
     achieved = kernels[dom]["gbs"]
     roofline = {"bound": "hbm", "kernel": dom, "achieved": achieved, "peak": peak, "peak_source": f"of {peak_kind}",
                 "unit": "GB/s", "frac": round(achieved / peak, 4),
-                "traffic": ncu_traffic(dom, U_applied if dom == "apply_message" else U),
+                "traffic": ncu_traffic(dom, kernels[dom]["algorithmic_bytes"]),
                 "algorithmic_bytes": kernels[dom]["algorithmic_bytes"],
                 "avg_ms": kernels[dom]["avg_ms"], "share_of_device_time": kernels[dom]["share"]}
     own = U * row + U * (row + 4) + U * (row + 4 + 2 * row)

@@ -345,6 +345,18 @@ class Context:
                "tensair_read_message", self._h)
         return ids, delta
 
+    def tensair_read_message_ids(self, replica, batch_index):
+        """The row ids of a held message (uint32[n]) without its delta rows, or None."""
+        n = C.c_uint32(0)
+        rc = lib().tensair_read_message(self._h, replica, batch_index, C.byref(n), None, None)
+        if rc == ENOTFOUND:
+            return None
+        _check(rc, "tensair_read_message", self._h)
+        ids = np.empty(n.value, np.uint32)
+        _check(lib().tensair_read_message(self._h, replica, batch_index, None, _np_ptr(ids), None),
+               "tensair_read_message", self._h)
+        return ids
+
     def tensair_read_sampler(self):
         V = self.cfg.V
         thresh, alias, counts = np.empty(V, np.uint32), np.empty(V, np.uint32), np.empty(V, np.uint64)
