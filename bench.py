@@ -43,7 +43,9 @@ FALLBACK_HBM_GBS = 6650.0
 # the ncu captures summarised under profiles/ on a reduced case; the apply kernels are pure streams over the rows
 # of their messages, so traffic grows in proportion to the algorithmic bytes of a launch.  Only valid for the
 # source file the capture ran (checked by its SHA-256), null otherwise.
-NCU_TRAFFIC = {}
+NCU_TRAFFIC = {"apply_fused": {"traffic_per_algorithmic_byte": 0.996, "source": "paper_2211_10280_b200/csrc/apply.cu",
+                               "sha256": "68c94b2b3562f04ec06ec7ab85632d6640ba520cbf1c509e65fdade149f06ed0",
+                               "profile": "profiles/k_apply_fused_small_case_V250k_W4.md"}}
 
 
 def ncu_traffic(kernel: str, algorithmic_bytes: float):
@@ -188,7 +190,7 @@ def run_ours(args):
                 _, inf = ctx.tensair_train_batch(i, toks_dev[t, i], t, want_info=info)
             if inf is not None:
                 n_rows[(i, t)] = (inf.n_rows, inf.n_in_rows)
-            if info:
+            if info or args.log_applies:
                 msg_ids[(i, t)] = ctx.tensair_read_message_ids(i, t)
         for j in range(wl.W):
             ctx.tensair_apply_messages(j, t)
@@ -279,6 +281,22 @@ def run_ours(args):
     }
     if fused_bytes:
         algo["apply_fused"] = float(np.mean(fused_bytes))
+    if args.log_applies:
+        # every apply call of the run in call order, with the bytes its launch has to move (for matching ncu captures)
+        calls = {}
+        for j in range(wl.W):
+            for origin, snd, due, at, _ in ctx.tensair_read_delivery_log(j).tolist():
+                calls.setdefault((at, j), []).append((snd, origin))
+        with open(args.log_applies, "w") as fh:
+            for (at, j), members in sorted(calls.items()):
+                ids = [msg_ids.get(m) for m in members]
+                if any(x is None for x in ids):
+                    continue
+                union = np.unique(np.concatenate(ids)).size
+                nbytes = sum(x.size for x in ids) * (row + 4) + union * 2 * row
+                fh.write(json.dumps({"step": at, "receiver": j, "messages": len(members), "kernel":
+                                     "k_apply_fused" if len(members) > 1 else "k_apply", "delta_rows": sum(x.size for x in ids),
+                                     "union_rows": union, "algorithmic_bytes": nbytes}) + "\n")
     tot_ms = sum(v[1] for v in prof.values()) or 1.0
     kernels = {}
     for name, (cnt, ms) in prof.items():
@@ -450,6 +468,7 @@ def main():
     ap.add_argument("--workload", default=synth.LARGE_DASGD.name)
     ap.add_argument("--override", default="", help="comma-separated field=value replacements of the workload")
     ap.add_argument("--tune", default="", help="comma-separated knob=value pairs passed to tensair_tune (sweeps)")
+    ap.add_argument("--log-applies", default="", help="write one JSON line per apply call (bytes to move) to this file")
     ap.add_argument("--sweep", action="store_true", help="run the 32-point throughput sweep instead (one line per point)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
     args = ap.parse_args()
