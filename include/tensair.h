@@ -74,7 +74,7 @@ typedef struct tensair_config {
     uint32_t batch;           /* maximum centre tokens per mini-batch */
     uint32_t W;               /* logical replicas ("Model instances"), 1 <= W <= 256 */
     float lr;                 /* learning rate alpha of Eq. 1 */
-    uint32_t max_grad_buffer; /* Algorithm 1's maxGradBuffer; only 1 is supported */
+    uint32_t max_grad_buffer; /* Algorithm 1's maxGradBuffer m, 1..8: a replica sends after every m-th of its batches */
     uint32_t max_delay;       /* messages are delivered 0..max_delay whole steps after their origin step */
     uint32_t row_stride;      /* floats between consecutive rows; 0 = d rounded up to a multiple of 8 */
     uint64_t seed;            /* key of the counter-based generator (negatives, delays, seeded init) */
@@ -149,6 +149,10 @@ TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
  *   message    one delta row fp32(-lr * gradient) per touched row, ids ascending;
  *   local GA   the message is applied to the replica at once (staleness 0);
  *   send       it is filed for every other replica at step batch_index + delay(batch_index, replica, j).
+ *              With max_grad_buffer = m > 1 (Algorithm 1: "gradients += gradient", sent when the count
+ *              reaches maxGradBuffer) only every m-th batch of a replica sends: the sum of its last m
+ *              messages over the union of their rows, each row's deltas added in fp32 in the order they
+ *              were computed; tensair_read_message then holds only for those batch indices.
  * tokens_dev   device, int32[n_tokens], borrowed until the stream has passed this call; n_tokens <= batch.
  * batch_index  the global step t of this batch (< 2^32); it selects the random draws and the message slot.
  * loss_out     host, nullable.  Non-NULL: receives the sum of the batch's pair losses and the call synchronises.
@@ -177,6 +181,7 @@ TENSAIR_API int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, con
  * tensair_init but from a fixed 32 MiB array inside the library image, which every GPU that loads the
  * library reserves until the process exits.  The call allocates nothing on the device, neither
  * directly nor through a library.
+ *   - Only for max_grad_buffer = 1 (TENSAIR_EINVAL otherwise).
  *   - TENSAIR_ENOMEM (with the sizes in tensair_last_error) when the context's configuration needs
  *     more per-batch memory than the array holds; roughly batch * 2 * window * (k+1) * 32 bytes plus
  *     batch * row_stride * 8 bytes must stay below 32 MiB.

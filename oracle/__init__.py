@@ -43,6 +43,7 @@ def lib():
             "orc_init_input_table": (None, [u64, u32, u32, vp]),
             "orc_create": (vp, [u32, u32, u32, u32, u32, u32, f32, u32, u64, u32, vp, vp, vp]),
             "orc_destroy": (None, [vp]),
+            "orc_set_max_grad_buffer": (None, [vp, u32]),
             "orc_update_sampler": (None, [vp]),
             "orc_get_sampler": (None, [vp, vp, vp, vp]),
             "orc_batch_loss": (f64, [vp, u32, vp, u32, u64]),
@@ -123,7 +124,7 @@ class Oracle:
     """The oracle's model replicas, sampler and message exchange."""
 
     def __init__(self, V, d, window, k, batch, W=1, lr=0.025, max_delay=0, seed=0,
-                 counts=None, init_in=None, init_out=None, reduction=0):
+                 counts=None, init_in=None, init_out=None, reduction=0, max_grad_buffer=1):
         self.V, self.d, self.window, self.k, self.batch, self.W = V, d, window, k, batch, W
         self.seed = seed
         if counts is not None:
@@ -137,6 +138,7 @@ class Oracle:
             assert init_out.shape == (V, d)
         self._h = lib().orc_create(V, d, window, k, batch, W, lr, max_delay, seed, reduction,
                                    _ptr(counts), _ptr(init_in), _ptr(init_out))
+        lib().orc_set_max_grad_buffer(self._h, max_grad_buffer)
 
     def close(self):
         if self._h:

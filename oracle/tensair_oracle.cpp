@@ -17,6 +17,10 @@
 //   * The loss is the textbook skip-gram negative-sampling objective (the paper only names "a
 //     default skip-gram model"): per pair  -log s(u_o.v_c) - sum_j log s(-u_nj.v_c).
 //
+// With maxGradBuffer = m > 1 a replica sends only after every m-th mini-batch: the sum of the m buffered
+// gradient messages over the union of their rows (fp32 additions in the order computed).  The
+// staleness snapshot G_i of such a message is taken when it is sent.
+//
 // Arithmetic: tables are stored in fp32; every dot product, sigmoid, loss term and gradient sum is
 // taken in fp64 from those fp32 values; a delta row is fp32(-scale * sum) with scale = (double)lr when
 // the batch loss is the sum of the pair losses and (double)lr / (number of pairs) when it is their
@@ -127,7 +131,7 @@ struct Delivery { uint64_t due, origin; uint32_t sender; };
 struct LogRec { uint64_t origin, due, applied_at; uint32_t sender, staleness; };
 
 struct Oracle {
-    uint32_t V, d, window, k, batch, W, max_delay, reduction;
+    uint32_t V, d, window, k, batch, W, max_delay, reduction, max_grad_buffer = 1;
     float lr;
     uint64_t seed;
     std::vector<std::vector<float>> tin, tout;   // per replica V*d
@@ -142,6 +146,7 @@ struct Oracle {
     std::vector<double> last_g;                               // P*(1+k), masked -> 0
     uint32_t last_pairs = 0;
     std::pair<uint32_t, uint64_t> last_key{0, 0};
+    std::vector<std::vector<Message>> buffered;               // per replica: gradients computed and not yet sent
 };
 
 uint32_t delay_of(const Oracle& o, uint64_t step, uint32_t sender, uint32_t receiver) {
@@ -231,7 +236,7 @@ Oracle* orc_create(uint32_t V, uint32_t d, uint32_t window, uint32_t k, uint32_t
     if (counts) std::copy(counts, counts + V, o->counts.begin());
     o->thresh.resize(V); o->alias.resize(V);
     build_alias(o->counts.data(), V, o->thresh.data(), o->alias.data());
-    o->inbox.resize(W); o->applied.resize(W); o->log.resize(W);
+    o->inbox.resize(W); o->applied.resize(W); o->log.resize(W); o->buffered.resize(W);
     return o;
 }
 
@@ -358,9 +363,38 @@ int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t
         for (uint32_t e = 0; e < d; ++e) m.delta[r * d + e] = (float)(-scale * sum[e]);
     }
 
-    // local apply (staleness 0), then send to every other replica
-    m.g_snapshot.assign(o->applied[replica].begin(), o->applied[replica].end());
+    // local apply (staleness 0)
     add_rows(*o, replica, m);
+    if (loss_out) *loss_out = loss;
+    if (n_rows_out) *n_rows_out = (uint32_t)U;
+    // Algorithm 1, train, mini-batch branch: "gradients += gradient; count += 1; if count >= maxGradBuffer:
+    // send".  The buffered gradients are summed row by row in the order they were computed (one fp32
+    // addition per element and buffered gradient; a row missing from a gradient adds nothing), over
+    // the union of their rows; the buffer is emptied after the send.
+    o->buffered[replica].push_back(std::move(m));
+    if (o->buffered[replica].size() < o->max_grad_buffer) return 0;
+    {
+        std::vector<Message>& buf = o->buffered[replica];
+        if (buf.size() == 1) {
+            m = std::move(buf[0]);
+        } else {
+            std::map<uint32_t, std::vector<float>> rows;
+            for (const Message& b : buf)
+                for (size_t r = 0; r < b.ids.size(); ++r) {
+                    auto it = rows.find(b.ids[r]);
+                    if (it == rows.end()) rows.emplace(b.ids[r], std::vector<float>(b.delta.begin() + r * d, b.delta.begin() + (r + 1) * d));
+                    else for (uint32_t e = 0; e < d; ++e) it->second[e] = it->second[e] + b.delta[r * d + e];
+                }
+            m = Message();
+            for (const auto& kv : rows) {
+                m.ids.push_back(kv.first);
+                m.delta.insert(m.delta.end(), kv.second.begin(), kv.second.end());
+            }
+        }
+        buf.clear();
+    }
+    // send to every other replica
+    m.g_snapshot.assign(o->applied[replica].begin(), o->applied[replica].end());
     o->applied[replica].insert(batch_index * o->W + replica);
     m.pending = (int)o->W - 1;
     auto key = std::make_pair(replica, batch_index);
@@ -372,10 +406,10 @@ int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t
     o->msgs[key] = std::move(m);
     auto it = o->msgs.find(prev);
     if (prev != key && it != o->msgs.end() && it->second.pending == 0) o->msgs.erase(it);
-    if (loss_out) *loss_out = loss;
-    if (n_rows_out) *n_rows_out = (uint32_t)U;
     return 0;
 }
+
+void orc_set_max_grad_buffer(Oracle* o, uint32_t m) { o->max_grad_buffer = m < 1 ? 1 : m; }
 
 // Algorithm 1, train(), gradient branch: every pending message for `replica` that is due at or
 // before `step`, in (origin step, sender) order.  Returns how many were applied.

@@ -198,14 +198,15 @@ class Context:
     """Owns the torch allocations a tensair_ctx borrows and forwards calls to the C ABI."""
 
     def __init__(self, V, d, window, k, batch, W=1, lr=0.025, max_delay=0, seed=0, counts=None,
-                 init_in=None, init_out=None, device=0, row_stride=0, stream=None, reduction=SUM):
+                 init_in=None, init_out=None, device=0, row_stride=0, stream=None, reduction=SUM,
+                 max_grad_buffer=1):
         import torch
 
         if not torch.cuda.is_available():
             raise RuntimeError("no CUDA device: the SGNS path has no CPU implementation")
         self.torch = torch
         self.device = torch.device("cuda", device)
-        self.cfg = Config(V=V, d=d, window=window, k=k, batch=batch, W=W, lr=lr, max_grad_buffer=1,
+        self.cfg = Config(V=V, d=d, window=window, k=k, batch=batch, W=W, lr=lr, max_grad_buffer=max_grad_buffer,
                           max_delay=max_delay, row_stride=row_stride, seed=seed, device=device, reduction=reduction)
         self.sizes = tensair_workspace_bytes(self.cfg)
         with torch.cuda.device(self.device):

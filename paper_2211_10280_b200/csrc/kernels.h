@@ -9,13 +9,13 @@ namespace tensair {
 enum KernelKind {
     K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
     K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
-    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_KINDS
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_KINDS
 };
 inline const char* kernel_name(int kind) {
     static const char* const names[K_KINDS] = {
         "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
         "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
-        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference"};
+        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge"};
     return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
 }
 
@@ -113,6 +113,16 @@ struct FusedMessages {
     const uint32_t* buckets[kMaxFused];
 };
 cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float* table, const Shape& s);
+// merge.cu: the sum of up to kMaxMerge buffered messages (each with its bucket index) into one message.
+constexpr int kMaxMerge = 8;
+struct MergeInputs {
+    uint32_t count;
+    const uint32_t* ids[kMaxMerge];
+    const float* delta[kMaxMerge];
+    const uint32_t* buckets[kMaxMerge];
+};
+cudaError_t launch_merge(const Launcher& L, const MergeInputs& in, MsgHeader* hdr, uint32_t* bucket_start, uint32_t* ids,
+                         float* delta, uint32_t* counts, const Shape& s);
 // out[r] = 1 - cos(table row r, snapshot row r) for nrows rows; rows of `rows` are strided, of `snap` dense.
 cudaError_t launch_cosine_difference(const Launcher& L, const float* rows, const float* snap, float* out, uint32_t nrows,
                                      const Shape& s);

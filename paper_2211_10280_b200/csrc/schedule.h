@@ -32,6 +32,7 @@ public:
     std::vector<Due> take_due(uint32_t receiver, uint64_t step, bool drain);
     uint64_t pending(uint32_t receiver) const { return inbox_[receiver].size(); }
     const std::vector<tensair_delivery>& log(uint32_t receiver) const { return log_[receiver]; }
+    bool slot_busy(uint32_t slot) const { return slots_[slot].used && slots_[slot].outstanding; }
     bool slot_holds(uint32_t slot, uint64_t step) const { return slots_[slot].used && slots_[slot].step == step; }
     uint32_t W() const { return W_; }
 

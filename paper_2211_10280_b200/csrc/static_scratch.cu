@@ -63,6 +63,7 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
     const tensair_config& c = ctx->cfg;
     const Carve& cv = ctx->cv;
     if (c.device < 0 || c.device >= kMaxDevices) return TENSAIR_EINVAL;
+    if (c.max_grad_buffer != 1) return TENSAIR_EINVAL;   // buffered gradients are only handled by tensair_train_batch
     StaticCarve sc;
     carve_static(c, cv, sc);
     if (sc.total > kStaticScratchBytes) {

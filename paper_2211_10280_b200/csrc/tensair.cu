@@ -22,7 +22,7 @@ int validate_config(const tensair_config* c) {
     if (c->k < 1 || c->k > 64) return TENSAIR_EINVAL;
     if (c->batch < 1 || c->batch > (1u << 22)) return TENSAIR_EINVAL;
     if (c->W < 1 || c->W > 256) return TENSAIR_EINVAL;
-    if (c->max_grad_buffer != 1) return TENSAIR_EINVAL;
+    if (c->max_grad_buffer < 1 || c->max_grad_buffer > (uint32_t)kMaxMerge) return TENSAIR_EINVAL;
     if (c->max_delay > 64) return TENSAIR_EINVAL;
     if (c->row_stride && (c->row_stride < c->d || c->row_stride % 4)) return TENSAIR_EINVAL;
     if (!(c->lr == c->lr)) return TENSAIR_EINVAL;
@@ -61,6 +61,7 @@ void carve(const tensair_config& c, Carve& k) {
     k.long_rows = take((uint64_t)k.max_long * sizeof(LongRow));
     k.chunk_items = take((uint64_t)k.max_chunks * sizeof(ChunkItem));
     k.partials = take((uint64_t)k.max_chunks * k.stride * 8);
+    k.merge_counts = take((uint64_t)(bucket_count(c.V) + 1) * 4);
     k.total = off;
     k.bucket_off = kHeaderBytes;
     k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
@@ -108,9 +109,18 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                double* loss_out, tensair_msg_info* info) {
     const tensair_config& c = ctx->cfg;
     const Carve& cv = ctx->cv;
-    const int rc = ctx->sched->on_train(replica, batch_index);
-    if (rc != TENSAIR_OK) return rc;
-    const uint32_t slot = ctx->sched->slot_of(replica, batch_index);
+    // maxGradBuffer = 1: the batch's message is built in its send slot and filed at once.  Otherwise it is built
+    // in a buffer slot of the replica, and after every m-th batch the m buffered messages are summed into a send slot.
+    const uint32_t m_buf = c.max_grad_buffer;
+    const uint32_t send_slot = ctx->sched->slot_of(replica, batch_index);
+    const bool sends = m_buf == 1 || ctx->buffered[replica] + 1 == m_buf;
+    if (sends && m_buf > 1 && ctx->sched->slot_busy(send_slot)) return TENSAIR_EPENDING;
+    if (m_buf == 1) {
+        const int rc = ctx->sched->on_train(replica, batch_index);
+        if (rc != TENSAIR_OK) return rc;
+    }
+    const uint32_t slot = m_buf == 1 ? send_slot
+                                     : c.W * (c.max_delay + 1) + replica * m_buf + ctx->buffered[replica];
     const uint32_t pairs = n >= 2 ? pair_count(n, c.window) : 0;
     const uint32_t contrib = pairs * (c.k + 1);
     const uint32_t n_items = pairs ? n + contrib : 0;
@@ -156,6 +166,26 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
         TENSAIR_CUDA(ctx, cudaMemsetAsync(hdr, 0, sizeof(MsgHeader), ctx->stream));
     }
     TENSAIR_CUDA(ctx, launch_bucket_index(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
+    if (m_buf > 1) {
+        ++ctx->buffered[replica];
+        if (sends) {
+            // Algorithm 1: "if gradients_count >= maxGradBuffer: send_gradients(gradients)"
+            MergeInputs in;
+            in.count = m_buf;
+            for (uint32_t b = 0; b < m_buf; ++b) {
+                const uint32_t bs = c.W * (c.max_delay + 1) + replica * m_buf + b;
+                in.ids[b] = ctx->slot_ids(bs);
+                in.delta[b] = ctx->slot_delta(bs);
+                in.buckets[b] = ctx->slot_buckets(bs);
+            }
+            TENSAIR_CUDA(ctx, launch_merge(ctx->L, in, ctx->slot_hdr(send_slot), ctx->slot_buckets(send_slot),
+                                           ctx->slot_ids(send_slot), ctx->slot_delta(send_slot),
+                                           ctx->at<uint32_t>(cv.merge_counts), ctx->shape));
+            const int rc = ctx->sched->on_train(replica, batch_index);
+            if (rc != TENSAIR_OK) return rc;
+            ctx->buffered[replica] = 0;
+        }
+    }
     TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err));
     ctx->last_n = n;
     ctx->last_pairs = pairs;
@@ -226,7 +256,9 @@ int tensair_workspace_bytes(const tensair_config* cfg, tensair_sizes* out) {
     carve(*cfg, cv);
     out->row_stride = cv.stride;
     out->tables_bytes = (uint64_t)cfg->W * 2 * cfg->V * cv.stride * 4;
-    out->pool_bytes = (uint64_t)cfg->W * (cfg->max_delay + 1) * cv.slot_bytes;
+    // one slot per message in flight, plus (maxGradBuffer > 1) the buffered messages of every replica
+    out->pool_bytes = ((uint64_t)cfg->W * (cfg->max_delay + 1) +
+                       (cfg->max_grad_buffer > 1 ? (uint64_t)cfg->W * cfg->max_grad_buffer : 0)) * cv.slot_bytes;
     out->scratch_bytes = cv.total;
     out->max_pairs = cv.max_pairs;
     out->max_rows = cv.max_rows;
@@ -271,6 +303,7 @@ int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const u
     ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount, &ctx->prof};
     if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->sched = new Schedule(cfg->W, cfg->max_delay, cfg->seed);
+    ctx->buffered.assign(cfg->W, 0);
     if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess)

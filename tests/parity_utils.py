@@ -21,13 +21,13 @@ def rel_err(got: np.ndarray, want: np.ndarray) -> float:
     return float(np.max(np.abs(got - want) / np.maximum(np.abs(want), tau)))
 
 
-def make_pair(wl: synth.Workload, counts=None, init_in=None, init_out=None, batch=None):
+def make_pair(wl: synth.Workload, counts=None, init_in=None, init_out=None, batch=None, max_grad_buffer=1):
     """An oracle and a CUDA context with identical configuration and initial state."""
     from paper_2211_10280_b200 import binding as B
 
     kw = dict(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=batch or wl.batch, W=wl.W, lr=wl.lr,
               max_delay=wl.max_delay, seed=wl.seed, counts=counts, init_in=init_in, init_out=init_out,
-              reduction=wl.reduction)
+              reduction=wl.reduction, max_grad_buffer=max_grad_buffer)
     return Oracle(**kw), B.Context(**kw)
 
 

@@ -423,3 +423,35 @@ def test_full_size_drift_workload_with_sampler_rebuild(torch):
         assert np.array_equal(o.delivery_log(j), g.tensair_read_delivery_log(j))
         for which in (0, 1):
             assert rel_err(g.tensair_read_embeddings(j, which), o.read_embeddings(j, which)) <= 1e-4
+
+
+# ------------------------------------------------------------------ maxGradBuffer > 1
+@pytest.mark.parametrize("m", [2, 3])
+def test_buffered_gradients_are_sent_every_mth_batch(torch, m):
+    """Algorithm 1 with maxGradBuffer = m: union of rows, summed deltas, m times fewer messages."""
+    wl = synth.scaled(synth.LARGE_DASGD, V=30_000, d=44, batch=512, k=6, W=3, stream_seeds=(2, 3, 4))
+    steps = 11
+    streams = synth.all_streams(wl, steps)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 21, scale=0.2)
+    o, g = make_pair(wl, counts=synth.stream_counts(streams, wl.V), init_in=t_in, init_out=t_out, max_grad_buffer=m)
+    applied = 0
+    for t in range(steps):
+        for i in range(wl.W):
+            assert o.train_batch(i, streams[i][t], t)[0] == 0
+            g.tensair_train_batch(i, dev(torch, streams[i][t]), t)
+            om, gm = o.read_message(i, t), g.tensair_read_message(i, t)
+            assert (om is None) == (gm is None) == (t % m != m - 1)
+            if om is not None:
+                assert np.array_equal(om[0], gm[0])
+                assert rel_err(gm[1], om[1]) <= TOL_200
+        for j in range(wl.W):
+            n = o.apply_messages(j, t)
+            assert n == g.tensair_apply_messages(j, t)
+            applied += n
+    assert o.drain() == g.tensair_drain()
+    sends = steps // m
+    for j in range(wl.W):
+        log = g.tensair_read_delivery_log(j)
+        assert np.array_equal(o.delivery_log(j), log) and log.shape[0] == sends * (wl.W - 1)
+        assert set((log[:, 0] % m).tolist()) == {m - 1}
+        compare_tables(o, g, j, TOL_200)

@@ -185,7 +185,7 @@ def test_workspace_sizes():
 
 
 @pytest.mark.parametrize("field,value", [("V", 1), ("d", 6), ("d", 2048), ("window", 0), ("window", 17), ("k", 0),
-                                         ("batch", 0), ("W", 0), ("max_grad_buffer", 2), ("row_stride", 2),
+                                         ("batch", 0), ("W", 0), ("max_grad_buffer", 0), ("max_grad_buffer", 9), ("row_stride", 2),
                                          ("reduction", 2)])
 def test_unsupported_configurations_are_rejected(field, value):
     kw = dict(V=100, d=8, window=2, k=3, batch=16, W=1, lr=0.025, max_grad_buffer=1, max_delay=0, row_stride=0,

@@ -557,3 +557,36 @@ def test_cosine_difference_special_cases_and_library_formula():
     z = np.zeros((2, 4), np.float32)
     assert oracle.cosine_difference(z, z).tolist() == [0.0, 0.0]
     assert oracle.cosine_difference(z, e[:2]).tolist() == [1.0, 1.0]
+
+
+# ------------------------------------------------------------------ maxGradBuffer > 1
+def test_buffered_gradients_are_summed_over_the_union_of_their_rows_and_sent_every_mth_batch():
+    # Algorithm 1: gradients += gradient; count += 1; send when count >= maxGradBuffer.
+    V, d, m, T = 300, 6, 3, 7
+    wl = synth.scaled(synth.TINY, V=V, d=d, batch=48, batches=T)
+    stream = synth.token_stream(wl, 0)
+    t_in, t_out = synth.random_tables(V, d, 4, scale=0.3)
+    kw = dict(V=V, d=d, window=wl.window, k=wl.k, batch=wl.batch, lr=0.05, seed=9, init_in=t_in, init_out=t_out)
+    solo = Oracle(W=1, **kw)                               # the same trajectory, every batch message visible
+    pair = Oracle(W=2, max_delay=0, max_grad_buffer=m, **kw)   # replica 1 never trains, so replica 0 receives nothing
+    per_batch = []
+    for t in range(T):
+        assert solo.train_batch(0, stream[t], t)[0] == 0
+        per_batch.append(solo.read_message(0, t))
+        assert pair.train_batch(0, stream[t], t)[0] == 0
+        applied = pair.apply_messages(1, t)
+        assert applied == (1 if t % m == m - 1 else 0)     # m times fewer messages
+        if t % m == m - 1:
+            ids, delta = pair.read_message(0, t)
+            want = {}
+            for bi, bd in per_batch[-m:]:
+                for r, i in enumerate(bi.tolist()):
+                    want[i] = bd[r].copy() if i not in want else (want[i] + bd[r]).astype(np.float32)
+            assert ids.tolist() == sorted(want)
+            assert np.array_equal(delta, np.stack([want[i] for i in ids.tolist()]))
+        else:
+            assert pair.read_message(0, t) is None
+    assert np.array_equal(pair.read_embeddings(0, 1), solo.read_embeddings(0, 1))
+    # the receiver holds init + the two merged messages; the 7th batch is still buffered at the sender
+    log = pair.delivery_log(1)
+    assert log[:, 0].tolist() == [2, 5] and pair.drain() == 0
