@@ -175,7 +175,8 @@ def run_ours(args):
     P = wl.pairs_per_batch
 
     ctx = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=wl.W, lr=wl.lr,
-                    max_delay=wl.max_delay, seed=wl.seed + rank, counts=counts, device=local, reduction=wl.reduction)
+                    max_delay=wl.max_delay, seed=wl.seed + rank, counts=counts, device=local, reduction=wl.reduction,
+                    max_grad_buffer=wl.max_grad_buffer)
     toks_dev = torch.from_numpy(toks_np).cuda()
     toks_pin = torch.from_numpy(toks_np).pin_memory()
     n_rows = {}
@@ -264,7 +265,8 @@ def run_ours(args):
     for j in range(wl.W):
         for origin, snd, due, at, _ in ctx.tensair_read_delivery_log(j).tolist():
             if first_prof <= at < first_prof + Kp and (snd, origin) in n_rows:
-                applied.append(n_rows[(snd, origin)][0])
+                ids_m = msg_ids.get((snd, origin))
+                applied.append(ids_m.size if ids_m is not None else n_rows[(snd, origin)][0])
                 groups.setdefault((j, at), []).append((snd, origin))
     U_applied = float(np.mean(applied)) if applied else U
     # one pass over the receiver's table for all messages due: every delta row read once, every row of the
@@ -317,8 +319,9 @@ def run_ours(args):
                 "algorithmic_bytes": kernels[dom]["algorithmic_bytes"],
                 "avg_ms": kernels[dom]["avg_ms"], "share_of_device_time": kernels[dom]["share"]}
     own = U * row + U * (row + 4) + U * (row + 4 + 2 * row)
-    remote = (wl.W - 1) * U * (row + 4 + 2 * row)
-    step_bytes = wl.W * (own + remote)
+    # remote part: every message applied in the per-kernel pass, per-message model (delta read, row read, row write)
+    remote_per_step = len(applied) / Kp * U_applied * (row + 4 + 2 * row) if applied else 0.0
+    step_bytes = wl.W * own + remote_per_step
     step_gbs = step_bytes / (ms_dev * 1e-3 / K) / 1e9
 
     out = {
@@ -327,7 +330,7 @@ def run_ours(args):
         "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
                    "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
-                   "pairs_per_batch": P, "storage": "f32", "l2": "inputs larger than L2 (tables %.1f GB)" %
+                   "max_grad_buffer": wl.max_grad_buffer, "pairs_per_batch": P, "storage": "f32", "l2": "inputs larger than L2 (tables %.1f GB)" %
                    (ctx.sizes.tables_bytes / 1e9), "parallelism": f"{world} independent replica groups"},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / K,
                 "h2d_bytes_per_step": wl.W * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4)},
@@ -353,7 +356,8 @@ def make_oracle(wl, counts):
     from oracle import Oracle
 
     return Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=wl.W, lr=wl.lr,
-                  max_delay=wl.max_delay, seed=wl.seed, counts=counts, reduction=wl.reduction)
+                  max_delay=wl.max_delay, seed=wl.seed, counts=counts, reduction=wl.reduction,
+                  max_grad_buffer=wl.max_grad_buffer)
 
 
 def cpu_baseline(wl, toks_np, counts, steps):

@@ -39,6 +39,7 @@ class Workload:
     lr: float = 0.025
     seed: int = 0         # library seed (negative sampler, delays)
     reduction: int = 0    # 0: batch loss = sum of the pair losses; 1: their mean
+    max_grad_buffer: int = 1  # a replica sends after every this many of its batches
 
     @property
     def pairs_per_batch(self) -> int:
