@@ -72,6 +72,9 @@ ONE_BATCH = [
     ("d512_k5", synth.scaled(synth.sweep_point(512, 2048, 5), V=30_000), True),
     ("d8_w1_k1", synth.scaled(synth.TINY, V=500, d=8, window=1, k=1, batch=100), True),
     ("d1024_w8_k3", synth.scaled(synth.TINY, V=2000, d=1024, window=8, k=3, batch=300), True),
+    ("w16_k2", synth.scaled(synth.TINY, V=3000, d=64, window=16, k=2, batch=600), True),
+    ("V2_every_other_negative_dropped", synth.scaled(synth.TINY, V=2, d=8, window=2, k=3, batch=50), True),
+    ("k40_d100", synth.scaled(synth.TINY, V=4000, d=100, window=2, k=40, batch=200, reduction=1), True),
 ]
 
 
@@ -118,6 +121,38 @@ def test_hot_rows_take_the_chunked_path(torch):
         g.tensair_train_batch(0, dev(torch, stream[b]), b)
         compare_message(o, g, 0, b, TOL_ONE)
     compare_tables(o, g, 0, 3 * TOL_ONE)
+
+
+def test_batch_of_one_repeated_token(torch):
+    # every pair is (x, x): all input and output contributions fall on two rows, and every draw of x
+    # as a negative is dropped because it equals the positive context
+    wl = synth.scaled(synth.TINY, V=50, d=24, window=4, k=6, batch=400, reduction=1)
+    toks = np.full(wl.batch, 7, np.int32)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 5, scale=0.3)
+    counts = np.ones(wl.V, np.uint64)
+    counts[7] = 1000
+    o, g = make_pair(wl, counts=counts, init_in=t_in, init_out=t_out)
+    rc, loss_o, nrows_o = o.train_batch(0, toks, 0)
+    assert rc == 0
+    loss_g, info = g.tensair_train_batch(0, dev(torch, toks), 0, want_loss=True, want_info=True)
+    assert info.n_in_rows == 1 and info.n_rows == nrows_o
+    neg = g.tensair_read_negatives()
+    assert np.array_equal(o.read_negatives(), neg)
+    go, gg = o.read_g(), g.tensair_read_scalars()
+    assert np.array_equal(go == 0.0, gg == 0.0) and np.max(np.abs(go - gg)) <= 1e-13
+    assert loss_g == pytest.approx(loss_o, rel=1e-12)
+    compare_message(o, g, 0, 0, TOL_ONE)
+    compare_tables(o, g, 0, TOL_ONE)
+
+
+def test_eight_replicas_with_delays_up_to_three_steps(torch):
+    wl = synth.scaled(synth.LARGE_DASGD, V=3000, d=20, batch=128, k=4, W=8, max_delay=3,
+                      stream_seeds=tuple(range(40, 48)))
+    o, g = _run_exchange(torch, wl, 9)
+    assert o.drain() == g.tensair_drain()
+    for j in range(wl.W):
+        assert np.array_equal(o.delivery_log(j), g.tensair_read_delivery_log(j))
+        compare_tables(o, g, j, TOL_200)
 
 
 @pytest.mark.parametrize("n", [0, 1, 2, 3, 5, 6, 10, 11, 12, 509, 512])
