@@ -66,6 +66,7 @@ def lib():
             "orc_book_apply": (u32, [vp, u32, u64]),
             "orc_book_size": (u32, [vp, u32]),
             "orc_cosine_difference": (None, [vp, vp, u32, u32, vp]),
+            "orc_top_drifted": (u32, [vp, u32, u32, vp, vp]),
             "orc_threads": (C.c_int, []),
         }
         for name, (res, args) in sig.items():
@@ -114,6 +115,16 @@ def cosine_difference(a, b):
     out = np.empty(a.shape[0], dtype=np.float32)
     lib().orc_cosine_difference(_ptr(a), _ptr(b), a.shape[0], a.shape[1], _ptr(out))
     return out
+
+
+def top_drifted(diff, k):
+    """(ids, values) of the k largest entries of a float32 array, largest first, smaller index first among equals."""
+    diff = np.ascontiguousarray(diff, dtype=np.float32)
+    ids = np.empty(min(k, diff.size), dtype=np.uint32)
+    vals = np.empty(min(k, diff.size), dtype=np.float32)
+    m = lib().orc_top_drifted(_ptr(diff), diff.size, k, _ptr(ids), _ptr(vals))
+    assert m == ids.size
+    return ids, vals
 
 
 def threads() -> int:

@@ -510,6 +510,29 @@ void orc_cosine_difference(const float* a, const float* b, uint32_t nrows, uint3
     }
 }
 
+// The k rows that drifted most (largest cosine difference first, the smaller row id first among equal
+// values), as Table 1 of Section 4.3 lists the words that moved most.  Values are ranked by the total
+// order of their fp32 bit patterns (-NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN), so the result is
+// defined for every input.  Returns min(k, n), the number of entries written.
+static uint32_t total_order_key(float x) {
+    uint32_t b;
+    std::memcpy(&b, &x, 4);
+    return (b & 0x80000000u) ? ~b : (b | 0x80000000u);
+}
+uint32_t orc_top_drifted(const float* diff, uint32_t n, uint32_t k, uint32_t* ids, float* vals) {
+    std::vector<uint32_t> order(n);
+    for (uint32_t i = 0; i < n; ++i) order[i] = i;
+    std::stable_sort(order.begin(), order.end(), [&](uint32_t a, uint32_t b) {
+        return total_order_key(diff[a]) > total_order_key(diff[b]);   // stable: equal values keep ascending ids
+    });
+    const uint32_t m = k < n ? k : n;
+    for (uint32_t i = 0; i < m; ++i) {
+        ids[i] = order[i];
+        vals[i] = diff[order[i]];
+    }
+    return m;
+}
+
 int orc_threads() {
 #ifdef _OPENMP
     return omp_get_max_threads();

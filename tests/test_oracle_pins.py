@@ -559,6 +559,38 @@ def test_cosine_difference_special_cases_and_library_formula():
     assert oracle.cosine_difference(z, e[:2]).tolist() == [1.0, 1.0]
 
 
+def test_top_drifted_rows_against_a_library_sort_brute_force_and_special_values():
+    rng = np.random.default_rng(11)
+    # distinct finite values: the library's argsort of the negated values is the definition
+    x = rng.permutation(5000).astype(np.float32) / 7.0 - 200.0
+    ids, vals = oracle.top_drifted(x, 37)
+    want = np.argsort(-x.astype(np.float64), kind="stable")[:37]
+    assert ids.tolist() == want.tolist() and np.array_equal(vals, x[want])
+    # heavy ties: equal values come out in ascending row order (lexsort: last key is the primary one)
+    y = rng.integers(0, 6, 2000).astype(np.float32) * 0.25
+    for k in (1, 5, 400, 1999, 2000, 5000):
+        ids, vals = oracle.top_drifted(y, k)
+        want = np.lexsort((np.arange(y.size), -y))[:k]
+        assert ids.tolist() == want.tolist() and np.array_equal(vals, y[want])
+    # brute force on tiny inputs: repeatedly take the maximum, the first one among equals
+    for n in range(0, 7):
+        z = rng.integers(-2, 3, n).astype(np.float32)
+        left = list(range(n))
+        want = []
+        while left:
+            best = max(left, key=lambda i: (z[i], -i))
+            want.append(best)
+            left.remove(best)
+        for k in range(0, n + 2):
+            assert oracle.top_drifted(z, k)[0].tolist() == want[:k]
+    # the total order of the bit patterns: +NaN above +inf, -0 below +0, -NaN lowest
+    s = np.array([0.0, -0.0, np.inf, -np.inf, 1.0, np.nan, -1.0, 0.0], np.float32)
+    s[5] = np.frombuffer(np.uint32(0x7FC00000).tobytes(), np.float32)[0]
+    neg_nan = np.frombuffer(np.uint32(0xFFC00000).tobytes(), np.float32)[0]
+    s = np.append(s, neg_nan).astype(np.float32)
+    assert oracle.top_drifted(s, 9)[0].tolist() == [5, 2, 4, 0, 7, 1, 6, 3, 8]
+
+
 # ------------------------------------------------------------------ maxGradBuffer > 1
 def test_buffered_gradients_are_summed_over_the_union_of_their_rows_and_sent_every_mth_batch():
     # Algorithm 1: gradients += gradient; count += 1; send when count >= maxGradBuffer.
