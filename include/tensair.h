@@ -237,6 +237,19 @@ TENSAIR_API int tensair_snapshot_rows(tensair_ctx* ctx, uint32_t replica, int wh
 TENSAIR_API int tensair_cosine_difference(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint32_t nrows,
                                           const float* snap_dev, float* out_dev);
 
+/*
+ * The rows that drifted most, as Table 1 of Section 4.3 lists the words whose embeddings moved most: the
+ * min(k, nrows) largest entries of diff_dev (device float[nrows], e.g. what tensair_cosine_difference wrote),
+ * largest first, the smaller index first among equal values.  Values are ranked by the total order of their
+ * fp32 bit patterns (-NaN < -inf < ... < -0 < +0 < ... < +inf < +NaN), so the result is defined for any input
+ * and is bit-exact.  ids_dev (device uint32[k], indices into diff_dev) and vals_dev (device float[k]) are the
+ * caller's; entries past min(k, nrows) are left alone; *n_out (host, nullable) receives min(k, nrows).
+ * k <= 4096, else TENSAIR_EINVAL.  Asynchronous on the context's stream; works in the context's scratch, which
+ * stream order keeps apart from the training calls.
+ */
+TENSAIR_API int tensair_top_drifted(tensair_ctx* ctx, const float* diff_dev, uint32_t nrows, uint32_t k, uint32_t* ids_dev,
+                                    float* vals_dev, uint32_t* n_out);
+
 /* ---- parity taps (synchronous; for tests and diagnostics) ---- */
 
 /* Raw negative draws of the last train_batch call: host uint32[n_pairs*k] (nullable); n_pairs nullable. */

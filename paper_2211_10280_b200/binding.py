@@ -75,6 +75,7 @@ SYMBOLS = {
     "tensair_write_embeddings": (_int, [_vp, _u32, _int, _u32, _u32, _vp]),
     "tensair_snapshot_rows": (_int, [_vp, _u32, _int, _u32, _u32, _vp]),
     "tensair_cosine_difference": (_int, [_vp, _u32, _int, _u32, _u32, _vp, _vp]),
+    "tensair_top_drifted": (_int, [_vp, _vp, _u32, _u32, _vp, _vp, _vp]),
     "tensair_read_negatives": (_int, [_vp, _vp, _P(_u32)]),
     "tensair_read_scalars": (_int, [_vp, _vp]),
     "tensair_read_message": (_int, [_vp, _u32, _u64, _P(_u32), _vp, _vp]),
@@ -318,6 +319,16 @@ class Context:
         _check(lib().tensair_cosine_difference(self._h, replica, which, row0, snap.shape[0], snap.data_ptr(),
                                                out.data_ptr()), "tensair_cosine_difference", self._h)
         return out
+
+    def tensair_top_drifted(self, diff, k):
+        """(ids int32-viewable uint32 CUDA tensor [m], values float32 CUDA tensor [m]), m = min(k, len(diff))."""
+        assert diff.is_cuda and diff.dtype == self.torch.float32 and diff.is_contiguous() and diff.dim() == 1
+        ids = self.torch.empty(k, dtype=self.torch.int32, device=self.device)
+        vals = self.torch.empty(k, dtype=self.torch.float32, device=self.device)
+        m = C.c_uint32(0)
+        _check(lib().tensair_top_drifted(self._h, diff.data_ptr(), diff.shape[0], k, ids.data_ptr(), vals.data_ptr(),
+                                         C.byref(m)), "tensair_top_drifted", self._h)
+        return ids[:m.value], vals[:m.value]
 
     def tensair_read_negatives(self) -> np.ndarray:
         n = C.c_uint32(0)

@@ -9,13 +9,13 @@ namespace tensair {
 enum KernelKind {
     K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
     K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
-    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_KINDS
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_KINDS
 };
 inline const char* kernel_name(int kind) {
     static const char* const names[K_KINDS] = {
         "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
         "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
-        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge"};
+        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted"};
     return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
 }
 
@@ -124,6 +124,17 @@ struct MergeInputs {
 cudaError_t launch_merge(const Launcher& L, const MergeInputs& in, MsgHeader* hdr, uint32_t* bucket_start, uint32_t* ids,
                          float* delta, uint32_t* counts, const Shape& s);
 // out[r] = 1 - cos(table row r, snapshot row r) for nrows rows; rows of `rows` are strided, of `snap` dense.
+// Working state of the most-drifted-rows selection, in the context's scratch.
+constexpr uint32_t kTopkMax = 4096;
+struct TopkState {
+    uint64_t prefix;        // leading bytes of the k-th largest rank key found so far
+    uint32_t remaining;     // rank of that key among the keys sharing the prefix
+    uint32_t n_out;
+    uint32_t hist[256];
+    uint64_t keys[kTopkMax];
+};
+cudaError_t launch_top_drifted(const Launcher& L, const float* diff, uint32_t n, uint32_t k, TopkState* st,
+                               uint32_t* ids, float* vals);
 cudaError_t launch_cosine_difference(const Launcher& L, const float* rows, const float* snap, float* out, uint32_t nrows,
                                      const Shape& s);
 // bucket_start[b] = first row of the message with id >= b << kBucketShift, for b in [0, bucket_count(V)].

@@ -62,6 +62,7 @@ void carve(const tensair_config& c, Carve& k) {
     k.chunk_items = take((uint64_t)k.max_chunks * sizeof(ChunkItem));
     k.partials = take((uint64_t)k.max_chunks * k.stride * 8);
     k.merge_counts = take((uint64_t)(bucket_count(c.V) + 1) * 4);
+    k.topk = take(sizeof(TopkState));
     k.total = off;
     k.bucket_off = kHeaderBytes;
     k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
@@ -460,6 +461,18 @@ int tensair_cosine_difference(tensair_ctx* ctx, uint32_t replica, int which, uin
     const tensair_config& c = ctx->cfg;
     const float* rows = ctx->table_of(replica) + ((size_t)which * c.V + row0) * ctx->cv.stride;
     TENSAIR_CUDA(ctx, launch_cosine_difference(ctx->L, rows, snap_dev, out_dev, nrows, ctx->shape));
+    return TENSAIR_OK;
+}
+
+int tensair_top_drifted(tensair_ctx* ctx, const float* diff_dev, uint32_t nrows, uint32_t k, uint32_t* ids_dev,
+                        float* vals_dev, uint32_t* n_out) {
+    if (!ctx || k > kTopkMax) return TENSAIR_EINVAL;
+    const uint32_t m = k < nrows ? k : nrows;
+    if (m && (!diff_dev || !ids_dev || !vals_dev)) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    TENSAIR_CUDA(ctx, launch_top_drifted(ctx->L, diff_dev, nrows, m, ctx->at<TopkState>(ctx->cv.topk), ids_dev, vals_dev));
+    if (n_out) *n_out = m;
     return TENSAIR_OK;
 }
 

@@ -404,6 +404,47 @@ def test_cosine_difference_of_a_snapshot_matches_the_oracle(torch):
 
 
 # ------------------------------------------------------------------ launch variants give the same bits
+@pytest.mark.parametrize("n,k", [(1, 1), (5, 9), (255, 4), (257, 257), (70_001, 1), (70_001, 1000), (70_001, 4096),
+                                 (1_000_000, 100)])
+def test_most_drifted_rows_are_bit_exact(torch, n, k):
+    import oracle
+
+    rng = np.random.default_rng(n + k)
+    wl = synth.scaled(synth.TINY, V=50, d=8)
+    _, g = make_pair(wl)
+    cases = [rng.standard_normal(n).astype(np.float32),                       # distinct values
+             (rng.integers(0, 5, n) * 0.5).astype(np.float32),                # few values, long runs of ties
+             np.zeros(n, np.float32)]                                         # all equal: the first k rows
+    special = rng.standard_normal(n).astype(np.float32)
+    special[rng.integers(0, n, 6)] = [np.inf, -np.inf, np.nan, -0.0, 0.0, 2.0]
+    cases.append(special)
+    for x in cases:
+        want_ids, want_vals = oracle.top_drifted(x, k)
+        ids, vals = g.tensair_top_drifted(torch.from_numpy(x).cuda(), k)
+        assert ids.shape[0] == min(n, k)
+        assert np.array_equal(ids.cpu().numpy().view(np.uint32), want_ids)
+        assert np.array_equal(vals.cpu().numpy().view(np.uint32), want_vals.view(np.uint32))
+
+
+def test_most_drifted_rows_of_a_trained_table(torch):
+    import oracle
+
+    wl = synth.scaled(synth.LARGE_DRIFT, V=4000, d=32, batch=256, W=1, k=5, max_delay=0, stream_seeds=(3,))
+    stream = synth.token_stream(wl, 0, 8)
+    o, g = make_pair(wl, counts=synth.stream_counts([stream], wl.V))
+    snap = g.tensair_snapshot_rows(0, 0)
+    for b in range(8):
+        g.tensair_train_batch(0, dev(torch, stream[b]), b)
+    diff = g.tensair_cosine_difference(0, 0, snap)
+    ids, vals = g.tensair_top_drifted(diff, 25)
+    want_ids, want_vals = oracle.top_drifted(diff.cpu().numpy(), 25)
+    assert np.array_equal(ids.cpu().numpy().view(np.uint32), want_ids)
+    assert np.array_equal(vals.cpu().numpy(), want_vals)
+    assert vals[0] > 0 and set(want_ids.tolist()) <= set(np.unique(stream).tolist())   # only trained rows move
+    with pytest.raises(Exception):
+        g.tensair_top_drifted(diff, 4097)
+
+
 def test_fused_and_one_by_one_application_are_bit_identical(torch):
     from paper_2211_10280_b200 import binding as B
 
