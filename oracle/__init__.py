@@ -48,6 +48,8 @@ def lib():
             "orc_get_sampler": (None, [vp, vp, vp, vp]),
             "orc_batch_loss": (f64, [vp, u32, vp, u32, u64]),
             "orc_train_batch": (C.c_int, [vp, u32, vp, u32, u64, P(f64), P(u32)]),
+            "orc_train_batch_routed": (C.c_int, [vp, u32, vp, u32, u64, P(f64), P(u32)]),
+            "orc_route": (u32, [u64, u32, u32]),
             "orc_apply_messages": (C.c_int, [vp, u32, u64]),
             "orc_drain": (C.c_int, [vp]),
             "orc_read_embeddings": (None, [vp, u32, C.c_int, u32, u32, vp]),
@@ -117,6 +119,10 @@ def cosine_difference(a, b):
     return out
 
 
+def route(seed, W, token) -> int:
+    return int(lib().orc_route(seed, W, token))
+
+
 def top_drifted(diff, k):
     """(ids, values) of the k largest entries of a float32 array, largest first, smaller index first among equals."""
     diff = np.ascontiguousarray(diff, dtype=np.float32)
@@ -169,6 +175,15 @@ class Oracle:
         nrows = C.c_uint32(0)
         rc = lib().orc_train_batch(self._h, replica, _ptr(tokens), tokens.size, batch_index,
                                    C.byref(loss), C.byref(nrows))
+        return rc, loss.value, nrows.value
+
+    def train_batch_routed(self, replica, tokens, batch_index):
+        """The replica's share of the batch (centre words routed to it).  Returns (status, loss, n_rows)."""
+        tokens = np.ascontiguousarray(tokens, dtype=np.int32)
+        loss = C.c_double(0.0)
+        nrows = C.c_uint32(0)
+        rc = lib().orc_train_batch_routed(self._h, replica, _ptr(tokens), tokens.size, batch_index,
+                                          C.byref(loss), C.byref(nrows))
         return rc, loss.value, nrows.value
 
     def batch_loss(self, replica, tokens, batch_index):

@@ -21,6 +21,13 @@
 // gradient messages over the union of their rows (fp32 additions in the order computed).  The
 // staleness snapshot G_i of such a message is taken when it is sent.
 //
+// Routed mini-batches (Section 4.3: the (x, y) pairs are spread over the Model instances by a hash
+// partitioner keyed by the word x): every replica is handed the same token batch and trains the pairs
+// whose centre word is routed to it, route(x) = mulhi32(Philox(x, 0, 0, tag 4; seed).word0, W).  The
+// replicas then compute disjoint parts of ONE mini-batch gradient: pair indices, negative draws
+// (replica tag 0) and the mean's denominator are those of the whole batch, so the routed messages of
+// the W replicas add up to the message a single model computes from that batch.
+//
 // Arithmetic: tables are stored in fp32; every dot product, sigmoid, loss term and gradient sum is
 // taken in fp64 from those fp32 values; a delta row is fp32(-scale * sum) with scale = (double)lr when
 // the batch loss is the sum of the pair losses and (double)lr / (number of pairs) when it is their
@@ -72,7 +79,7 @@ U4 philox4x32_10(U4 ctr, uint32_t k0, uint32_t k1) {
     return ctr;
 }
 
-enum : uint32_t { TAG_NEGATIVE = 1, TAG_DELAY = 2, TAG_INIT = 3 };
+enum : uint32_t { TAG_NEGATIVE = 1, TAG_DELAY = 2, TAG_INIT = 3, TAG_ROUTE = 4 };
 
 inline uint32_t mulhi32(uint32_t a, uint32_t b) { return (uint32_t)(((uint64_t)a * b) >> 32); }
 
@@ -280,28 +287,39 @@ double orc_batch_loss(Oracle* o, uint32_t replica, const int32_t* tokens, uint32
     return loss;
 }
 
+// The Model instance that trains the pairs whose centre word is `token` (Section 4.3: hash partitioner keyed by x).
+uint32_t orc_route(uint64_t seed, uint32_t W, uint32_t token) {
+    U4 c{{token, 0u, 0u, TAG_ROUTE << 24}};
+    U4 r = philox4x32_10(c, (uint32_t)seed, (uint32_t)(seed >> 32));
+    return mulhi32(r.v[0], W);
+}
+
 // Algorithm 1, train(), mini-batch branch.  Returns 0, or -1 when a token id is out of range (then
-// nothing has changed).  n_rows_out (nullable) receives the message's row count.
-int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t n, uint64_t batch_index,
-                    double* loss_out, uint32_t* n_rows_out) {
+// nothing has changed).  n_rows_out (nullable) receives the message's row count.  routed: the replica
+// trains only the pairs of the batch whose centre word is routed to it (taps of the other pairs: draws
+// 0xFFFFFFFF, scalars 0).
+static int train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t n, uint64_t batch_index,
+                       double* loss_out, uint32_t* n_rows_out, bool routed) {
     const uint32_t V = o->V, d = o->d, k = o->k, w = o->window;
     if (replica >= o->W) return -2;
     for (uint32_t q = 0; q < n; ++q) if (tokens[q] < 0 || (uint32_t)tokens[q] >= V) return -1;
-    for (uint32_t q = 0; q < n; ++q) o->counts[tokens[q]] += 1;
+    auto mine = [&](uint32_t token) { return !routed || orc_route(o->seed, o->W, token) == replica; };
+    for (uint32_t q = 0; q < n; ++q) if (mine((uint32_t)tokens[q])) o->counts[tokens[q]] += 1;
 
     // pairs in (centre position ascending, context offset ascending) order
-    struct Pair { uint32_t centre, ctx; };
+    struct Pair { uint32_t centre, ctx; bool own; };
     std::vector<Pair> pairs;
     for (uint32_t q = 0; q < n; ++q)
         for (int64_t c = (int64_t)q - w; c <= (int64_t)q + w; ++c)
-            if (c >= 0 && c < (int64_t)n && c != (int64_t)q) pairs.push_back(Pair{(uint32_t)tokens[q], (uint32_t)tokens[c]});
+            if (c >= 0 && c < (int64_t)n && c != (int64_t)q)
+                pairs.push_back(Pair{(uint32_t)tokens[q], (uint32_t)tokens[c], mine((uint32_t)tokens[q])});
     const size_t P = pairs.size();
 
     // negatives
-    o->last_neg.assign(P * k, 0);
+    o->last_neg.assign(P * k, 0xFFFFFFFFu);
     for (size_t p = 0; p < P; ++p)
-        for (uint32_t j = 0; j < k; ++j)
-            o->last_neg[p * k + j] = orc_negative(o->seed, replica, batch_index, (uint32_t)p, j,
+        for (uint32_t j = 0; j < k && pairs[p].own; ++j)
+            o->last_neg[p * k + j] = orc_negative(o->seed, routed ? 0u : replica, batch_index, (uint32_t)p, j,
                                                   o->thresh.data(), o->alias.data(), V);
 
     // scalars at the snapshot
@@ -314,7 +332,7 @@ int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t
 #pragma omp parallel for schedule(static)
     for (int64_t p = 0; p < (int64_t)P; ++p) {
         const float* v = tin + (size_t)pairs[p].centre * d;
-        for (uint32_t j = 0; j < K1; ++j) {
+        for (uint32_t j = 0; j < K1 && pairs[p].own; ++j) {
             uint32_t row = j == 0 ? pairs[p].ctx : o->last_neg[p * k + (j - 1)];
             if (j > 0 && row == pairs[p].ctx) continue;   // a negative equal to the positive is dropped
             const float* u = tout + (size_t)row * d;
@@ -407,6 +425,15 @@ int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t
     auto it = o->msgs.find(prev);
     if (prev != key && it != o->msgs.end() && it->second.pending == 0) o->msgs.erase(it);
     return 0;
+}
+
+int orc_train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t n, uint64_t batch_index,
+                    double* loss_out, uint32_t* n_rows_out) {
+    return train_batch(o, replica, tokens, n, batch_index, loss_out, n_rows_out, false);
+}
+int orc_train_batch_routed(Oracle* o, uint32_t replica, const int32_t* tokens, uint32_t n, uint64_t batch_index,
+                           double* loss_out, uint32_t* n_rows_out) {
+    return train_batch(o, replica, tokens, n, batch_index, loss_out, n_rows_out, true);
 }
 
 void orc_set_max_grad_buffer(Oracle* o, uint32_t m) { o->max_grad_buffer = m < 1 ? 1 : m; }

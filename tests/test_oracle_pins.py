@@ -591,6 +591,81 @@ def test_top_drifted_rows_against_a_library_sort_brute_force_and_special_values(
     assert oracle.top_drifted(s, 9)[0].tolist() == [5, 2, 4, 0, 7, 1, 6, 3, 8]
 
 
+# ------------------------------------------------------------------ routed mini-batches (hash partition by centre word)
+def test_route_is_a_partition_of_the_vocabulary_and_roughly_even():
+    for W in (1, 2, 3, 8):
+        r = np.array([oracle.route(77, W, x) for x in range(6000)])
+        assert r.min() == 0 and r.max() == W - 1
+        share = np.bincount(r, minlength=W) / r.size
+        assert np.all(np.abs(share - 1.0 / W) < 0.03)
+    assert [oracle.route(77, 5, x) for x in range(50)] == [oracle.route(77, 5, x) for x in range(50)]
+    assert [oracle.route(77, 5, x) for x in range(50)] != [oracle.route(78, 5, x) for x in range(50)]
+
+
+@pytest.mark.parametrize("reduction", [0, 1])
+def test_routed_parts_of_a_minibatch_add_up_to_the_gradient_of_the_whole_batch(reduction):
+    # Section 4.3: pairs are spread over the Model instances by the hash of x.  The parts are disjoint
+    # sets of pairs of one batch, so they must add up to what a single model computes from that batch.
+    V, d, W, w, k = 200, 6, 3, 3, 4
+    wl = synth.scaled(synth.TINY, V=V, d=d, window=w, k=k, batch=64, batches=2)
+    stream = synth.token_stream(wl, 0)
+    counts = synth.stream_counts([stream], V)
+    t_in, t_out = synth.random_tables(V, d, 8, scale=0.4)
+    kw = dict(V=V, d=d, window=w, k=k, batch=64, lr=0.05, seed=21, counts=counts, init_in=t_in, init_out=t_out,
+              reduction=reduction)
+    solo, many = Oracle(W=1, **kw), Oracle(W=W, max_delay=0, **kw)
+    for b in range(2):
+        toks = stream[b]
+        rc, loss_solo, _ = solo.train_batch(0, toks, b)
+        assert rc == 0
+        neg_solo, g_solo = solo.read_negatives(), solo.read_g()
+        ids_solo, delta_solo = solo.read_message(0, b)
+        before = [many.read_embeddings(r, 0).copy() for r in range(W)]
+        losses, owners, g_sum = [], np.zeros(neg_solo.shape[0], int), np.zeros_like(g_solo)
+        summed = np.zeros((2 * V, d))
+        seen_in = set()
+        for r in range(W):
+            rc, loss_r, _ = many.train_batch_routed(r, toks, b)
+            assert rc == 0
+            losses.append(loss_r)
+            neg_r, g_r = many.read_negatives(), many.read_g()
+            own = neg_r[:, 0] != 0xFFFFFFFF
+            assert np.array_equal(neg_r[own], neg_solo[own])                     # the whole batch's draws
+            assert np.all(g_r[~own] == 0.0)
+            if b == 0:
+                assert np.array_equal(g_r[own], g_solo[own])
+            owners += own
+            g_sum += g_r
+            ids_r, delta_r = many.read_message(r, b)
+            ins = ids_r[ids_r < V]
+            assert all(oracle.route(21, W, int(x)) == r for x in ins)           # only its own centre words
+            assert not (set(ins.tolist()) & seen_in)
+            seen_in |= set(ins.tolist())
+            summed[ids_r] += delta_r
+            # rows outside its message are untouched by its own step
+            after = many.read_embeddings(r, 0)
+            mask = np.ones(V, bool)
+            mask[ins] = False
+            assert np.array_equal(after[mask], before[r][mask])
+        assert np.all(owners == 1)                                               # every pair trained exactly once
+        # batch 0 starts from identical tables; later the replicas differ from the single model by fp32 rounding order
+        assert sum(losses) == pytest.approx(loss_solo, rel=1e-12 if b == 0 else 1e-6)
+        if b == 0:
+            np.testing.assert_array_equal(g_sum, g_solo)
+            touched = np.flatnonzero(np.abs(summed).sum(axis=1) > 0)
+            assert set(touched.tolist()) <= set(ids_solo.tolist())
+            np.testing.assert_allclose(summed[ids_solo], delta_solo, rtol=0, atol=3e-7 * np.abs(delta_solo).max())
+        for r in range(W):
+            assert many.apply_messages(r, b) == W - 1
+        if b == 0:
+            for r in range(W):
+                for which in (0, 1):
+                    np.testing.assert_allclose(many.read_embeddings(r, which), solo.read_embeddings(0, which),
+                                               rtol=0, atol=2e-7)
+    # the running unigram counts saw every token once
+    assert np.array_equal(many.sampler()[2], solo.sampler()[2])
+
+
 # ------------------------------------------------------------------ maxGradBuffer > 1
 def test_buffered_gradients_are_summed_over_the_union_of_their_rows_and_sent_every_mth_batch():
     # Algorithm 1: gradients += gradient; count += 1; send when count >= maxGradBuffer.
