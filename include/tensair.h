@@ -172,6 +172,24 @@ TENSAIR_API int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, con
                              uint64_t batch_index, double* loss_out, tensair_msg_info* info);
 
 /*
+ * The same step for a mini-batch that the W replicas share (Section 4.3: the (x, y) pairs are spread over the
+ * Model instances by a hash partitioner keyed by the word x).  Every replica is handed the same tokens_dev and
+ * trains the pairs whose centre word is routed to it:
+ *     route(x) = (Philox4x32-10(counter = (x, 0, 0, 4 << 24), key = seed).word0 * W) >> 32     (tensair_route).
+ * The W calls compute disjoint parts of one mini-batch gradient: the pair index p, the negative draws (replica
+ * tag 0 in their counter) and, for TENSAIR_MEAN, the divisor are those of the whole batch, so the W messages add
+ * up to the message one model computes from the batch; their input rows are disjoint.  The running unigram
+ * counts take each token once, from the replica that owns it.  info->n_pairs is the pair count of the whole
+ * batch.  Arguments, asynchrony and errors as for tensair_train_batch; the taps tensair_read_negatives and
+ * tensair_read_scalars are defined only for the pairs the replica owns.
+ */
+TENSAIR_API int tensair_train_batch_routed(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_dev,
+                                           uint32_t n_tokens, uint64_t batch_index, double* loss_out,
+                                           tensair_msg_info* info);
+/* The replica that owns centre word `token` under the routing above (host only). */
+TENSAIR_API int tensair_route(uint64_t seed, uint32_t W, uint32_t token, uint32_t* replica);
+
+/*
  * The same step for callers that may not allocate device memory when they train - a plug-in that is
  * handed its tables and message pool by a host application with a fixed memory plan, or a service
  * thread that must stay out of the allocator.  (The paper has no counterpart: this is an addition of

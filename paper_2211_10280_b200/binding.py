@@ -66,6 +66,8 @@ SYMBOLS = {
     "tensair_destroy": (None, [_vp]),
     "tensair_train_batch": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
     "tensair_train_batch_host": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
+    "tensair_train_batch_routed": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
+    "tensair_route": (_int, [_u64, _u32, _u32, _vp]),
     "tensair_train_batch_static": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
     "tensair_apply_messages": (_int, [_vp, _u32, _u64, _P(_u32)]),
     "tensair_drain": (_int, [_vp, _P(_u32)]),
@@ -159,6 +161,14 @@ def tensair_tune(name: str, value: int):
 
 def tensair_delay(seed: int, max_delay: int, step: int, sender: int, receiver: int) -> int:
     return int(lib().tensair_delay(seed, max_delay, step, sender, receiver))
+
+
+def tensair_route(seed: int, W: int, token: int) -> int:
+    out = C.c_uint32(0)
+    rc = lib().tensair_route(seed, W, token, C.byref(out))
+    if rc != OK:
+        raise TensairError(rc, "tensair_route")
+    return int(out.value)
 
 
 class Schedule:
@@ -257,6 +267,12 @@ class Context:
         assert tokens_dev.is_cuda and tokens_dev.dtype == self.torch.int32 and tokens_dev.is_contiguous()
         return self._train(lib().tensair_train_batch, "tensair_train_batch", replica, tokens_dev.data_ptr(),
                            tokens_dev.numel(), batch_index, want_loss, want_info)
+
+    def tensair_train_batch_routed(self, replica, tokens_dev, batch_index, want_loss=False, want_info=False):
+        """The replica's share of a batch all replicas are handed: the pairs whose centre word is routed to it."""
+        assert tokens_dev.is_cuda and tokens_dev.dtype == self.torch.int32 and tokens_dev.is_contiguous()
+        return self._train(lib().tensair_train_batch_routed, "tensair_train_batch_routed", replica,
+                           tokens_dev.data_ptr(), tokens_dev.numel(), batch_index, want_loss, want_info)
 
     def tensair_train_batch_static(self, replica, tokens_dev, batch_index, want_loss=False, want_info=False):
         """tensair_train_batch with the per-batch working memory taken from the library's built-in array."""

@@ -59,7 +59,8 @@ template <int NV, int CR>
 __global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, uint32_t stride4, uint32_t w,
           uint32_t k, uint32_t chunk_rows, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
-          Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err) {
+          Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err,
+          const uint8_t* __restrict__ owner) {
     if (*err) return;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -75,6 +76,10 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
     const uint32_t warp = blockIdx.x * kFwdWarps + wib, nwarps = gridDim.x * kFwdWarps;
 
     for (uint32_t q = warp; q < n && !failed; q += nwarps) {
+        if (owner && !owner[q]) {   // routed batch: another replica trains this centre word
+            if (lane == 0) loss_pos[q] = 0.0;
+            continue;
+        }
         const uint32_t centre = (uint32_t)tok[q];
         const float4* __restrict__ vin = table + (size_t)centre * stride4;
         double v[NV][4], acc[NV][4];
@@ -205,7 +210,8 @@ void set_forward_shape(int rows, int blocks_per_sm) {
 }
 
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
-                           const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err) {
+                           const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err,
+                           const uint8_t* owner) {
     if (n < 2) return cudaSuccess;
     const size_t row = (size_t)s.stride * 4;
     const int cr = g_forward_rows == 4 || g_forward_rows == 8 || g_forward_rows == 16 ? g_forward_rows : 8;
@@ -232,7 +238,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
         }                                                                                                       \
         k_forward<NV, CR><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,     \
                                                                       chunk_rows, t4, rows, rec, gin_pos,      \
-                                                                      loss_pos, err);                           \
+                                                                      loss_pos, err, owner);                    \
     } while (0)
 #define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)
     if (s.d4 <= 32) TENSAIR_FWD_NV(1);

@@ -18,6 +18,7 @@ constexpr uint32_t kWeyl1 = 0xBB67AE85u;
 constexpr uint32_t kTagNegative = 1u << 24;
 constexpr uint32_t kTagDelay = 2u << 24;
 constexpr uint32_t kTagInit = 3u << 24;
+constexpr uint32_t kTagRoute = 4u << 24;
 
 struct Philox4 {
     uint32_t x, y, z, w;

@@ -47,18 +47,26 @@ void build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint
     }
 }
 
-__global__ void k_validate(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t* err) {
+// Checks the token ids; for a routed batch (owner != nullptr) also marks the centre positions whose word the
+// hash partitioner gives to this replica: route(x) = mulhi32(Philox(x, 0, 0, route tag; seed).word0, W).
+__global__ void k_validate(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t* err, uint8_t* owner,
+                           uint32_t W, uint32_t replica, uint32_t key0, uint32_t key1) {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) {
         const int32_t t = tok[i];
         if (t < 0 || (uint32_t)t >= V) atomicOr(err, 1u);
+        if (owner) {
+            const Philox4 r = philox4x32_10(Philox4{(uint32_t)t, 0u, 0u, kTagRoute}, key0, key1);
+            owner[i] = __umulhi(r.x, W) == replica ? 1 : 0;
+        }
     }
 }
 
-cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, uint32_t V, uint32_t* err) {
+cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, uint32_t V, uint32_t* err, uint8_t* owner,
+                            uint32_t W, uint32_t replica, uint64_t seed) {
     if (n == 0) return cudaSuccess;
     Timed timed(L, K_VALIDATE);
-    k_validate<<<(n + 255) / 256, 256, 0, L.stream>>>(tok, n, V, err);
+    k_validate<<<(n + 255) / 256, 256, 0, L.stream>>>(tok, n, V, err, owner, W, replica, (uint32_t)seed, (uint32_t)(seed >> 32));
     return cudaGetLastError();
 }
 
@@ -71,12 +79,13 @@ __device__ inline uint32_t alias_pick(const uint2* __restrict__ tab, uint32_t V,
 // One thread per (centre position q, window slot s, draw pair jp).  Window slot s in [0, 2w) stands
 // for context position q + (s < w ? s - w : s - w + 1); slots outside the batch do nothing.
 // Thread jp = 0 also emits the positive contribution; thread (s = 0, jp = 0) emits the position's
-// input-row item and counts the token.
+// input-row item and counts the token.  In a routed batch (owner != nullptr) the positions of other
+// replicas' centre words emit only items that sort past every row and are never read.
 __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t w, uint32_t k,
                           uint32_t replica, uint32_t batch_lo, uint32_t key0, uint32_t key1,
                           const uint2* __restrict__ alias_tab, uint32_t* __restrict__ rows,
                           item_t* __restrict__ items, unsigned long long* __restrict__ counts,
-                          const uint32_t* __restrict__ err) {
+                          const uint32_t* __restrict__ err, const uint8_t* __restrict__ owner) {
     if (*err) return;
     const uint32_t JP = (k + 1) / 2;
     const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -87,9 +96,10 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
     const uint32_t s = ps % (2 * w);
     const uint32_t q = ps / (2 * w);
     const uint32_t centre = (uint32_t)tok[q];
+    const bool own = !owner || owner[q];
     if (s == 0 && jp == 0) {
-        atomicAdd(counts + centre, 1ULL);
-        if (n >= 2) items[q] = make_item(centre, q);
+        if (own) atomicAdd(counts + centre, 1ULL);
+        if (n >= 2) items[q] = make_item(own ? centre : 2 * V, q);
     }
     const int64_t c = (int64_t)q + (s < w ? (int64_t)s - (int64_t)w : (int64_t)s - (int64_t)w + 1);
     if (c < 0 || c >= (int64_t)n) return;
@@ -98,6 +108,13 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
     const uint32_t K1 = k + 1;
     const uint32_t ctx = (uint32_t)tok[c];
     const uint32_t cbase = p * K1;
+    if (!own) {
+        if (jp == 0) items[n + cbase] = make_item(2 * V, cbase);
+        const uint32_t j0 = 2 * jp;
+        items[n + cbase + 1 + j0] = make_item(2 * V, cbase + 1 + j0);
+        if (j0 + 1 < k) items[n + cbase + 2 + j0] = make_item(2 * V, cbase + 2 + j0);
+        return;
+    }
     if (jp == 0) {
         rows[cbase] = ctx;
         items[n + cbase] = make_item(V + ctx, cbase);
@@ -116,13 +133,13 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
 
 cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, uint32_t replica,
                            uint32_t batch_lo, uint64_t seed, const uint2* alias_tab, uint32_t* rows,
-                           item_t* items, unsigned long long* counts, const uint32_t* err) {
+                           item_t* items, unsigned long long* counts, const uint32_t* err, const uint8_t* owner) {
     if (n == 0) return cudaSuccess;
     const uint64_t total = (uint64_t)n * 2 * s.w * ((s.k + 1) / 2);
     const uint32_t blocks = (uint32_t)((total + 255) / 256);
     Timed timed(L, K_PREPARE);
     k_prepare<<<blocks, 256, 0, L.stream>>>(tok, n, s.V, s.w, s.k, replica, batch_lo, (uint32_t)seed,
-                                            (uint32_t)(seed >> 32), alias_tab, rows, items, counts, err);
+                                            (uint32_t)(seed >> 32), alias_tab, rows, items, counts, err, owner);
     return cudaGetLastError();
 }
 

@@ -112,6 +112,13 @@ uint32_t tensair_delay(uint64_t seed, uint32_t max_delay, uint64_t step, uint32_
     return Schedule(1, max_delay, seed).delay(step, sender, receiver);
 }
 
+int tensair_route(uint64_t seed, uint32_t W, uint32_t token, uint32_t* replica) {
+    if (!replica || W == 0) return TENSAIR_EINVAL;
+    const tensair::Philox4 r = tensair::philox4x32_10(tensair::Philox4{token, 0u, 0u, tensair::kTagRoute}, (uint32_t)seed, (uint32_t)(seed >> 32));
+    *replica = (uint32_t)(((uint64_t)r.x * W) >> 32);
+    return TENSAIR_OK;
+}
+
 void tensair_philox4x32_10(const uint32_t counter[4], const uint32_t key[2], uint32_t out[4]) {
     const tensair::Philox4 r =
         tensair::philox4x32_10(tensair::Philox4{counter[0], counter[1], counter[2], counter[3]}, key[0], key[1]);

@@ -63,6 +63,7 @@ void carve(const tensair_config& c, Carve& k) {
     k.partials = take((uint64_t)k.max_chunks * k.stride * 8);
     k.merge_counts = take((uint64_t)(bucket_count(c.V) + 1) * 4);
     k.topk = take(sizeof(TopkState));
+    k.owner = take(c.batch);
     k.total = off;
     k.bucket_off = kHeaderBytes;
     k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
@@ -106,8 +107,10 @@ int upload_sampler(tensair_ctx* ctx, const uint64_t* counts_host) {
     return TENSAIR_OK;
 }
 
+// routed: the replica trains only the centre positions whose word the hash partitioner gives it (Section 4.3);
+// pair indices, negative draws (replica tag 0) and the mean's denominator stay those of the whole batch.
 int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint32_t n, uint64_t batch_index,
-               double* loss_out, tensair_msg_info* info) {
+               double* loss_out, tensair_msg_info* info, bool routed = false) {
     const tensair_config& c = ctx->cfg;
     const Carve& cv = ctx->cv;
     // maxGradBuffer = 1: the batch's message is built in its send slot and filed at once.  Otherwise it is built
@@ -131,10 +134,11 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
     // Eq. 1's alpha, divided by the number of pairs when the batch loss is the mean of the pair losses
     const double scale = c.reduction == TENSAIR_MEAN && pairs ? (double)c.lr / (double)pairs : (double)c.lr;
 
-    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err));
-    TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tok_dev, n, ctx->shape, replica, (uint32_t)batch_index, c.seed,
+    uint8_t* owner = routed ? ctx->at<uint8_t>(cv.owner) : nullptr;
+    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err, owner, c.W, replica, c.seed));
+    TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tok_dev, n, ctx->shape, routed ? 0u : replica, (uint32_t)batch_index, c.seed,
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows),
-                                     ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err));
+                                     ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err, owner));
     if (n_items) {
         // The sort needs only the items written by the prepare kernel and the forward kernel does not
         // touch them: the two run side by side (the sort is latency-bound and leaves the machine idle).
@@ -147,7 +151,8 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
         TENSAIR_CUDA(ctx, launch_sort(fork ? ctx->L_side : ctx->L, ctx->at<item_t>(cv.items_a), ctx->at<item_t>(cv.items_b),
                                       n_items, bits_for(2 * c.V), ctx->at<uint32_t>(cv.hist), &sorted));
         TENSAIR_CUDA(ctx, launch_forward(ctx->L, tok_dev, n, ctx->shape, table, ctx->at<uint32_t>(cv.rows),
-                                         ctx->at<Rec>(cv.rec), ctx->at<double>(cv.gin_pos), ctx->at<double>(cv.loss_pos), err));
+                                         ctx->at<Rec>(cv.rec), ctx->at<double>(cv.gin_pos), ctx->at<double>(cv.loss_pos), err,
+                                         owner));
         if (fork) {
             TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
             TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0));
@@ -367,6 +372,16 @@ int tensair_train_batch(tensair_ctx* ctx, uint32_t replica, const int32_t* token
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return TENSAIR_ECUDA;
     return train_impl(ctx, replica, tokens_dev, n_tokens, batch_index, loss_out, info);
+}
+
+int tensair_train_batch_routed(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_dev, uint32_t n_tokens,
+                               uint64_t batch_index, double* loss_out, tensair_msg_info* info) {
+    if (!ctx || replica >= ctx->cfg.W || n_tokens > ctx->cfg.batch || (n_tokens && !tokens_dev) ||
+        batch_index >= (1ull << 32))
+        return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    return train_impl(ctx, replica, tokens_dev, n_tokens, batch_index, loss_out, info, true);
 }
 
 int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_host, uint32_t n_tokens,

@@ -349,6 +349,101 @@ def test_drift_rebuilds_the_sampler_from_running_counts(torch):
         compare_tables(o, g, j, TOL_200)
 
 
+# ------------------------------------------------------------------ routed mini-batches (hash partition by centre word)
+def _routed_step(torch, o, g, wl, toks, b, tol):
+    """One shared batch through every replica of both sides, compared piece by piece; returns the GPU losses."""
+    from paper_2211_10280_b200 import binding as B
+
+    t_dev = dev(torch, toks)
+    losses = []
+    for r in range(wl.W):
+        rc, loss_o, nrows_o = o.train_batch_routed(r, toks, b)
+        assert rc == 0
+        loss_g, info = g.tensair_train_batch_routed(r, t_dev, b, want_loss=True, want_info=True)
+        assert info.n_rows == nrows_o and info.n_pairs == synth.n_pairs(len(toks), wl.window)
+        assert loss_g == pytest.approx(loss_o, rel=1e-9, abs=1e-12)
+        losses.append(loss_g)
+        no, go = o.read_negatives(), o.read_g()
+        own = no[:, 0] != 0xFFFFFFFF if no.size else np.zeros(0, bool)
+        centre_owner = np.array([B.tensair_route(wl.seed, wl.W, int(x)) for x in toks])
+        assert info.n_in_rows == len(set(toks[centre_owner == r].tolist()))
+        if own.any():
+            assert np.array_equal(g.tensair_read_negatives()[own], no[own])
+            gg = g.tensair_read_scalars()[own]
+            assert np.array_equal(go[own] == 0.0, gg == 0.0) and np.max(np.abs(go[own] - gg)) <= 1e-9
+        if nrows_o:
+            compare_message(o, g, r, b, tol)
+        else:
+            assert g.tensair_read_message(r, b)[0].size == 0
+    for r in range(wl.W):
+        assert o.apply_messages(r, b) == g.tensair_apply_messages(r, b)
+    return losses
+
+
+@pytest.mark.parametrize("W,reduction", [(1, 1), (2, 0), (4, 1), (8, 1)])
+def test_routed_minibatch_matches_the_oracle(torch, W, reduction):
+    wl = synth.scaled(synth.LARGE_DASGD, V=3000, d=36, batch=700, k=6, W=W, max_delay=1, reduction=reduction,
+                      lr=0.025 if reduction else 0.002, stream_seeds=tuple(range(W)))
+    stream = synth.token_stream(wl, 0, 3)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 5, scale=0.3)
+    o, g = make_pair(wl, counts=synth.stream_counts([stream], wl.V), init_in=t_in, init_out=t_out)
+    for b in range(3):
+        _routed_step(torch, o, g, wl, stream[b], b, TOL_ONE if b == 0 else TOL_200)
+    assert o.drain() == g.tensair_drain()
+    for r in range(W):
+        assert np.array_equal(o.delivery_log(r), g.tensair_read_delivery_log(r))
+        compare_tables(o, g, r, TOL_200)
+    assert np.array_equal(o.sampler()[2], g.tensair_read_sampler()[2])
+
+
+def test_routed_parts_add_up_to_the_single_model_step(torch):
+    # the property that holds at any size: W routed parts of a batch == one model's step on the batch
+    wl = synth.scaled(synth.LARGE_DASGD, V=40_000, d=64, batch=4096, k=8, W=4, max_delay=0)
+    stream = synth.token_stream(wl, 0, 1)
+    counts = synth.stream_counts([stream], wl.V)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 6, scale=0.2)
+    _, many = make_pair(wl, counts=counts, init_in=t_in, init_out=t_out)
+    _, solo = make_pair(synth.scaled(wl, W=1), counts=counts, init_in=t_in, init_out=t_out)
+    t_dev = dev(torch, stream[0])
+    loss_solo, _ = solo.tensair_train_batch(0, t_dev, 0, want_loss=True)
+    ids_solo, delta_solo = solo.tensair_read_message(0, 0)
+    summed = np.zeros((2 * wl.V, wl.d))
+    total, n_in = 0.0, 0
+    for r in range(wl.W):
+        loss_r, info = many.tensair_train_batch_routed(r, t_dev, 0, want_loss=True, want_info=True)
+        total += loss_r
+        n_in += info.n_in_rows
+        ids_r, delta_r = many.tensair_read_message(r, 0)
+        summed[ids_r] += delta_r
+    assert total == pytest.approx(loss_solo, rel=1e-12)
+    assert n_in == int((ids_solo < wl.V).sum())                   # input rows: a partition of the single model's
+    assert set(np.flatnonzero(np.abs(summed).sum(axis=1) > 0).tolist()) <= set(ids_solo.tolist())
+    # each part is rounded to fp32 on its own and parts of opposite sign cancel: a few fp32 roundings of the
+    # largest part, measured against a sum that can be much smaller
+    assert rel_err(summed[ids_solo], delta_solo) <= 1e-4
+    for r in range(wl.W):
+        assert many.tensair_apply_messages(r, 0) == wl.W - 1
+    for r in range(wl.W):
+        for which in (0, 1):
+            assert rel_err(many.tensair_read_embeddings(r, which), solo.tensair_read_embeddings(0, which)) <= 1e-6
+
+
+def test_routed_batch_of_one_word_belongs_to_one_replica(torch):
+    from paper_2211_10280_b200 import binding as B
+
+    wl = synth.scaled(synth.TINY, V=60, d=16, window=2, k=3, batch=80, W=3, max_delay=0, reduction=1,
+                      stream_seeds=(1, 2, 3))
+    toks = np.full(wl.batch, 11, np.int32)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 2, scale=0.3)
+    o, g = make_pair(wl, init_in=t_in, init_out=t_out)
+    _routed_step(torch, o, g, wl, toks, 0, TOL_ONE)
+    owner = B.tensair_route(wl.seed, wl.W, 11)
+    for r in range(wl.W):
+        ids, _ = g.tensair_read_message(r, 0)
+        assert (ids.size > 0) == (r == owner)
+        compare_tables(o, g, r, TOL_ONE)
+
+
 # ------------------------------------------------------------------ full size, the benchmark's configuration
 def test_full_size_large_dasgd_two_steps(torch):
     """V = 1M, d = 300, batch 8192, k = 15, W = 4, delay <= 2: the whole first two steps against the oracle."""

@@ -88,6 +88,15 @@ def test_delay_matches_the_oracle_and_is_uniform():
     assert all(B.tensair_delay(1, 0, t, 0, 1) == 0 for t in range(20))
 
 
+def test_route_matches_the_oracle():
+    for W in (1, 2, 3, 4, 8):
+        for seed in (0, 0xABCDEF0123):
+            assert [B.tensair_route(seed, W, x) for x in range(300)] == [oracle.route(seed, W, x) for x in range(300)]
+    out = C.c_uint32(0)
+    assert B.lib().tensair_route(1, 0, 5, C.byref(out)) == B.EINVAL
+    assert B.lib().tensair_route(1, 2, 5, None) == B.EINVAL
+
+
 def _oracle_logs(W, D, T, seed, skip=()):
     o = Oracle(V=16, d=4, window=1, k=1, batch=4, W=W, max_delay=D, seed=seed)
     toks = np.array([1, 2, 3, 4], np.int32)
