@@ -184,8 +184,12 @@ def run_ours(args):
     msg_ids = {}
 
     def step(t, host=False, info=False):
+        shared = toks_pin[t, 0].to("cuda", non_blocking=True) if (wl.routed and host) else None
         for i in range(wl.W):
-            if host:
+            if wl.routed:       # one batch for all replicas, split by the hash of the centre word
+                _, inf = ctx.tensair_train_batch_routed(i, shared if host else toks_dev[t, 0], t, want_loss=host,
+                                                        want_info=host or info)
+            elif host:
                 _, inf = ctx.tensair_train_batch_host(i, toks_pin[t, i], t, want_loss=True, want_info=True)
             else:
                 _, inf = ctx.tensair_train_batch(i, toks_dev[t, i], t, want_info=info)
@@ -251,7 +255,7 @@ def run_ours(args):
     if ctx.tensair_sync() != B.OK:
         raise SystemExit("the device reported a bad token during the benchmark")
 
-    pairs_per_step = wl.W * P
+    pairs_per_step = P if wl.routed else wl.W * P
     value = world * pairs_per_step * K / (ms_dev * 1e-3)
     e2e_value = world * pairs_per_step * K / (ms_e2e * 1e-3)
 
@@ -330,10 +334,11 @@ def run_ours(args):
         "dtype": "f64", "data": "synthetic",
         "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
                    "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
-                   "max_grad_buffer": wl.max_grad_buffer, "pairs_per_batch": P, "storage": "f32", "l2": "inputs larger than L2 (tables %.1f GB)" %
+                   "max_grad_buffer": wl.max_grad_buffer, "routing": "hash of the centre word, one batch shared by the replicas" if wl.routed else "one substream per replica",
+                   "pairs_per_batch": P, "storage": "f32", "l2": "inputs larger than L2 (tables %.1f GB)" %
                    (ctx.sizes.tables_bytes / 1e9), "parallelism": f"{world} independent replica groups"},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / K,
-                "h2d_bytes_per_step": wl.W * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4)},
+                "h2d_bytes_per_step": (1 if wl.routed else wl.W) * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4)},
         "gpu_launches": int(launches),
         "clocks": sampler.summary(wall0, wall1),
         "roofline": roofline,

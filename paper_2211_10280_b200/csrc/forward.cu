@@ -60,7 +60,7 @@ __global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, uint32_t stride4, uint32_t w,
           uint32_t k, uint32_t chunk_rows, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
           Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err,
-          const uint8_t* __restrict__ owner) {
+          const uint32_t* __restrict__ owned, const uint32_t* __restrict__ n_owned) {
     if (*err) return;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -75,11 +75,10 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
     const float4* __restrict__ tout = table + (size_t)V * stride4;
     const uint32_t warp = blockIdx.x * kFwdWarps + wib, nwarps = gridDim.x * kFwdWarps;
 
-    for (uint32_t q = warp; q < n && !failed; q += nwarps) {
-        if (owner && !owner[q]) {   // routed batch: another replica trains this centre word
-            if (lane == 0) loss_pos[q] = 0.0;
-            continue;
-        }
+    // routed batch: only the listed centre positions are this replica's
+    const uint32_t n_mine = owned ? *n_owned : n;
+    for (uint32_t at = warp; at < n_mine && !failed; at += nwarps) {
+        const uint32_t q = owned ? owned[at] : at;
         const uint32_t centre = (uint32_t)tok[q];
         const float4* __restrict__ vin = table + (size_t)centre * stride4;
         double v[NV][4], acc[NV][4];
@@ -211,7 +210,7 @@ void set_forward_shape(int rows, int blocks_per_sm) {
 
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err,
-                           const uint8_t* owner) {
+                           const uint32_t* owned, const uint32_t* n_owned) {
     if (n < 2) return cudaSuccess;
     const size_t row = (size_t)s.stride * 4;
     const int cr = g_forward_rows == 4 || g_forward_rows == 8 || g_forward_rows == 16 ? g_forward_rows : 8;
@@ -238,7 +237,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
         }                                                                                                       \
         k_forward<NV, CR><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,     \
                                                                       chunk_rows, t4, rows, rec, gin_pos,      \
-                                                                      loss_pos, err, owner);                    \
+                                                                      loss_pos, err, owned, n_owned);                  \
     } while (0)
 #define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)
     if (s.d4 <= 32) TENSAIR_FWD_NV(1);
@@ -251,13 +250,15 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     return cudaGetLastError();
 }
 
-// Sum of the per-position losses in a fixed order, in fp64.
+// Sum of the per-position losses (in a routed batch: of the replica's own positions) in a fixed order, in fp64.
 __global__ void __launch_bounds__(1024)
-k_loss_sum(const double* __restrict__ loss_pos, uint32_t n, double* __restrict__ loss, const uint32_t* __restrict__ err) {
+k_loss_sum(const double* __restrict__ loss_pos, uint32_t n, double* __restrict__ loss, const uint32_t* __restrict__ err,
+           const uint8_t* __restrict__ owner) {
     __shared__ double part[1024];
     double s = 0.0;
     if (!*err)
-        for (uint32_t i = threadIdx.x; i < n; i += 1024) s += loss_pos[i];
+        for (uint32_t i = threadIdx.x; i < n; i += 1024)
+            if (!owner || owner[i]) s += loss_pos[i];
     part[threadIdx.x] = s;
     __syncthreads();
     for (int o = 512; o > 0; o >>= 1) {
@@ -267,9 +268,10 @@ k_loss_sum(const double* __restrict__ loss_pos, uint32_t n, double* __restrict__
     if (threadIdx.x == 0) *loss = part[0];
 }
 
-cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err) {
+cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err,
+                            const uint8_t* owner) {
     Timed timed(L, K_LOSS_SUM);
-    k_loss_sum<<<1, 1024, 0, L.stream>>>(loss_pos, n < 2 ? 0 : n, loss, err);
+    k_loss_sum<<<1, 1024, 0, L.stream>>>(loss_pos, n < 2 ? 0 : n, loss, err, owner);
     return cudaGetLastError();
 }
 

@@ -70,7 +70,7 @@ struct Timed {
 
 // sampler.cu
 cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, uint32_t V, uint32_t* err, uint8_t* owner,
-                            uint32_t W, uint32_t replica, uint64_t seed);
+                            uint32_t* owned, uint32_t* n_owned, uint32_t W, uint32_t replica, uint64_t seed);
 cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, uint32_t replica,
                            uint32_t batch_lo, uint64_t seed, const uint2* alias_tab, uint32_t* rows,
                            item_t* items, unsigned long long* counts, const uint32_t* err, const uint8_t* owner);
@@ -88,9 +88,10 @@ uint32_t sort_hist_words(uint32_t n);
 // forward.cu
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err,
-                           const uint8_t* owner);
+                           const uint32_t* owned, const uint32_t* n_owned);
 void set_forward_shape(int rows, int blocks_per_sm);
-cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err);
+cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err,
+                            const uint8_t* owner);
 
 // message.cu
 uint32_t heads_tiles(uint32_t n_items);

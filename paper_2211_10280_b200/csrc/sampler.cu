@@ -48,25 +48,35 @@ void build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint
 }
 
 // Checks the token ids; for a routed batch (owner != nullptr) also marks the centre positions whose word the
-// hash partitioner gives to this replica: route(x) = mulhi32(Philox(x, 0, 0, route tag; seed).word0, W).
+// hash partitioner gives to this replica, route(x) = mulhi32(Philox(x, 0, 0, route tag; seed).word0, W), and
+// lists them (in no particular order: nothing downstream depends on it) so that the forward kernel can spread
+// them evenly over its warps.
 __global__ void k_validate(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t* err, uint8_t* owner,
-                           uint32_t W, uint32_t replica, uint32_t key0, uint32_t key1) {
+                           uint32_t* __restrict__ owned, uint32_t* __restrict__ n_owned, uint32_t W, uint32_t replica,
+                           uint32_t key0, uint32_t key1) {
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) {
         const int32_t t = tok[i];
         if (t < 0 || (uint32_t)t >= V) atomicOr(err, 1u);
         if (owner) {
             const Philox4 r = philox4x32_10(Philox4{(uint32_t)t, 0u, 0u, kTagRoute}, key0, key1);
-            owner[i] = __umulhi(r.x, W) == replica ? 1 : 0;
+            const bool mine = __umulhi(r.x, W) == replica;
+            owner[i] = mine ? 1 : 0;
+            if (mine) owned[atomicAdd(n_owned, 1u)] = i;
         }
     }
 }
 
 cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, uint32_t V, uint32_t* err, uint8_t* owner,
-                            uint32_t W, uint32_t replica, uint64_t seed) {
+                            uint32_t* owned, uint32_t* n_owned, uint32_t W, uint32_t replica, uint64_t seed) {
     if (n == 0) return cudaSuccess;
+    if (owner) {
+        const cudaError_t e = cudaMemsetAsync(n_owned, 0, 4, L.stream);
+        if (e != cudaSuccess) return e;
+    }
     Timed timed(L, K_VALIDATE);
-    k_validate<<<(n + 255) / 256, 256, 0, L.stream>>>(tok, n, V, err, owner, W, replica, (uint32_t)seed, (uint32_t)(seed >> 32));
+    k_validate<<<(n + 255) / 256, 256, 0, L.stream>>>(tok, n, V, err, owner, owned, n_owned, W, replica, (uint32_t)seed,
+                                                      (uint32_t)(seed >> 32));
     return cudaGetLastError();
 }
 

@@ -105,13 +105,13 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
 
     // the array keeps what the previous call left: the list counters must start at zero
     TENSAIR_CUDA(ctx, cudaMemsetAsync(long_counters, 0, 8, ctx->stream));
-    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tokens_dev, n_tokens, c.V, err, nullptr, c.W, replica, c.seed));
+    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tokens_dev, n_tokens, c.V, err, nullptr, nullptr, nullptr, c.W, replica, c.seed));
     TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tokens_dev, n_tokens, ctx->shape, replica, (uint32_t)batch_index, c.seed,
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows), items_a,
                                      ctx->at<unsigned long long>(cv.counts), err, nullptr));
     if (n_items) {
         TENSAIR_CUDA(ctx, launch_forward(ctx->L, tokens_dev, n_tokens, ctx->shape, table, ctx->at<uint32_t>(cv.rows),
-                                         ctx->at<Rec>(cv.rec), gin_pos, loss_pos, err, nullptr));
+                                         ctx->at<Rec>(cv.rec), gin_pos, loss_pos, err, nullptr, nullptr));
         item_t* sorted = nullptr;
         TENSAIR_CUDA(ctx, launch_sort(ctx->L, items_a, items_b, n_items, bits_for(2 * c.V),
                                       reinterpret_cast<uint32_t*>(in_ws(sc.hist)), &sorted));
@@ -129,7 +129,7 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
         TENSAIR_CUDA(ctx, cudaMemsetAsync(hdr, 0, sizeof(MsgHeader), ctx->stream));
     }
     TENSAIR_CUDA(ctx, launch_bucket_index(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
-    TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, loss_pos, n_tokens, ctx->at<double>(cv.loss), err));
+    TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, loss_pos, n_tokens, ctx->at<double>(cv.loss), err, nullptr));
     ctx->last_n = n_tokens;
     ctx->last_pairs = pairs;
     ctx->have_last = true;

@@ -64,6 +64,8 @@ void carve(const tensair_config& c, Carve& k) {
     k.merge_counts = take((uint64_t)(bucket_count(c.V) + 1) * 4);
     k.topk = take(sizeof(TopkState));
     k.owner = take(c.batch);
+    k.owned = take((uint64_t)c.batch * 4);
+    k.n_owned = take(4);
     k.total = off;
     k.bucket_off = kHeaderBytes;
     k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
@@ -135,7 +137,9 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
     const double scale = c.reduction == TENSAIR_MEAN && pairs ? (double)c.lr / (double)pairs : (double)c.lr;
 
     uint8_t* owner = routed ? ctx->at<uint8_t>(cv.owner) : nullptr;
-    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err, owner, c.W, replica, c.seed));
+    uint32_t* owned = routed ? ctx->at<uint32_t>(cv.owned) : nullptr;
+    uint32_t* n_owned = routed ? ctx->at<uint32_t>(cv.n_owned) : nullptr;
+    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err, owner, owned, n_owned, c.W, replica, c.seed));
     TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tok_dev, n, ctx->shape, routed ? 0u : replica, (uint32_t)batch_index, c.seed,
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows),
                                      ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err, owner));
@@ -152,7 +156,7 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                                       n_items, bits_for(2 * c.V), ctx->at<uint32_t>(cv.hist), &sorted));
         TENSAIR_CUDA(ctx, launch_forward(ctx->L, tok_dev, n, ctx->shape, table, ctx->at<uint32_t>(cv.rows),
                                          ctx->at<Rec>(cv.rec), ctx->at<double>(cv.gin_pos), ctx->at<double>(cv.loss_pos), err,
-                                         owner));
+                                         owned, n_owned));
         if (fork) {
             TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
             TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0));
@@ -192,7 +196,7 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
             ctx->buffered[replica] = 0;
         }
     }
-    TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err));
+    TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err, owner));
     ctx->last_n = n;
     ctx->last_pairs = pairs;
     ctx->have_last = true;

@@ -40,6 +40,7 @@ class Workload:
     seed: int = 0         # library seed (negative sampler, delays)
     reduction: int = 0    # 0: batch loss = sum of the pair losses; 1: their mean
     max_grad_buffer: int = 1  # a replica sends after every this many of its batches
+    routed: int = 0       # 1: the replicas share replica 0's batches, each training the centre words routed to it
 
     @property
     def pairs_per_batch(self) -> int:
