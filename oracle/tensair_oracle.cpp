@@ -84,35 +84,75 @@ enum : uint32_t { TAG_NEGATIVE = 1, TAG_DELAY = 2, TAG_INIT = 3, TAG_ROUTE = 4 }
 inline uint32_t mulhi32(uint32_t a, uint32_t b) { return (uint32_t)(((uint64_t)a * b) >> 32); }
 
 // ---------------------------------------------------------------------------------------------
-// Walker / Vose alias table over weights count^0.75
+// Walker alias table over weights count^0.75, built in exact integer arithmetic
 // ---------------------------------------------------------------------------------------------
-// weight_i = s*s*s with s = sqrt(sqrt(count_i)) (square roots are correctly rounded everywhere, pow
-// is not); total = sequential fp64 sum in ascending index; scaled p_i = weight_i * V / total.
-// Vose with two first-in-first-out work lists filled in ascending index order.  A "small" entry
-// s takes thresh = floor(p_s * 2^32) (capped at 2^32 - 1) and alias = front of the large list,
-// whose p becomes (p_large + p_s) - 1; when that falls below 1 it moves to the back of the small
-// list.  Whatever is left on either list accepts always (thresh all-ones, alias = itself).
+// The paper does not describe the negative sampler; the table is defined here so that its result does
+// not depend on the order in which a builder visits the entries (a sequential sweep, as below, and a
+// parallel builder working from prefix sums must produce the same bits).
+//   weight_i = s*s*s, s = sqrt(sqrt(count_i))      (fp64; square roots are correctly rounded, pow is not)
+//   u_i      = floor(weight_i * 2^sh), sh = bits - e, 2^(e-1) <= max weight < 2^e,
+//              bits = min(42, 62 - ceil(log2 V))    (integer masses below 2^bits)
+//   C        = ceil(sum u / V); the first entry of largest u takes C*V - sum u more, so that sum u = C*V:
+//              V buckets of capacity C.
+// Entries with u < C are light, the others heavy, each kind in ascending index order.  The current heavy
+// entry h, with what is left of its mass r (at first u_h), tops up light buckets in order while r > C:
+// light l keeps u_l of its bucket, alias[l] = h, r -= C - u_l.  Once r <= C the heavy entry's own bucket
+// is closed with r of its own mass, topped up by the next heavy entry h' (alias[h] = h'), which goes on
+// with r' = u_h' - (C - r).  A bucket keeping all of C accepts always (thresh all-ones, alias = itself);
+// otherwise thresh = floor(kept / C * 2^32) with the quotient taken in fp64 (both operands are exact).
+static uint32_t kept_to_thresh(uint64_t kept, uint64_t C) {
+    return (uint32_t)std::floor((double)kept / (double)C * 4294967296.0);
+}
+
 void build_alias(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias) {
-    std::vector<double> p(V);
-    double total = 0.0;
+    std::vector<double> weight(V);
+    double wmax = 0.0;
     for (uint32_t i = 0; i < V; ++i) {
         double c = (double)(counts ? counts[i] : 1);
         double s = std::sqrt(std::sqrt(c));
-        p[i] = s * s * s;
-        total += p[i];
+        weight[i] = s * s * s;
+        if (weight[i] > wmax) wmax = weight[i];
     }
-    for (uint32_t i = 0; i < V; ++i) p[i] = (p[i] * (double)V) / total;
-    std::deque<uint32_t> small, large;
-    for (uint32_t i = 0; i < V; ++i) (p[i] < 1.0 ? small : large).push_back(i);
-    for (uint32_t i = 0; i < V; ++i) { thresh[i] = 0xFFFFFFFFu; alias[i] = i; }
-    while (!small.empty() && !large.empty()) {
-        uint32_t s = small.front(); small.pop_front();
-        uint32_t l = large.front();
-        double q = std::floor(p[s] * 4294967296.0);
-        thresh[s] = q >= 4294967295.0 ? 0xFFFFFFFFu : (uint32_t)q;
-        alias[s] = l;
-        p[l] = (p[l] + p[s]) - 1.0;
-        if (p[l] < 1.0) { large.pop_front(); small.push_back(l); }
+    int e = 0;
+    std::frexp(wmax, &e);                       // wmax = f * 2^e, 0.5 <= f < 1
+    int log2V = 0;
+    while ((1ull << log2V) < V) ++log2V;
+    const int bits = 62 - log2V < 42 ? 62 - log2V : 42;
+    std::vector<uint64_t> u(V);
+    uint64_t total = 0;
+    uint32_t biggest = 0;
+    for (uint32_t i = 0; i < V; ++i) {
+        u[i] = (uint64_t)std::floor(std::ldexp(weight[i], bits - e));
+        total += u[i];
+        if (u[i] > u[biggest]) biggest = i;     // first among equals
+    }
+    const uint64_t C = (total + V - 1) / V;
+    u[biggest] += C * V - total;
+
+    std::vector<uint32_t> light, heavy;
+    for (uint32_t i = 0; i < V; ++i) {
+        (u[i] < C ? light : heavy).push_back(i);
+        thresh[i] = 0xFFFFFFFFu;
+        alias[i] = i;
+    }
+    size_t li = 0, hi = 0;
+    uint64_t r = u[heavy[0]];                   // the largest entry is never light
+    for (;;) {
+        if (r > C) {                            // top up the next light bucket
+            const uint32_t l = light[li++];
+            thresh[l] = kept_to_thresh(u[l], C);
+            alias[l] = heavy[hi];
+            r -= C - u[l];
+        } else {                                // close the heavy entry's own bucket
+            if (hi + 1 == heavy.size()) break;  // the last one keeps exactly C
+            const uint32_t h = heavy[hi], next = heavy[hi + 1];
+            if (r < C) {
+                thresh[h] = kept_to_thresh(r, C);
+                alias[h] = next;
+            }
+            r = u[next] - (C - r);
+            ++hi;
+        }
     }
 }
 

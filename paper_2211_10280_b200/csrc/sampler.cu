@@ -1,5 +1,6 @@
 // Negative sampler: alias table over count^0.75 (host build), token validation, and the kernel that
 // draws the negatives of a batch and emits the sort items of all its contributions.
+#include <algorithm>
 #include <cmath>
 #include <vector>
 
@@ -8,41 +9,72 @@
 
 namespace tensair {
 
-// Walker/Vose alias table.  weight = (sqrt(sqrt(count)))^3 so that only correctly rounded operations
-// are involved; scaled probability p = weight * V / total with total summed in index order.  Entries
-// with p < 1 ("small") and p >= 1 ("large") are queued in index order; each small entry s is paired
-// with the large entry l at the head of its queue: thresh[s] = floor(p_s * 2^32) (saturated), alias[s]
-// = l, p_l = (p_l + p_s) - 1, and l joins the tail of the small queue once p_l < 1.  Entries never
-// paired accept always (thresh = 2^32-1, alias = self).
+// Walker alias table over weights count^0.75 in exact integer arithmetic, so that this host builder and the
+// parallel device builder (alias_build.cu) give the same bits whatever order they work in.
+//   weight = (sqrt(sqrt(count)))^3 in fp64 (only correctly rounded operations);
+//   u = floor(weight * 2^(bits - e)) with 2^(e-1) <= largest weight < 2^e and bits = min(42, 62 - ceil(log2 V));
+//   C = ceil(sum u / V), the first entry of largest u is raised so that sum u = C * V: V buckets of capacity C.
+// Entries with u < C are light (deficit C - u), the others heavy (surplus u - C), each kind ranked in index
+// order, with running sums D over the deficits and S over the surpluses.  Heavy entries give their mass
+// away in rank order, to the light buckets in rank order and then to the bucket of the heavy entry before
+// them; in terms of the sums: light n is topped up by the first heavy t with S_t > D_{n-1}; heavy t keeps
+// C + S_t - D_n of its own bucket, n the first rank with D_n >= S_t, the rest comes from heavy t + 1.
+// A bucket that keeps all of C accepts always (thresh 2^32-1, alias = self), otherwise
+// thresh = floor(kept / C * 2^32), the quotient in fp64 from two exact operands.
+int alias_mass_bits(uint32_t V) {
+    int log2V = 0;
+    while ((1ull << log2V) < V) ++log2V;
+    return 62 - log2V < 42 ? 62 - log2V : 42;
+}
+
 void build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias) {
-    std::vector<double> prob(V);
-    double total = 0.0;
+    std::vector<double> weight(V);
+    double heaviest = 0.0;
     for (uint32_t i = 0; i < V; ++i) {
         const double root4 = std::sqrt(std::sqrt(counts ? (double)counts[i] : 1.0));
-        prob[i] = root4 * root4 * root4;
-        total += prob[i];
+        weight[i] = root4 * root4 * root4;
+        heaviest = std::max(heaviest, weight[i]);
     }
-    // queues as arrays with a read cursor: at most V entries ever enter each
-    std::vector<uint32_t> q_small, q_large;
-    q_small.reserve(2 * (size_t)V);
-    q_large.reserve(V);
+    const int shift = alias_mass_bits(V) - (std::ilogb(heaviest) + 1);
+    std::vector<uint64_t> mass(V);
+    uint64_t sum = 0, top = 0;
     for (uint32_t i = 0; i < V; ++i) {
-        prob[i] = prob[i] * (double)V / total;
+        mass[i] = (uint64_t)std::floor(std::ldexp(weight[i], shift));
+        sum += mass[i];
+        top = std::max(top, mass[i]);
+    }
+    const uint64_t cap = (sum + V - 1) / V;
+    *std::find(mass.begin(), mass.end(), top) += cap * V - sum;
+
+    std::vector<uint32_t> light_at, heavy_at;        // rank -> index
+    std::vector<uint64_t> deficit_sum, surplus_sum;  // inclusive running sums by rank
+    for (uint32_t i = 0; i < V; ++i) {
+        if (mass[i] < cap) {
+            light_at.push_back(i);
+            deficit_sum.push_back((deficit_sum.empty() ? 0 : deficit_sum.back()) + (cap - mass[i]));
+        } else {
+            heavy_at.push_back(i);
+            surplus_sum.push_back((surplus_sum.empty() ? 0 : surplus_sum.back()) + (mass[i] - cap));
+        }
         thresh[i] = 0xFFFFFFFFu;
         alias[i] = i;
-        if (prob[i] < 1.0) q_small.push_back(i); else q_large.push_back(i);
     }
-    size_t rs = 0, rl = 0;
-    while (rs < q_small.size() && rl < q_large.size()) {
-        const uint32_t s = q_small[rs++];
-        const uint32_t l = q_large[rl];
-        const double scaled = std::floor(prob[s] * 4294967296.0);
-        thresh[s] = scaled < 4294967295.0 ? (uint32_t)scaled : 0xFFFFFFFFu;
-        alias[s] = l;
-        prob[l] = (prob[l] + prob[s]) - 1.0;
-        if (prob[l] < 1.0) {
-            ++rl;
-            q_small.push_back(l);
+    auto to_thresh = [cap](uint64_t kept) { return (uint32_t)std::floor((double)kept / (double)cap * 4294967296.0); };
+    for (size_t n = 0; n < light_at.size(); ++n) {
+        const uint32_t i = light_at[n];
+        const uint64_t before = deficit_sum[n] - (cap - mass[i]);
+        const size_t t = std::upper_bound(surplus_sum.begin(), surplus_sum.end(), before) - surplus_sum.begin();
+        thresh[i] = to_thresh(mass[i]);
+        alias[i] = heavy_at[t];
+    }
+    for (size_t t = 0; t + 1 < heavy_at.size(); ++t) {
+        const uint64_t given = surplus_sum[t];
+        if (given == 0) continue;                    // nothing to give: its bucket is its own
+        const size_t n = std::lower_bound(deficit_sum.begin(), deficit_sum.end(), given) - deficit_sum.begin();
+        const uint64_t kept = cap + given - deficit_sum[n];
+        if (kept < cap) {
+            thresh[heavy_at[t]] = to_thresh(kept);
+            alias[heavy_at[t]] = heavy_at[t + 1];
         }
     }
 }

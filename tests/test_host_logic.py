@@ -57,6 +57,21 @@ def test_alias_table_is_bit_identical_to_the_oracle(V, seed):
     assert np.array_equal(t0, t1) and np.array_equal(a0, a1)
 
 
+@pytest.mark.parametrize("case", ["huge", "ones_and_one_big", "two_values", "powers_of_16", "V3"])
+def test_alias_table_corner_cases_are_bit_identical_to_the_oracle(case):
+    rng = np.random.default_rng(8)
+    counts = {
+        "huge": rng.integers(1, 1 << 62, 4000, dtype=np.uint64),
+        "ones_and_one_big": np.concatenate([np.ones(999, np.uint64), np.array([10 ** 12], np.uint64)]),
+        "two_values": rng.choice(np.array([3, 48], np.uint64), 2048),
+        "powers_of_16": np.uint64(16) ** rng.integers(0, 8, 1000).astype(np.uint64),   # exact weights 8^j
+        "V3": np.array([5, 5, 1], np.uint64),
+    }[case]
+    t0, a0 = oracle.build_alias(counts)
+    t1, a1 = B.tensair_build_alias_host(counts, counts.size)
+    assert np.array_equal(t0, t1) and np.array_equal(a0, a1)
+
+
 def test_alias_table_of_a_zipf_stream_matches_the_oracle():
     wl = synth.scaled(synth.MID, batches=20)
     counts = synth.stream_counts([synth.token_stream(wl, 0)], wl.V)

@@ -73,6 +73,26 @@ def test_alias_reconstructs_count_pow_075(V, seed):
     assert np.all(alias < V)
 
 
+def test_alias_targets_are_heavy_and_heavy_entries_chain_forward():
+    rng = np.random.default_rng(5)
+    V = 3000
+    counts = (rng.zipf(1.2, V).astype(np.uint64) % 50000) + 1
+    thresh, alias = oracle.build_alias(counts)
+    w = counts.astype(np.float64) ** 0.75
+    mean = w.mean()
+    partial = thresh != 0xFFFFFFFF
+    assert partial.any() and not partial.all()
+    # whatever tops up a bucket has at least the mean weight (the quantisation moves the border by < 1e-9)
+    assert np.all(w[alias[partial]] >= mean * (1 - 1e-9))
+    # a light entry keeps its own share: thresh / 2^32 = w_i / mean, to the 32-bit floor
+    light = partial & (w < mean * (1 - 1e-9))
+    np.testing.assert_allclose(thresh[light] / 2.0 ** 32, w[light] / mean, rtol=0, atol=2e-9)
+    # a heavy entry whose bucket is topped up is topped up by a later heavy entry
+    heavy_partial = partial & (w > mean * (1 + 1e-9))
+    assert np.all(alias[heavy_partial] > np.flatnonzero(heavy_partial))
+    assert np.array_equal(alias[~partial], np.flatnonzero(~partial))
+
+
 def test_alias_equal_counts_accept_always():
     thresh, alias = oracle.build_alias(np.full(64, 9, dtype=np.uint64))
     assert np.all(thresh == 0xFFFFFFFF)
