@@ -184,6 +184,8 @@ def run_ours(args):
     msg_ids = {}
 
     def step(t, host=False, info=False):
+        if wl.drift_every and t and t % wl.drift_every == 0:
+            ctx.tensair_update_sampler()                      # passive drift adaptation: the sampler follows the stream
         shared = toks_pin[t, 0].to("cuda", non_blocking=True) if (wl.routed and host) else None
         for i in range(wl.W):
             if wl.routed:       # one batch for all replicas, split by the hash of the centre word
@@ -254,6 +256,21 @@ def run_ours(args):
     ctx.tensair_profile(False)
     if ctx.tensair_sync() != B.OK:
         raise SystemExit("the device reported a bad token during the benchmark")
+
+    rebuild = None
+    if wl.drift_every:
+        # the sampler's rebuild on its own: on the device (asynchronous) and, for comparison, on one host thread
+        rebuild = {}
+        for mode, knob in (("device_ms", 1), ("host_ms", 0)):
+            B.tensair_tune("device_alias_build", knob)
+            ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            torch.cuda.synchronize()
+            ev0.record()
+            ctx.tensair_update_sampler()
+            ev1.record()
+            torch.cuda.synchronize()
+            rebuild[mode] = round(ev0.elapsed_time(ev1), 3)
+        B.tensair_tune("device_alias_build", 1)
 
     pairs_per_step = P if wl.routed else wl.W * P
     value = world * pairs_per_step * K / (ms_dev * 1e-3)
@@ -346,6 +363,8 @@ def run_ours(args):
                      "frac_of_peak": round(step_gbs / peak, 4), "rows_per_message": int(U)},
         "kernels": kernels,
     }
+    if rebuild:
+        out["sampler_rebuild"] = dict(rebuild, every_batches=wl.drift_every)
     if rank == 0 and world == 1 and not args.no_cpu_baseline:
         out["cpu_baseline"] = cpu_baseline(wl, toks_np, counts, steps=2)
     ctx.close()

@@ -228,7 +228,10 @@ TENSAIR_API int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint6
 TENSAIR_API int tensair_drain(tensair_ctx* ctx, uint32_t* n_applied);
 
 /* Rebuilds the negative sampler's alias table from the running unigram counts (initial counts plus
- * every token trained on so far).  Synchronises; the table is built by one host thread. */
+ * every token trained on so far).  The table is built on the device, asynchronously on the context's
+ * stream, bit-identical to what tensair_build_alias_host gives for the same counts.  (With the knob
+ * "device_alias_build" = 0 of tensair_tune the counts are read back, one host thread builds the table
+ * and the call synchronises.) */
 TENSAIR_API int tensair_update_sampler(tensair_ctx* ctx);
 
 /* Waits for the stream; returns and clears a pending TENSAIR_EBADTOKEN. */
@@ -304,7 +307,8 @@ TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
  * = resident blocks per multiprocessor the forward grid is sized for (0 = default),
  * "reduce_blocks_per_sm" / "apply_blocks_per_sm" = blocks per multiprocessor of the row-sum / message-apply grids,
  * "fuse_apply" = 0 applies the messages due for a receiver one launch each instead of in one pass,
- * "fused_blocks_per_sm" = blocks per multiprocessor of that pass, "overlap_sort" = 0 keeps the sort of a batch on the caller's stream instead of an internal second stream. */
+ * "fused_blocks_per_sm" = blocks per multiprocessor of that pass, "overlap_sort" = 0 keeps the sort of a batch on the caller's stream instead of an internal second stream,
+ * "device_alias_build" = 0 makes tensair_update_sampler build the table on the host. */
 TENSAIR_API int tensair_tune(const char* name, int value);
 TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);
 

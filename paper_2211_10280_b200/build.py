@@ -20,7 +20,7 @@ LIB = HERE / "libtensair.so"
 OBJ = HERE / "_build"
 
 SOURCES = ["tensair.cu", "schedule.cu", "sampler.cu", "radix_sort.cu", "forward.cu", "message.cu", "apply.cu",
-           "static_scratch.cu", "merge.cu", "topk.cu"]
+           "static_scratch.cu", "merge.cu", "topk.cu", "alias_build.cu"]
 
 NVCC_FLAGS = ["-gencode", "arch=compute_100a,code=sm_100a", "-lineinfo", "-O3", "-std=c++17",
               "-Xcompiler", "-fPIC", "-Xcompiler", "-fvisibility=hidden"]

@@ -16,7 +16,7 @@ inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 // Offsets (bytes) of everything the library keeps in the caller's scratch buffer.
 struct Carve {
     uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, terms, gin_pos, loss_pos, hist,
-        tile_counts, seg_start, long_rows, chunk_items, partials, merge_counts, topk, owner, owned, n_owned, total;
+        tile_counts, seg_start, long_rows, chunk_items, partials, merge_counts, topk, owner, owned, n_owned, alias_state, alias_work, total;
     uint64_t slot_bytes, bucket_off, ids_off, delta_off;
     uint32_t stride, max_pairs, max_contrib, max_items, max_rows, max_long, max_chunks;
 };

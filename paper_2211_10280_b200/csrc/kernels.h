@@ -9,13 +9,13 @@ namespace tensair {
 enum KernelKind {
     K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
     K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
-    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_KINDS
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_ALIAS_BUILD, K_KINDS
 };
 inline const char* kernel_name(int kind) {
     static const char* const names[K_KINDS] = {
         "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
         "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
-        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted"};
+        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted", "alias_build"};
     return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
 }
 
@@ -45,6 +45,7 @@ struct Launcher {
 struct GridShape {
     int fuse_apply = 1;              // apply the messages due for a receiver in one pass over its table
     int overlap_sort = 1;            // run the radix sort on a second stream while the forward kernel runs
+    int device_alias_build = 1;      // rebuild the sampler's alias table on the device (0: on the host, with a synchronisation)
     int reduce_blocks_per_sm = 64;
     int apply_blocks_per_sm = 64;
     int fused_blocks_per_sm = 256;
@@ -76,6 +77,18 @@ cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, co
                            item_t* items, unsigned long long* counts, const uint32_t* err, const uint8_t* owner);
 cudaError_t launch_init_input_table(const Launcher& L, float* table, const Shape& s, uint64_t seed);
 void build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias);
+int alias_mass_bits(uint32_t V);
+
+// alias_build.cu: the same table built on the device from the running counts
+struct AliasState {
+    unsigned long long heaviest_bits;   // bit pattern of the largest weight
+    unsigned long long sum, top;        // sum and maximum of the integer masses
+    unsigned long long first_top;       // smallest index holding the maximum
+    uint32_t lights, pad;               // entries lighter than a bucket's capacity
+};
+size_t alias_work_bytes(uint32_t V);
+cudaError_t launch_alias_build(const Launcher& L, const unsigned long long* counts, uint32_t V, AliasState* st,
+                               uint8_t* work, uint2* table);
 
 // radix_sort.cu
 // Stable least-significant-digit radix sort of `n` items by the low `key_bits` bits of their keys.

@@ -66,6 +66,8 @@ void carve(const tensair_config& c, Carve& k) {
     k.owner = take(c.batch);
     k.owned = take((uint64_t)c.batch * 4);
     k.n_owned = take(4);
+    k.alias_state = take(sizeof(AliasState));
+    k.alias_work = take(alias_work_bytes(c.V));
     k.total = off;
     k.bucket_off = kHeaderBytes;
     k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
@@ -429,6 +431,12 @@ int tensair_update_sampler(tensair_ctx* ctx) {
     if (!ctx) return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return TENSAIR_ECUDA;
+    if (grid_shape().device_alias_build) {
+        TENSAIR_CUDA(ctx, launch_alias_build(ctx->L, ctx->at<unsigned long long>(ctx->cv.counts), ctx->cfg.V,
+                                             ctx->at<AliasState>(ctx->cv.alias_state), ctx->at<uint8_t>(ctx->cv.alias_work),
+                                             ctx->at<uint2>(ctx->cv.alias_tab)));
+        return TENSAIR_OK;
+    }
     std::vector<uint64_t> counts(ctx->cfg.V);
     TENSAIR_CUDA(ctx, cudaMemcpyAsync(counts.data(), ctx->at<uint64_t>(ctx->cv.counts), (size_t)ctx->cfg.V * 8, cudaMemcpyDeviceToHost, ctx->stream));
     TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
@@ -580,6 +588,7 @@ int tensair_tune(const char* name, int value) {
     else if (!std::strcmp(name, "fused_blocks_per_sm") && value > 0) { grid_shape().fused_blocks_per_sm = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "fuse_apply")) { grid_shape().fuse_apply = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "overlap_sort")) { grid_shape().overlap_sort = value; return TENSAIR_OK; }
+    else if (!std::strcmp(name, "device_alias_build")) { grid_shape().device_alias_build = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "reduce_blocks_per_sm") && value > 0) { grid_shape().reduce_blocks_per_sm = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "apply_blocks_per_sm") && value > 0) { grid_shape().apply_blocks_per_sm = value; return TENSAIR_OK; }
     else return TENSAIR_EINVAL;

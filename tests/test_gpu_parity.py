@@ -349,6 +349,56 @@ def test_drift_rebuilds_the_sampler_from_running_counts(torch):
         compare_tables(o, g, j, TOL_200)
 
 
+@pytest.mark.parametrize("V,zipf", [(2, 1.0), (3, 1.0), (1023, 1.0), (1025, 0.2), (40_000, 1.2), (1_000_000, 1.0)])
+def test_alias_table_built_on_the_device_is_bit_identical(torch, V, zipf):
+    """The sampler rebuilt on the device from the running counts == the oracle's table == the host builder's."""
+    from paper_2211_10280_b200 import binding as B
+
+    wl = synth.scaled(synth.TINY, V=V, d=8, window=2, k=2, batch=512, zipf_s=zipf)
+    stream = synth.token_stream(wl, 0, 6)
+    rng = np.random.default_rng(V)
+    counts = rng.integers(1, 1000, V).astype(np.uint64) if V < 100_000 else np.ones(V, np.uint64)
+    o, g = make_pair(wl, counts=counts)
+    for b in range(6):
+        assert o.train_batch(0, stream[b], b)[0] == 0
+        g.tensair_train_batch(0, dev(torch, stream[b]), b)
+    o.update_sampler()
+    g.tensair_update_sampler()
+    to, ao, co = o.sampler()
+    tg, ag, cg = g.tensair_read_sampler()
+    assert np.array_equal(co, cg)
+    assert np.array_equal(to, tg) and np.array_equal(ao, ag)
+    th, ah = B.tensair_build_alias_host(cg, V)
+    assert np.array_equal(th, tg) and np.array_equal(ah, ag)
+    B.tensair_tune("device_alias_build", 0)
+    try:
+        g.tensair_update_sampler()
+        t2, a2, _ = g.tensair_read_sampler()
+    finally:
+        B.tensair_tune("device_alias_build", 1)
+    assert np.array_equal(t2, tg) and np.array_equal(a2, ag)
+    # and the draws of the next batch follow the new table on both sides
+    toks = synth.token_stream(wl, 0, 7)[6]
+    assert o.train_batch(0, toks, 6)[0] == 0
+    g.tensair_train_batch(0, dev(torch, toks), 6)
+    assert np.array_equal(o.read_negatives(), g.tensair_read_negatives())
+
+
+def test_alias_table_of_extreme_counts_on_the_device(torch):
+    V = 5000
+    wl = synth.scaled(synth.TINY, V=V, d=8, window=2, k=2, batch=64)
+    rng = np.random.default_rng(1)
+    for counts in (rng.integers(1, 1 << 62, V, dtype=np.uint64), np.full(V, 7, np.uint64),
+                   np.concatenate([np.ones(V - 1, np.uint64), np.array([10 ** 15], np.uint64)]),
+                   np.uint64(16) ** rng.integers(0, 8, V).astype(np.uint64)):
+        o, g = make_pair(wl, counts=counts)
+        o.update_sampler()
+        g.tensair_update_sampler()
+        to, ao, _ = o.sampler()
+        tg, ag, _ = g.tensair_read_sampler()
+        assert np.array_equal(to, tg) and np.array_equal(ao, ag)
+
+
 # ------------------------------------------------------------------ routed mini-batches (hash partition by centre word)
 def _routed_step(torch, o, g, wl, toks, b, tol):
     """One shared batch through every replica of both sides, compared piece by piece; returns the GPU losses."""
