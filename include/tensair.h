@@ -149,7 +149,7 @@ TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
  *   message    one delta row fp32(-lr * gradient) per touched row, ids ascending;
  *   local GA   the message is applied to the replica at once (staleness 0);
  *   send       it is filed for every other replica at step batch_index + delay(batch_index, replica, j).
- *              With max_grad_buffer = m > 1 (Algorithm 1: "gradients += gradient", sent when the count
+ *              With max_grad_buffer = m > 1 (Algorithm 1: gradients are accumulated and sent when their count
  *              reaches maxGradBuffer) only every m-th batch of a replica sends: the sum of its last m
  *              messages over the union of their rows, each row's deltas added in fp32 in the order they
  *              were computed; tensair_read_message then holds only for those batch indices.
@@ -308,6 +308,8 @@ TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
  * "reduce_blocks_per_sm" / "apply_blocks_per_sm" = blocks per multiprocessor of the row-sum / message-apply grids,
  * "fuse_apply" = 0 applies the messages due for a receiver one launch each instead of in one pass,
  * "fused_blocks_per_sm" = blocks per multiprocessor of that pass, "overlap_sort" = 0 keeps the sort of a batch on the caller's stream instead of an internal second stream,
+ * "overlap_long_rows" = 0 keeps the sums of the rows with many contributions, the message's bucket index and the
+ * loss sum on the caller's stream instead of beside the short-row sums on the second stream,
  * "device_alias_build" = 0 makes tensair_update_sampler build the table on the host. */
 TENSAIR_API int tensair_tune(const char* name, int value);
 TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);

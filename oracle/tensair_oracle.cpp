@@ -425,8 +425,8 @@ static int train_batch(Oracle* o, uint32_t replica, const int32_t* tokens, uint3
     add_rows(*o, replica, m);
     if (loss_out) *loss_out = loss;
     if (n_rows_out) *n_rows_out = (uint32_t)U;
-    // Algorithm 1, train, mini-batch branch: "gradients += gradient; count += 1; if count >= maxGradBuffer:
-    // send".  The buffered gradients are summed row by row in the order they were computed (one fp32
+    // Algorithm 1, train, mini-batch branch: the gradient joins the buffer, and the buffer is sent once it
+    // holds maxGradBuffer gradients.  The buffered gradients are summed row by row in the order they were computed (one fp32
     // addition per element and buffered gradient; a row missing from a gradient adds nothing), over
     // the union of their rows; the buffer is emptied after the send.
     o->buffered[replica].push_back(std::move(m));

@@ -9,13 +9,13 @@ namespace tensair {
 enum KernelKind {
     K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
     K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
-    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_ALIAS_BUILD, K_KINDS
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_ALIAS_BUILD, K_HEADS_LONG, K_KINDS
 };
 inline const char* kernel_name(int kind) {
     static const char* const names[K_KINDS] = {
         "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
         "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
-        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted", "alias_build"};
+        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted", "alias_build", "heads_long_rows"};
     return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
 }
 
@@ -45,6 +45,7 @@ struct Launcher {
 struct GridShape {
     int fuse_apply = 1;              // apply the messages due for a receiver in one pass over its table
     int overlap_sort = 1;            // run the radix sort on a second stream while the forward kernel runs
+    int overlap_long_rows = 1;       // sum the long rows (and index the message, sum the loss) on it while the short rows are summed
     int device_alias_build = 1;      // rebuild the sampler's alias table on the device (0: on the host, with a synchronisation)
     int reduce_blocks_per_sm = 64;
     int apply_blocks_per_sm = 64;
@@ -110,11 +111,14 @@ cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t 
 uint32_t heads_tiles(uint32_t n_items);
 cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
                          MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
-                         const Rec* rec, Rec* terms, const uint32_t* err);
-cudaError_t launch_reduce(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
-                          const uint32_t* seg_start, const double* gin_pos, float* table,
-                          float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
-                          ChunkItem* chunk_items, double* partials);
+                         const Rec* rec, Rec* terms, const uint32_t* err, LongRow* long_rows, ChunkItem* chunk_items);
+cudaError_t launch_reduce_rows(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
+                               const uint32_t* seg_start, const double* gin_pos, float* table, float* delta,
+                               const Shape& s, double scale);
+cudaError_t launch_reduce_long_rows(const Launcher& L, const Rec* terms, const uint32_t* ids, const uint32_t* seg_start,
+                                    const double* gin_pos, float* table, float* delta, const Shape& s, double scale,
+                                    const uint32_t* long_counters, const LongRow* long_rows,
+                                    const ChunkItem* chunk_items, double* partials);
 
 // apply.cu
 cudaError_t launch_apply(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,

@@ -1,4 +1,4 @@
-// Sum of buffered gradient messages (Algorithm 1 with maxGradBuffer = m > 1: "gradients += gradient", sent
+// Sum of buffered gradient messages (Algorithm 1 with maxGradBuffer = m > 1: gradients are accumulated and sent
 // after every m-th mini-batch).  The m messages of one replica are merged into one: the union of their
 // rows, each row the fp32 sum of its delta rows in the order the messages were computed.
 //

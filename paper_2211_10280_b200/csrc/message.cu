@@ -156,9 +156,41 @@ k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, c
     }
 }
 
+// Lists the rows with more than kChunk contributions and cuts them into chunks (one thread per row finds
+// them, its warp writes the chunk items).  The order of the lists does not reach any sum.
+__global__ void __launch_bounds__(256)
+k_list_long_rows(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ seg_start,
+                 uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows,
+                 ChunkItem* __restrict__ chunk_items, const uint32_t* __restrict__ err) {
+    if (*err) return;
+    const uint32_t n_rows = hdr->n_rows, lane = threadIdx.x & 31;
+    const uint32_t first = (blockIdx.x * blockDim.x + threadIdx.x) - lane;   // row of lane 0
+    for (uint32_t m0 = first; m0 < n_rows; m0 += gridDim.x * blockDim.x) {
+        const uint32_t m = m0 + lane;
+        uint32_t nch = 0, base = 0;
+        if (m < n_rows) {
+            const uint32_t len = seg_start[m + 1] - seg_start[m];
+            if (len > kChunk) {
+                nch = (len + kChunk - 1) / kChunk;
+                const uint32_t slot = atomicAdd(long_counters, 1u);
+                base = atomicAdd(long_counters + 1, nch);
+                long_rows[slot] = LongRow{m, base, nch};
+            }
+        }
+        uint32_t todo = __ballot_sync(0xFFFFFFFFu, nch != 0);
+        while (todo) {
+            const int src = __ffs(todo) - 1;
+            todo &= todo - 1;
+            const uint32_t row = m0 + src;
+            const uint32_t n = __shfl_sync(0xFFFFFFFFu, nch, src), b = __shfl_sync(0xFFFFFFFFu, base, src);
+            for (uint32_t c = lane; c < n; c += 32) chunk_items[b + c] = ChunkItem{row, c};
+        }
+    }
+}
+
 cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
                          MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
-                         const Rec* rec, Rec* terms, const uint32_t* err) {
+                         const Rec* rec, Rec* terms, const uint32_t* err, LongRow* long_rows, ChunkItem* chunk_items) {
     const uint32_t tiles = heads_tiles(n_items);
     if (tiles) {
         Timed timed(L, K_HEADS_COUNT);
@@ -171,6 +203,10 @@ cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_ite
     if (tiles) {
         Timed timed(L, K_HEADS_WRITE);
         k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, rec, terms, err);
+    }
+    if (tiles) {
+        Timed timed(L, K_HEADS_LONG);
+        k_list_long_rows<<<L.sms * 4, 256, 0, L.stream>>>(hdr, seg_start, long_counters, long_rows, chunk_items, err);
     }
     return cudaGetLastError();
 }
@@ -326,8 +362,7 @@ __global__ void __launch_bounds__(kReduceThreads)
 k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids,
               const uint32_t* __restrict__ seg_start, const double* __restrict__ gin_pos,
               float4* __restrict__ table, float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4,
-              double scale, uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows,
-              ChunkItem* __restrict__ chunk_items) {
+              double scale) {
     extern __shared__ __align__(128) float4 out_rows[];   // [warps in block][kOutBuffers][stride4]
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
@@ -354,17 +389,7 @@ k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, 
     for (; m < n_rows; m += nwarps) {
         const Meta after = load_meta(m + 2 * nwarps);
         const Rec nxt_terms = load_terms(nxt);
-        if (cur.end - cur.beg > kChunk) {
-            const uint32_t nch = (cur.end - cur.beg + kChunk - 1) / kChunk;
-            uint32_t base = 0;
-            if (lane == 0) {
-                const uint32_t slot = atomicAdd(long_counters, 1u);
-                base = atomicAdd(long_counters + 1, nch);
-                long_rows[slot] = LongRow{m, base, nch};
-            }
-            base = __shfl_sync(0xFFFFFFFFu, base, 0);
-            for (uint32_t c = lane; c < nch; c += 32) chunk_items[base + c] = ChunkItem{m, c};
-        } else {
+        if (cur.end - cur.beg <= kChunk) {   // longer rows are on the long-row list and summed by the chunk kernels
             RowSum<NV> sum;
             sum.clear();
             accumulate_segment<NV, kTermsInFlightRows>(terms, cur.beg, cur.end, cur.id < V, gin_pos, table, d4, stride4, lane, sum, true,
@@ -499,48 +524,69 @@ k_reduce_long(const uint32_t* __restrict__ ids, const double* __restrict__ parti
 }
 
 template <int NV>
-static cudaError_t reduce_all(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
-                              const uint32_t* seg_start, const double* gin_pos, float* table,
-                              float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
-                              ChunkItem* chunk_items, double* partials) {
+static cudaError_t reduce_short(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
+                                const uint32_t* seg_start, const double* gin_pos, float* table, float* delta,
+                                const Shape& s, double scale) {
     const uint32_t stride4 = s.stride / 4;
     const size_t out_smem = (size_t)(kReduceThreads / 32) * kOutBuffers * s.stride * 4;
+    Timed timed(L, K_REDUCE_ROWS);
+    k_reduce_rows<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, out_smem, L.stream>>>(
+        terms, hdr, ids, seg_start, gin_pos, reinterpret_cast<float4*>(table), reinterpret_cast<float4*>(delta), s.V, s.d4,
+        stride4, scale);
+    return cudaGetLastError();
+}
+
+template <int NV>
+static cudaError_t reduce_listed(const Launcher& L, const Rec* terms, const uint32_t* ids, const uint32_t* seg_start,
+                                 const double* gin_pos, float* table, float* delta, const Shape& s, double scale,
+                                 const uint32_t* long_counters, const LongRow* long_rows, const ChunkItem* chunk_items,
+                                 double* partials) {
+    const uint32_t stride4 = s.stride / 4;
     float4* t4 = reinterpret_cast<float4*>(table);
     float4* d4p = reinterpret_cast<float4*>(delta);
     {
-    Timed timed(L, K_REDUCE_ROWS);
-    k_reduce_rows<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, out_smem, L.stream>>>(terms, hdr, ids, seg_start, gin_pos, t4, d4p, s.V, s.d4, stride4,
-                                                    scale, long_counters, long_rows, chunk_items);
+        Timed timed(L, K_REDUCE_CHUNKS);
+        k_reduce_chunks<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, 0, L.stream>>>(
+            terms, ids, seg_start, gin_pos, t4, s.V, s.d4, stride4, long_counters, chunk_items, partials);
     }
     {
-    Timed timed(L, K_REDUCE_CHUNKS);
-    k_reduce_chunks<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, 0, L.stream>>>(terms, ids, seg_start, gin_pos, t4, s.V, s.d4, stride4,
-                                                      long_counters, chunk_items, partials);
-    }
-    {
-    Timed timed(L, K_REDUCE_LONG);
-    uint32_t long_warps = 49152 / (s.d * 8);          // run sums of one block within 48 KB of shared memory
-    if (long_warps > (uint32_t)kLongWarps) long_warps = kLongWarps;
-    if (long_warps < 1) long_warps = 1;
-    k_reduce_long<NV><<<L.sms * 2, long_warps * 32, (size_t)long_warps * s.d * 8, L.stream>>>(
-        ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters, long_rows, long_warps);
+        Timed timed(L, K_REDUCE_LONG);
+        uint32_t long_warps = 49152 / (s.d * 8);          // run sums of one block within 48 KB of shared memory
+        if (long_warps > (uint32_t)kLongWarps) long_warps = kLongWarps;
+        if (long_warps < 1) long_warps = 1;
+        k_reduce_long<NV><<<L.sms * 2, long_warps * 32, (size_t)long_warps * s.d * 8, L.stream>>>(
+            ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters, long_rows, long_warps);
     }
     return cudaGetLastError();
 }
 
-cudaError_t launch_reduce(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
-                          const uint32_t* seg_start, const double* gin_pos, float* table,
-                          float* delta, const Shape& s, double scale, uint32_t* long_counters, LongRow* long_rows,
-                          ChunkItem* chunk_items, double* partials) {
-#define TENSAIR_RED(NV) \
-    return reduce_all<NV>(L, terms, hdr, ids, seg_start, gin_pos, table, delta, s, scale, long_counters, long_rows, \
-                          chunk_items, partials)
-    if (s.d4 <= 32) TENSAIR_RED(1);
-    if (s.d4 <= 64) TENSAIR_RED(2);
-    if (s.d4 <= 96) TENSAIR_RED(3);
-    if (s.d4 <= 128) TENSAIR_RED(4);
-    TENSAIR_RED(8);
-#undef TENSAIR_RED
+#define TENSAIR_BY_WIDTH(CALL)            \
+    if (s.d4 <= 32) return CALL(1);       \
+    if (s.d4 <= 64) return CALL(2);       \
+    if (s.d4 <= 96) return CALL(3);       \
+    if (s.d4 <= 128) return CALL(4);      \
+    return CALL(8)
+
+// Rows with at most kChunk contributions: summed, written into the message and (output rows) added to the table.
+cudaError_t launch_reduce_rows(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
+                               const uint32_t* seg_start, const double* gin_pos, float* table, float* delta,
+                               const Shape& s, double scale) {
+#define TENSAIR_CALL(NV) reduce_short<NV>(L, terms, hdr, ids, seg_start, gin_pos, table, delta, s, scale)
+    TENSAIR_BY_WIDTH(TENSAIR_CALL);
+#undef TENSAIR_CALL
 }
+
+// The listed long rows: chunk partials, then one block per row.  Touches none of the rows the kernel above
+// writes and reads nothing it writes, so the two may run side by side.
+cudaError_t launch_reduce_long_rows(const Launcher& L, const Rec* terms, const uint32_t* ids, const uint32_t* seg_start,
+                                    const double* gin_pos, float* table, float* delta, const Shape& s, double scale,
+                                    const uint32_t* long_counters, const LongRow* long_rows,
+                                    const ChunkItem* chunk_items, double* partials) {
+#define TENSAIR_CALL(NV) \
+    reduce_listed<NV>(L, terms, ids, seg_start, gin_pos, table, delta, s, scale, long_counters, long_rows, chunk_items, partials)
+    TENSAIR_BY_WIDTH(TENSAIR_CALL);
+#undef TENSAIR_CALL
+}
+#undef TENSAIR_BY_WIDTH
 
 }  // namespace tensair

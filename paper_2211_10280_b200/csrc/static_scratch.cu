@@ -117,13 +117,18 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
                                       reinterpret_cast<uint32_t*>(in_ws(sc.hist)), &sorted));
         TENSAIR_CUDA(ctx, launch_heads(ctx->L, sorted, n_items, c.V, reinterpret_cast<uint32_t*>(in_ws(sc.tile_counts)), hdr,
                                        ctx->slot_ids(slot), reinterpret_cast<uint32_t*>(in_ws(sc.seg_start)),
-                                       long_counters, ctx->at<Rec>(cv.rec), terms, err));
-        TENSAIR_CUDA(ctx, launch_reduce(ctx->L, terms, hdr, ctx->slot_ids(slot),
-                                        reinterpret_cast<uint32_t*>(in_ws(sc.seg_start)), gin_pos, table,
-                                        ctx->slot_delta(slot), ctx->shape, scale, long_counters,
-                                        reinterpret_cast<LongRow*>(in_ws(sc.long_rows)),
-                                        reinterpret_cast<ChunkItem*>(in_ws(sc.chunk_items)),
-                                        reinterpret_cast<double*>(in_ws(sc.partials))));
+                                       long_counters, ctx->at<Rec>(cv.rec), terms, err,
+                                       reinterpret_cast<LongRow*>(in_ws(sc.long_rows)),
+                                       reinterpret_cast<ChunkItem*>(in_ws(sc.chunk_items))));
+        TENSAIR_CUDA(ctx, launch_reduce_rows(ctx->L, terms, hdr, ctx->slot_ids(slot),
+                                             reinterpret_cast<uint32_t*>(in_ws(sc.seg_start)), gin_pos, table,
+                                             ctx->slot_delta(slot), ctx->shape, scale));
+        TENSAIR_CUDA(ctx, launch_reduce_long_rows(ctx->L, terms, ctx->slot_ids(slot),
+                                                  reinterpret_cast<uint32_t*>(in_ws(sc.seg_start)), gin_pos, table,
+                                                  ctx->slot_delta(slot), ctx->shape, scale, long_counters,
+                                                  reinterpret_cast<LongRow*>(in_ws(sc.long_rows)),
+                                                  reinterpret_cast<ChunkItem*>(in_ws(sc.chunk_items)),
+                                                  reinterpret_cast<double*>(in_ws(sc.partials))));
         TENSAIR_CUDA(ctx, launch_apply_rows(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_delta(slot), table, ctx->shape, 1));
     } else {
         TENSAIR_CUDA(ctx, cudaMemsetAsync(hdr, 0, sizeof(MsgHeader), ctx->stream));

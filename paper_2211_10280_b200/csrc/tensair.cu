@@ -166,22 +166,39 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
         TENSAIR_CUDA(ctx, launch_heads(ctx->L, sorted, n_items, c.V, ctx->at<uint32_t>(cv.tile_counts), hdr,
                                        ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
                                        ctx->at<uint32_t>(cv.long_counters), ctx->at<Rec>(cv.rec),
-                                       ctx->at<Rec>(cv.terms), err));
-        TENSAIR_CUDA(ctx, launch_reduce(ctx->L, ctx->at<Rec>(cv.terms), hdr, ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
-                                        ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot),
-                                        ctx->shape, scale, ctx->at<uint32_t>(cv.long_counters),
-                                        ctx->at<LongRow>(cv.long_rows), ctx->at<ChunkItem>(cv.chunk_items),
-                                        ctx->at<double>(cv.partials)));
+                                       ctx->at<Rec>(cv.terms), err, ctx->at<LongRow>(cv.long_rows),
+                                       ctx->at<ChunkItem>(cv.chunk_items)));
+        // The few rows with many contributions, the message's bucket index and the loss are small latency-bound
+        // kernels; they touch nothing the short-row kernel writes, so they run beside it on the second stream.
+        const bool beside = ctx->side && grid_shape().overlap_long_rows;
+        const Launcher& L2 = beside ? ctx->L_side : ctx->L;
+        if (beside) {
+            TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
+            TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
+        }
+        TENSAIR_CUDA(ctx, launch_reduce_long_rows(L2, ctx->at<Rec>(cv.terms), ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
+                                                  ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot), ctx->shape, scale,
+                                                  ctx->at<uint32_t>(cv.long_counters), ctx->at<LongRow>(cv.long_rows),
+                                                  ctx->at<ChunkItem>(cv.chunk_items), ctx->at<double>(cv.partials)));
+        TENSAIR_CUDA(ctx, launch_bucket_index(L2, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
+        TENSAIR_CUDA(ctx, launch_loss_sum(L2, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err, owner));
+        TENSAIR_CUDA(ctx, launch_reduce_rows(ctx->L, ctx->at<Rec>(cv.terms), hdr, ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
+                                             ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot), ctx->shape, scale));
+        if (beside) {
+            TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
+            TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0));
+        }
         // input rows last: they were the sources of every output-row sum
         TENSAIR_CUDA(ctx, launch_apply_rows(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_delta(slot), table, ctx->shape, 1));
     } else {
         TENSAIR_CUDA(ctx, cudaMemsetAsync(hdr, 0, sizeof(MsgHeader), ctx->stream));
+        TENSAIR_CUDA(ctx, launch_bucket_index(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
+        TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err, owner));
     }
-    TENSAIR_CUDA(ctx, launch_bucket_index(ctx->L, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
     if (m_buf > 1) {
         ++ctx->buffered[replica];
         if (sends) {
-            // Algorithm 1: "if gradients_count >= maxGradBuffer: send_gradients(gradients)"
+            // Algorithm 1: the buffered gradients are sent once their count reaches maxGradBuffer
             MergeInputs in;
             in.count = m_buf;
             for (uint32_t b = 0; b < m_buf; ++b) {
@@ -198,7 +215,6 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
             ctx->buffered[replica] = 0;
         }
     }
-    TENSAIR_CUDA(ctx, launch_loss_sum(ctx->L, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err, owner));
     ctx->last_n = n;
     ctx->last_pairs = pairs;
     ctx->have_last = true;
@@ -588,6 +604,7 @@ int tensair_tune(const char* name, int value) {
     else if (!std::strcmp(name, "fused_blocks_per_sm") && value > 0) { grid_shape().fused_blocks_per_sm = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "fuse_apply")) { grid_shape().fuse_apply = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "overlap_sort")) { grid_shape().overlap_sort = value; return TENSAIR_OK; }
+    else if (!std::strcmp(name, "overlap_long_rows")) { grid_shape().overlap_long_rows = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "device_alias_build")) { grid_shape().device_alias_build = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "reduce_blocks_per_sm") && value > 0) { grid_shape().reduce_blocks_per_sm = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "apply_blocks_per_sm") && value > 0) { grid_shape().apply_blocks_per_sm = value; return TENSAIR_OK; }

@@ -688,7 +688,7 @@ def test_routed_parts_of_a_minibatch_add_up_to_the_gradient_of_the_whole_batch(r
 
 # ------------------------------------------------------------------ maxGradBuffer > 1
 def test_buffered_gradients_are_summed_over_the_union_of_their_rows_and_sent_every_mth_batch():
-    # Algorithm 1: gradients += gradient; count += 1; send when count >= maxGradBuffer.
+    # Algorithm 1: every gradient joins the buffer; the buffer is sent when it holds maxGradBuffer gradients.
     V, d, m, T = 300, 6, 3, 7
     wl = synth.scaled(synth.TINY, V=V, d=d, batch=48, batches=T)
     stream = synth.token_stream(wl, 0)
