@@ -46,14 +46,14 @@ __device__ inline double neg_log_sigmoid(double x) { return (x < 0.0 ? -x : 0.0)
 
 constexpr int kFwdWarps = 2;       // warps per block
 
-// One warp per centre position (grid-stride), no block-level cooperation.  For every pair of the
-// position the warp stages the pair's 1 + k output rows into its own shared-memory buffer with one
+// One warp per side of a centre position (grid-stride), no block-level cooperation.  For every pair of
+// its side the warp stages the pair's 1 + k output rows into its own shared-memory buffer with one
 // bulk asynchronous copy per row (all in flight together, completion counted by an mbarrier), then
 //   1. takes the partial dot products of all staged rows with the centre row held in registers,
 //   2. reduces them with a transposing shuffle network that leaves row j's dot product in lanes 2j, 2j+1,
 //   3. evaluates sigmoid and loss for all rows at once (one row per lane pair instead of one per warp),
 //   4. re-reads the staged rows and adds g * u to the centre gradient kept in registers.
-// The centre gradient is written once per position; nothing is shared between warps.
+// The partial centre gradient of the side is written once; nothing is shared between warps.
 // NV: float4 slices per lane.  CR: rows reduced together (16 or 8); 32 / CR lanes share a row's scalar.
 template <int NV, int CR>
 __global__ void __launch_bounds__(kFwdWarps * 32)
@@ -75,10 +75,13 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
     const float4* __restrict__ tout = table + (size_t)V * stride4;
     const uint32_t warp = blockIdx.x * kFwdWarps + wib, nwarps = gridDim.x * kFwdWarps;
 
+    // A unit of work is one side of a centre position: the pairs with the context to its left, or to its
+    // right (half a position's work, so that the units spread evenly over the warps).
     // routed batch: only the listed centre positions are this replica's
-    const uint32_t n_mine = owned ? *n_owned : n;
-    for (uint32_t at = warp; at < n_mine && !failed; at += nwarps) {
-        const uint32_t q = owned ? owned[at] : at;
+    const uint32_t n_units = 2 * (owned ? *n_owned : n);
+    for (uint32_t at = warp; at < n_units && !failed; at += nwarps) {
+        const uint32_t q = owned ? owned[at >> 1] : (at >> 1);
+        const uint32_t side = at & 1u;
         const uint32_t centre = (uint32_t)tok[q];
         const float4* __restrict__ vin = table + (size_t)centre * stride4;
         double v[NV][4], acc[NV][4];
@@ -92,9 +95,9 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
         double loss = 0.0;
         const uint32_t lo = q > w ? q - w : 0;
         const uint32_t hi = q + w < n ? q + w : n - 1;
-        uint32_t p = pair_offset(q, n, w);
-        for (uint32_t c = lo; c <= hi && !failed; ++c) {
-            if (c == q) continue;
+        const uint32_t c_beg = side ? q + 1 : lo, c_end = side ? hi + 1 : q;
+        uint32_t p = pair_offset(q, n, w) + (side ? q - lo : 0u);
+        for (uint32_t c = c_beg; c < c_end && !failed; ++c) {
             const uint32_t ctx = (uint32_t)tok[c];
             const uint32_t cbase = p * K1;
             ++p;
@@ -183,7 +186,7 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
             }
         }
         if (failed) break;
-        double2* out = reinterpret_cast<double2*>(gin_pos + (size_t)q * stride4 * 4);
+        double2* out = reinterpret_cast<double2*>(gin_pos + (size_t)(2 * q + side) * stride4 * 4);
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             const uint32_t e = lane + 32 * i;
@@ -194,7 +197,7 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
         }
 #pragma unroll
         for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xFFFFFFFFu, loss, o);
-        if (lane == 0) loss_pos[q] = loss;
+        if (lane == 0) loss_pos[2 * q + side] = loss;
     }
     if (failed && lane == 0) atomicOr(err, 2u);
 }
@@ -223,7 +226,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
     const uint32_t stride4 = s.stride / 4;
     const float4* t4 = reinterpret_cast<const float4*>(table);
-    uint32_t blocks = (n + kFwdWarps - 1) / kFwdWarps;
+    uint32_t blocks = (2 * n + kFwdWarps - 1) / kFwdWarps;
     const uint32_t resident = (uint32_t)(L.sms * blocks_per_sm);
     if (blocks > resident) blocks = resident;
     Timed timed(L, K_FORWARD);
@@ -250,15 +253,15 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     return cudaGetLastError();
 }
 
-// Sum of the per-position losses (in a routed batch: of the replica's own positions) in a fixed order, in fp64.
+// Sum of the losses of the 2n half positions (in a routed batch: of the replica's own positions) in a fixed order, in fp64.
 __global__ void __launch_bounds__(1024)
 k_loss_sum(const double* __restrict__ loss_pos, uint32_t n, double* __restrict__ loss, const uint32_t* __restrict__ err,
            const uint8_t* __restrict__ owner) {
     __shared__ double part[1024];
     double s = 0.0;
     if (!*err)
-        for (uint32_t i = threadIdx.x; i < n; i += 1024)
-            if (!owner || owner[i]) s += loss_pos[i];
+        for (uint32_t i = threadIdx.x; i < 2 * n; i += 1024)
+            if (!owner || owner[i >> 1]) s += loss_pos[i];
     part[threadIdx.x] = s;
     __syncthreads();
     for (int o = 512; o > 0; o >>= 1) {

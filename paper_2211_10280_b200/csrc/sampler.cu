@@ -120,8 +120,10 @@ __device__ inline uint32_t alias_pick(const uint2* __restrict__ tab, uint32_t V,
 
 // One thread per (centre position q, window slot s, draw pair jp).  Window slot s in [0, 2w) stands
 // for context position q + (s < w ? s - w : s - w + 1); slots outside the batch do nothing.
-// Thread jp = 0 also emits the positive contribution; thread (s = 0, jp = 0) emits the position's
-// input-row item and counts the token.  In a routed batch (owner != nullptr) the positions of other
+// Thread jp = 0 also emits the positive contribution; thread (s = 0, jp = 0) counts the token and emits the
+// position's two input-row items: the forward kernel leaves one partial centre gradient for the pairs
+// to the left of the position and one for those to its right (items 2q and 2q + 1; the contributions
+// follow from item 2n on).  In a routed batch (owner != nullptr) the positions of other
 // replicas' centre words emit only items that sort past every row and are never read.
 __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t w, uint32_t k,
                           uint32_t replica, uint32_t batch_lo, uint32_t key0, uint32_t key1,
@@ -141,7 +143,10 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
     const bool own = !owner || owner[q];
     if (s == 0 && jp == 0) {
         if (own) atomicAdd(counts + centre, 1ULL);
-        if (n >= 2) items[q] = make_item(own ? centre : 2 * V, q);
+        if (n >= 2) {
+            items[2 * q] = make_item(own ? centre : 2 * V, 2 * q);
+            items[2 * q + 1] = make_item(own ? centre : 2 * V, 2 * q + 1);
+        }
     }
     const int64_t c = (int64_t)q + (s < w ? (int64_t)s - (int64_t)w : (int64_t)s - (int64_t)w + 1);
     if (c < 0 || c >= (int64_t)n) return;
@@ -151,25 +156,25 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
     const uint32_t ctx = (uint32_t)tok[c];
     const uint32_t cbase = p * K1;
     if (!own) {
-        if (jp == 0) items[n + cbase] = make_item(2 * V, cbase);
+        if (jp == 0) items[2 * n + cbase] = make_item(2 * V, cbase);
         const uint32_t j0 = 2 * jp;
-        items[n + cbase + 1 + j0] = make_item(2 * V, cbase + 1 + j0);
-        if (j0 + 1 < k) items[n + cbase + 2 + j0] = make_item(2 * V, cbase + 2 + j0);
+        items[2 * n + cbase + 1 + j0] = make_item(2 * V, cbase + 1 + j0);
+        if (j0 + 1 < k) items[2 * n + cbase + 2 + j0] = make_item(2 * V, cbase + 2 + j0);
         return;
     }
     if (jp == 0) {
         rows[cbase] = ctx;
-        items[n + cbase] = make_item(V + ctx, cbase);
+        items[2 * n + cbase] = make_item(V + ctx, cbase);
     }
     const Philox4 r = philox4x32_10(Philox4{p, jp, batch_lo, kTagNegative | replica}, key0, key1);
     const uint32_t j0 = 2 * jp;
     const uint32_t n0 = alias_pick(alias_tab, V, r.x, r.y);
     rows[cbase + 1 + j0] = n0;
-    items[n + cbase + 1 + j0] = make_item(n0 == ctx ? 2 * V : V + n0, cbase + 1 + j0);
+    items[2 * n + cbase + 1 + j0] = make_item(n0 == ctx ? 2 * V : V + n0, cbase + 1 + j0);
     if (j0 + 1 < k) {
         const uint32_t n1 = alias_pick(alias_tab, V, r.z, r.w);
         rows[cbase + 2 + j0] = n1;
-        items[n + cbase + 2 + j0] = make_item(n1 == ctx ? 2 * V : V + n1, cbase + 2 + j0);
+        items[2 * n + cbase + 2 + j0] = make_item(n1 == ctx ? 2 * V : V + n1, cbase + 2 + j0);
     }
 }
 

@@ -41,8 +41,8 @@ void carve_static(const tensair_config& c, const Carve& cv, StaticCarve& k) {
     k.items_a = take((uint64_t)cv.max_items * 8);
     k.items_b = take((uint64_t)cv.max_items * 8);
     k.terms = take((uint64_t)cv.max_items * sizeof(Rec));
-    k.gin_pos = take((uint64_t)c.batch * cv.stride * 8);
-    k.loss_pos = take((uint64_t)c.batch * 8);
+    k.gin_pos = take((uint64_t)2 * c.batch * cv.stride * 8);
+    k.loss_pos = take((uint64_t)2 * c.batch * 8);
     k.hist = take((uint64_t)sort_hist_words(cv.max_items) * 4);
     k.tile_counts = take((uint64_t)(heads_tiles(cv.max_items) + 1) * 4);
     k.seg_start = take((uint64_t)(cv.max_rows + 2) * 4);
@@ -91,7 +91,7 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
     if (rc != TENSAIR_OK) return rc;
     const uint32_t slot = ctx->sched->slot_of(replica, batch_index);
     const uint32_t pairs = n_tokens >= 2 ? pair_count(n_tokens, c.window) : 0;
-    const uint32_t n_items = pairs ? n_tokens + pairs * (c.k + 1) : 0;
+    const uint32_t n_items = pairs ? 2 * n_tokens + pairs * (c.k + 1) : 0;
     uint32_t* err = ctx->at<uint32_t>(cv.err);
     float* table = ctx->table_of(replica);
     MsgHeader* hdr = ctx->slot_hdr(slot);

@@ -36,7 +36,7 @@ void carve(const tensair_config& c, Carve& k) {
     k.stride = c.row_stride ? c.row_stride : (uint32_t)round_up(c.d, 8);
     k.max_pairs = pair_count(c.batch, c.window);
     k.max_contrib = k.max_pairs * (c.k + 1);
-    k.max_items = c.batch + k.max_contrib;
+    k.max_items = 2 * c.batch + k.max_contrib;   // two input-row items per position, then the contributions
     k.max_rows = (c.batch < c.V ? c.batch : c.V) + (k.max_contrib < c.V ? k.max_contrib : c.V);
     k.max_long = k.max_items / kChunk + 1;
     k.max_chunks = 2 * (k.max_items / kChunk) + 2;
@@ -53,8 +53,8 @@ void carve(const tensair_config& c, Carve& k) {
     k.items_b = take((uint64_t)k.max_items * 8);
     k.rec = take((uint64_t)k.max_contrib * sizeof(Rec));
     k.terms = take((uint64_t)k.max_items * sizeof(Rec));
-    k.gin_pos = take((uint64_t)c.batch * k.stride * 8);
-    k.loss_pos = take((uint64_t)c.batch * 8);
+    k.gin_pos = take((uint64_t)2 * c.batch * k.stride * 8);
+    k.loss_pos = take((uint64_t)2 * c.batch * 8);
     k.hist = take((uint64_t)sort_hist_words(k.max_items) * 4);
     k.tile_counts = take((uint64_t)(heads_tiles(k.max_items) + 1) * 4);
     k.seg_start = take((uint64_t)(k.max_rows + 2) * 4);
@@ -131,7 +131,7 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                                      : c.W * (c.max_delay + 1) + replica * m_buf + ctx->buffered[replica];
     const uint32_t pairs = n >= 2 ? pair_count(n, c.window) : 0;
     const uint32_t contrib = pairs * (c.k + 1);
-    const uint32_t n_items = pairs ? n + contrib : 0;
+    const uint32_t n_items = pairs ? 2 * n + contrib : 0;
     uint32_t* err = ctx->at<uint32_t>(cv.err);
     float* table = ctx->table_of(replica);
     MsgHeader* hdr = ctx->slot_hdr(slot);
@@ -332,7 +332,11 @@ int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const u
     if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->sched = new Schedule(cfg->W, cfg->max_delay, cfg->seed);
     ctx->buffered.assign(cfg->W, 0);
-    if (cudaStreamCreateWithFlags(&ctx->side, cudaStreamNonBlocking) != cudaSuccess ||
+    // The second stream carries small latency-bound kernels that run beside a long one on the caller's
+    // stream; the highest priority lets their blocks in as soon as a slot is free.
+    int prio_low = 0, prio_high = 0;
+    if (cudaDeviceGetStreamPriorityRange(&prio_low, &prio_high) != cudaSuccess) return bail(TENSAIR_ECUDA);
+    if (cudaStreamCreateWithPriority(&ctx->side, cudaStreamNonBlocking, prio_high) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_fork, cudaEventDisableTiming) != cudaSuccess ||
         cudaEventCreateWithFlags(&ctx->ev_join, cudaEventDisableTiming) != cudaSuccess)
         return bail(TENSAIR_ECUDA);
