@@ -61,6 +61,17 @@ __host__ __device__ inline uint32_t pair_count(uint32_t n, uint32_t w) {
     return (uint32_t)(2 * neighbours_before(n, w));
 }
 
+// fp32 -> fp64 without the conversion unit.  A finite float with sign s, exponent field e and fraction m, read
+// as the double with the same sign, exponent field e (not re-biased) and fraction m << 29, is f * 2^-896 exactly:
+// normal, subnormal and zero alike.  The bits come from one sign-extending shift of the float's word by 29 places
+// and one mask; the factor 2^896 goes, exactly, into the other operand of the product the value enters.
+// Infinities and NaNs are not preserved (they read as finite values): table rows must be finite.
+__device__ inline double widen_down(float f) {
+    const long long w = (long long)__float_as_int(f) << 29;
+    return __hiloint2double((int)(w >> 32) & (int)0x8FFFFFFFu, (int)w);
+}
+constexpr double kWidenUp = 0x1p896;   // widen_down(f) * kWidenUp == (double)f
+
 struct Shape {
     uint32_t V, d, d4, stride, w, k, K1;
 };

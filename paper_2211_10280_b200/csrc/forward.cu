@@ -40,9 +40,16 @@ __device__ inline void bulk_copy_g2s(void* dst_smem, const void* src_global, uin
 // Orders this thread's earlier shared-memory reads before later asynchronous writes to the same memory.
 __device__ inline void fence_generic_to_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
 
-__device__ inline double sigmoid(double x) { return 1.0 / (1.0 + exp(-x)); }
-// -log(sigmoid(x)) without overflow
-__device__ inline double neg_log_sigmoid(double x) { return (x < 0.0 ? -x : 0.0) + log1p(exp(-fabs(x))); }
+// sigmoid(x) and -log(sigmoid(y)) for y = x or -x from one exponential e = exp(-|x|):
+//   sigmoid(x) = 1 / (1 + e) for x >= 0, e / (1 + e) for x < 0;   -log(sigmoid(y)) = max(-y, 0) + log1p(e).
+struct SigmoidLoss {
+    double sig, softplus;   // sigmoid(x); log1p(exp(-|x|))
+};
+__device__ inline SigmoidLoss sigmoid_loss(double x) {
+    const double e = exp(-fabs(x));
+    const double r = 1.0 / (1.0 + e);
+    return SigmoidLoss{x < 0.0 ? e * r : r, log1p(e)};
+}
 
 constexpr int kFwdWarps = 2;       // warps per block
 
@@ -58,14 +65,16 @@ constexpr int kFwdWarps = 2;       // warps per block
 template <int NV, int CR>
 __global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, uint32_t stride4, uint32_t w,
-          uint32_t k, uint32_t chunk_rows, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
+          uint32_t k, uint32_t chunk_rows, uint32_t warp_stage4, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
           Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err,
           const uint32_t* __restrict__ owned, const uint32_t* __restrict__ n_owned) {
     if (*err) return;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    float4* stage = reinterpret_cast<float4*>(smem_raw) + (size_t)wib * chunk_rows * stride4;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)kFwdWarps * chunk_rows * stride4 * sizeof(float4)) + wib;
+    // warp_stage4 float4 per warp: chunk_rows rows plus padding, so that slice lane + 32 * i (i < NV) of every
+    // staged row is inside the buffer whatever the lane
+    float4* stage = reinterpret_cast<float4*>(smem_raw) + (size_t)wib * warp_stage4;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)kFwdWarps * warp_stage4 * sizeof(float4)) + wib;
     if (lane == 0) mbar_init(bar, 1);
     __syncwarp();
     uint32_t parity = 0;
@@ -89,7 +98,9 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
         for (int i = 0; i < NV; ++i) {
             const uint32_t e = lane + 32 * i;
             const float4 f = e < d4 ? __ldg(vin + e) : make_float4(0.f, 0.f, 0.f, 0.f);
-            v[i][0] = (double)f.x; v[i][1] = (double)f.y; v[i][2] = (double)f.z; v[i][3] = (double)f.w;
+            // the centre row carries the factor 2^896 that the staged rows lack (widen_down)
+            v[i][0] = (double)f.x * kWidenUp; v[i][1] = (double)f.y * kWidenUp;
+            v[i][2] = (double)f.z * kWidenUp; v[i][3] = (double)f.w * kWidenUp;
             acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0;
         }
         double loss = 0.0;
@@ -120,21 +131,44 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                 parity ^= 1;
 
                 // 1. partial dot products of the staged rows
+                // A chunk whose CR rows are all live takes loops without predicates, which the compiler is free to
+                // interleave: a lane whose slice lies past the row's end reads whatever the buffer holds there
+                // (finite once widened) against a centre value of zero.
+                const bool full = live == (CR == 32 ? 0xFFFFFFFFu : (1u << CR) - 1u);
                 double xp[CR];
+                if (full) {
 #pragma unroll
-                for (int j = 0; j < CR; ++j) {
-                    xp[j] = 0.0;
-                    if ((live >> j) & 1u) {
-                        const float4* __restrict__ u = stage + (size_t)j * stride4;
+                    for (int j = 0; j < CR; ++j) xp[j] = 0.0;
 #pragma unroll
-                        for (int i = 0; i < NV; ++i) {
-                            const uint32_t e = lane + 32 * i;
-                            if (e < d4) {
-                                const float4 f = u[e];
-                                xp[j] = fma((double)f.x, v[i][0], xp[j]);
-                                xp[j] = fma((double)f.y, v[i][1], xp[j]);
-                                xp[j] = fma((double)f.z, v[i][2], xp[j]);
-                                xp[j] = fma((double)f.w, v[i][3], xp[j]);
+                    for (int i = 0; i < NV; ++i) {
+                        float4 f[CR];
+#pragma unroll
+                        for (int j = 0; j < CR; ++j) f[j] = stage[(size_t)j * stride4 + lane + 32 * i];
+#pragma unroll
+                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].x), v[i][0], xp[j]);
+#pragma unroll
+                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].y), v[i][1], xp[j]);
+#pragma unroll
+                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].z), v[i][2], xp[j]);
+#pragma unroll
+                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].w), v[i][3], xp[j]);
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < CR; ++j) {
+                        xp[j] = 0.0;
+                        if ((live >> j) & 1u) {
+                            const float4* __restrict__ u = stage + (size_t)j * stride4;
+#pragma unroll
+                            for (int i = 0; i < NV; ++i) {
+                                const uint32_t e = lane + 32 * i;
+                                if (e < d4) {
+                                    const float4 f = u[e];
+                                    xp[j] = fma(widen_down(f.x), v[i][0], xp[j]);
+                                    xp[j] = fma(widen_down(f.y), v[i][1], xp[j]);
+                                    xp[j] = fma(widen_down(f.z), v[i][2], xp[j]);
+                                    xp[j] = fma(widen_down(f.w), v[i][3], xp[j]);
+                                }
                             }
                         }
                     }
@@ -159,26 +193,44 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                 double g = 0.0;
                 if ((live >> jr) & 1u) {
                     const bool positive = j0 + jr == 0;
-                    const double sig = sigmoid(x);
-                    g = positive ? sig - 1.0 : sig;
-                    if (writer) loss += neg_log_sigmoid(positive ? x : -x);
+                    const SigmoidLoss sl = sigmoid_loss(x);
+                    g = positive ? sl.sig - 1.0 : sl.sig;
+                    const double y = positive ? x : -x;   // the term is -log(sigmoid(y))
+                    if (writer) loss += (y < 0.0 ? -y : 0.0) + sl.softplus;
                 }
                 if (writer && jr < nr) rec[cbase + j0 + jr] = Rec{g, centre, 0u};
                 // 4. centre gradient: acc += g_j * u_j
+                if (full) {
+                    double gw[CR];
 #pragma unroll
-                for (int j = 0; j < CR; ++j) {
-                    const double gj = __shfl_sync(0xFFFFFFFFu, g, LPR * j);
-                    if ((live >> j) & 1u) {
-                        const float4* __restrict__ u = stage + (size_t)j * stride4;
+                    for (int j = 0; j < CR; ++j) gw[j] = __shfl_sync(0xFFFFFFFFu, g, LPR * j) * kWidenUp;   // exact: |g| <= 1
 #pragma unroll
-                        for (int i = 0; i < NV; ++i) {
-                            const uint32_t e = lane + 32 * i;
-                            if (e < d4) {
-                                const float4 f = u[e];
-                                acc[i][0] = fma(gj, (double)f.x, acc[i][0]);
-                                acc[i][1] = fma(gj, (double)f.y, acc[i][1]);
-                                acc[i][2] = fma(gj, (double)f.z, acc[i][2]);
-                                acc[i][3] = fma(gj, (double)f.w, acc[i][3]);
+                    for (int i = 0; i < NV; ++i) {
+#pragma unroll
+                        for (int j = 0; j < CR; ++j) {
+                            const float4 f = stage[(size_t)j * stride4 + lane + 32 * i];
+                            acc[i][0] = fma(gw[j], widen_down(f.x), acc[i][0]);
+                            acc[i][1] = fma(gw[j], widen_down(f.y), acc[i][1]);
+                            acc[i][2] = fma(gw[j], widen_down(f.z), acc[i][2]);
+                            acc[i][3] = fma(gw[j], widen_down(f.w), acc[i][3]);
+                        }
+                    }
+                } else {
+#pragma unroll
+                    for (int j = 0; j < CR; ++j) {
+                        const double gj = __shfl_sync(0xFFFFFFFFu, g, LPR * j) * kWidenUp;
+                        if ((live >> j) & 1u) {
+                            const float4* __restrict__ u = stage + (size_t)j * stride4;
+#pragma unroll
+                            for (int i = 0; i < NV; ++i) {
+                                const uint32_t e = lane + 32 * i;
+                                if (e < d4) {
+                                    const float4 f = u[e];
+                                    acc[i][0] = fma(gj, widen_down(f.x), acc[i][0]);
+                                    acc[i][1] = fma(gj, widen_down(f.y), acc[i][1]);
+                                    acc[i][2] = fma(gj, widen_down(f.z), acc[i][2]);
+                                    acc[i][3] = fma(gj, widen_down(f.w), acc[i][3]);
+                                }
                             }
                         }
                     }
@@ -221,8 +273,12 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     // rows staged per chunk: as many of the cr as fit the shared memory share of one block
     uint32_t chunk_rows = s.K1 < (uint32_t)cr ? s.K1 : (uint32_t)cr;
     const size_t budget = (size_t)216 * 1024 / blocks_per_sm - 1024;
-    while (chunk_rows > 1 && (size_t)kFwdWarps * chunk_rows * row + kFwdWarps * 8 > budget) --chunk_rows;
-    const size_t smem = (size_t)kFwdWarps * chunk_rows * row + kFwdWarps * 8;
+    // a warp's buffer ends with padding up to slice 32 * NV of its last row (see the kernel)
+    const uint32_t nv = s.d4 <= 32 ? 1 : s.d4 <= 64 ? 2 : s.d4 <= 96 ? 3 : s.d4 <= 128 ? 4 : 8;
+    const size_t pad = 32u * nv * 16 > row ? 32u * nv * 16 - row : 0;
+    while (chunk_rows > 1 && (size_t)kFwdWarps * (chunk_rows * row + pad) + kFwdWarps * 8 > budget) --chunk_rows;
+    const uint32_t warp_stage4 = (uint32_t)((chunk_rows * row + pad) / 16);
+    const size_t smem = (size_t)kFwdWarps * warp_stage4 * 16 + kFwdWarps * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
     const uint32_t stride4 = s.stride / 4;
     const float4* t4 = reinterpret_cast<const float4*>(table);
@@ -239,7 +295,8 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
             attr_set = true;                                                                                    \
         }                                                                                                       \
         k_forward<NV, CR><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,     \
-                                                                      chunk_rows, t4, rows, rec, gin_pos,      \
+                                                                      chunk_rows, warp_stage4, t4, rows, rec,  \
+                                                                      gin_pos,                                 \
                                                                       loss_pos, err, owned, n_owned);                  \
     } while (0)
 #define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)

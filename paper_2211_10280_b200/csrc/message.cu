@@ -267,7 +267,7 @@ __device__ inline void accumulate_segment(const Rec* __restrict__ terms, uint32_
                 const double g = __shfl_sync(0xFFFFFFFFu, mine.g, from);
                 const uint32_t centre = __shfl_sync(0xFFFFFFFFu, mine.centre, from);
                 const bool on = t0 + t < cnt;
-                coef[t] = on ? g : 0.0;
+                coef[t] = on ? g * kWidenUp : 0.0;   // exact (|g| <= 1); the factor the widened source lacks
                 src[t] = table + (size_t)(on ? centre : 0u) * stride4;
             }
             float4 x[kTermsInFlight][NV];
@@ -282,10 +282,10 @@ __device__ inline void accumulate_segment(const Rec* __restrict__ terms, uint32_
             for (int t = 0; t < kTermsInFlight; ++t)
 #pragma unroll
                 for (int i = 0; i < NV; ++i) {
-                    sum.a[i][0] = fma(coef[t], (double)x[t][i].x, sum.a[i][0]);
-                    sum.a[i][1] = fma(coef[t], (double)x[t][i].y, sum.a[i][1]);
-                    sum.a[i][2] = fma(coef[t], (double)x[t][i].z, sum.a[i][2]);
-                    sum.a[i][3] = fma(coef[t], (double)x[t][i].w, sum.a[i][3]);
+                    sum.a[i][0] = fma(coef[t], widen_down(x[t][i].x), sum.a[i][0]);
+                    sum.a[i][1] = fma(coef[t], widen_down(x[t][i].y), sum.a[i][1]);
+                    sum.a[i][2] = fma(coef[t], widen_down(x[t][i].z), sum.a[i][2]);
+                    sum.a[i][3] = fma(coef[t], widen_down(x[t][i].w), sum.a[i][3]);
                 }
         }
     }
