@@ -135,6 +135,67 @@ TENSAIR_API int tensair_workspace_bytes(const tensair_config* cfg, tensair_sizes
 TENSAIR_API int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const uint64_t* counts_host,
                  const float* init_in_host, const float* init_out_host, tensair_ctx** out);
 
+/*
+ * The same constructor for a job whose replicas are spread over several processes, one GPU each - the paper's
+ * own placement: data parallelism with one Model instance per worker (Section 2.2) that sends each gradient to
+ * every other instance (Section 3, "Stream Processing"; Algorithm 1, send_gradients).  The job has world_W
+ * replicas with global ids 0..world_W-1; this context holds the tables of cfg->W of them, global ids
+ * first_replica .. first_replica + cfg->W - 1.  Every process keeps the delivery schedule of the whole job (it
+ * is a function of the seed) and a pool slot for every message in flight of every replica, local or not, so a
+ * received message is applied from this GPU's own memory by the same kernels.  What differs from tensair_init:
+ *   - negative draws, delivery delays and routing use the replica's global id, so the job computes what one
+ *     process holding all world_W replicas computes, bit for bit (given the same batches per global replica);
+ *   - `replica` arguments of the calls that touch tables (train, apply, read/write embeddings, snapshots, pending,
+ *     delivery log) stay local indices 0..cfg->W-1; calls that name a message (tensair_read_message,
+ *     tensair_message_buffers, tensair_commit_message) and tensair_shadow_apply take global ids;
+ *   - per step, after the local tensair_train_batch calls: move every remote replica's message into the buffers
+ *     tensair_message_buffers names (any transport: an NCCL broadcast or all-gather straight into the pool),
+ *     tensair_commit_message each, then tensair_apply_messages for the local replicas and tensair_shadow_apply
+ *     for the others.
+ * tensair_workspace_bytes_sharded sizes the pool for world_W senders.  max_grad_buffer must be 1.
+ * world_W == cfg->W and first_replica == 0 is tensair_init.
+ */
+TENSAIR_API int tensair_workspace_bytes_sharded(const tensair_config* cfg, uint32_t world_W, tensair_sizes* out);
+TENSAIR_API int tensair_init_sharded(const tensair_config* cfg, const tensair_buffers* bufs, const uint64_t* counts_host,
+                                     const float* init_in_host, const float* init_out_host, uint32_t first_replica,
+                                     uint32_t world_W, tensair_ctx** out);
+
+/* Where the message of (global sender, batch_index) lives in this context's pool (device pointers). */
+typedef struct tensair_msg_view {
+    uint32_t* ids;            /* device, uint32[max_rows]: the message's row ids, ascending */
+    float* delta;             /* device, float[max_rows * row_stride]: its delta rows, row m at m * row_stride */
+    uint32_t max_rows;        /* capacity of both arrays in rows */
+    uint32_t row_stride;      /* floats between consecutive delta rows */
+    uint64_t ids_offset;      /* byte offsets of the two arrays in the pool buffer given at init */
+    uint64_t delta_offset;
+} tensair_msg_view;
+/*
+ * The "wire" of send_gradients (Algorithm 1) between processes.  Host-only, no synchronisation.
+ *   local sender   the slot holding the message tensair_train_batch built for batch_index (TENSAIR_ENOTFOUND if
+ *                  it is no longer held): the source of a send, valid once the stream has passed that call.
+ *   remote sender  the slot the message must be received into; TENSAIR_EPENDING while the slot's previous
+ *                  message still has local recipients (apply them first).  Write the first n_rows ids and
+ *                  n_rows * row_stride floats in stream order, then call tensair_commit_message.
+ */
+TENSAIR_API int tensair_message_buffers(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, tensair_msg_view* out);
+/* Row counts of a LOCAL replica's message (what a sender announces before its rows travel).  Synchronises. */
+TENSAIR_API int tensair_message_rows(tensair_ctx* ctx, uint32_t replica, uint64_t batch_index, uint32_t* n_rows,
+                                     uint32_t* n_in_rows);
+/*
+ * Files the received message of a REMOTE sender for this context's replicas (and books it for the others), as
+ * tensair_train_batch does for a local one: writes the slot's header, builds the message's bucket index
+ * (asynchronously on the context's stream, after whatever the stream already holds) and enters it in the delivery
+ * schedule.  n_in_rows = how many of the ids are input rows (< V).  TENSAIR_EPENDING as for tensair_train_batch.
+ */
+TENSAIR_API int tensair_commit_message(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, uint32_t n_rows,
+                                       uint32_t n_in_rows);
+/*
+ * Book-keeping of a REMOTE receiver: marks what is due for it at `step` (or everything, drain != 0) as applied,
+ * which the process holding that replica does for real.  Keeps slot reuse and the staleness of Section 3.1
+ * (which needs every replica's set of applied gradients) exact in every process.  Host-only.
+ */
+TENSAIR_API int tensair_shadow_apply(tensair_ctx* ctx, uint32_t receiver, uint64_t step, int drain, uint32_t* n_applied);
+
 /* Frees host state only; synchronises the stream first. */
 TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
 

@@ -42,6 +42,11 @@ class MsgInfo(C.Structure):
                 ("pool_offset", C.c_uint64)]
 
 
+class MsgView(C.Structure):
+    _fields_ = [("ids", C.c_void_p), ("delta", C.c_void_p), ("max_rows", C.c_uint32), ("row_stride", C.c_uint32),
+                ("ids_offset", C.c_uint64), ("delta_offset", C.c_uint64)]
+
+
 class Delivery(C.Structure):
     _fields_ = [("origin_step", C.c_uint64), ("sender", C.c_uint64), ("due_step", C.c_uint64),
                 ("applied_at", C.c_uint64), ("staleness", C.c_uint64)]
@@ -63,6 +68,12 @@ _P = C.POINTER
 SYMBOLS = {
     "tensair_workspace_bytes": (_int, [_P(Config), _P(Sizes)]),
     "tensair_init": (_int, [_P(Config), _P(Buffers), _vp, _vp, _vp, _P(_vp)]),
+    "tensair_workspace_bytes_sharded": (_int, [_P(Config), _u32, _P(Sizes)]),
+    "tensair_init_sharded": (_int, [_P(Config), _P(Buffers), _vp, _vp, _vp, _u32, _u32, _P(_vp)]),
+    "tensair_message_buffers": (_int, [_vp, _u32, _u64, _P(MsgView)]),
+    "tensair_message_rows": (_int, [_vp, _u32, _u64, _P(_u32), _P(_u32)]),
+    "tensair_commit_message": (_int, [_vp, _u32, _u64, _u32, _u32]),
+    "tensair_shadow_apply": (_int, [_vp, _u32, _u64, _int, _P(_u32)]),
     "tensair_destroy": (None, [_vp]),
     "tensair_train_batch": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
     "tensair_train_batch_host": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
@@ -138,6 +149,13 @@ def tensair_workspace_bytes(cfg: Config) -> Sizes:
     return out
 
 
+def tensair_workspace_bytes_sharded(cfg: Config, world_replicas: int) -> Sizes:
+    out = Sizes()
+    _check(lib().tensair_workspace_bytes_sharded(C.byref(cfg), world_replicas, C.byref(out)),
+           "tensair_workspace_bytes_sharded")
+    return out
+
+
 def tensair_build_alias_host(counts: Optional[np.ndarray], V: int):
     if counts is not None:
         counts = np.ascontiguousarray(counts, dtype=np.uint64)
@@ -210,7 +228,9 @@ class Context:
 
     def __init__(self, V, d, window, k, batch, W=1, lr=0.025, max_delay=0, seed=0, counts=None,
                  init_in=None, init_out=None, device=0, row_stride=0, stream=None, reduction=SUM,
-                 max_grad_buffer=1):
+                 max_grad_buffer=1, world_replicas=None, first_replica=0):
+        """W replicas live in this context.  world_replicas (default W) > W makes it one shard of a job whose
+        replicas are spread over several processes: see tensair_init_sharded."""
         import torch
 
         if not torch.cuda.is_available():
@@ -219,7 +239,9 @@ class Context:
         self.device = torch.device("cuda", device)
         self.cfg = Config(V=V, d=d, window=window, k=k, batch=batch, W=W, lr=lr, max_grad_buffer=max_grad_buffer,
                           max_delay=max_delay, row_stride=row_stride, seed=seed, device=device, reduction=reduction)
-        self.sizes = tensair_workspace_bytes(self.cfg)
+        self.world_replicas = W if world_replicas is None else world_replicas
+        self.first_replica = first_replica
+        self.sizes = tensair_workspace_bytes_sharded(self.cfg, self.world_replicas)
         with torch.cuda.device(self.device):
             self.stream = stream if stream is not None else torch.cuda.current_stream()
             self.tables = torch.empty(self.sizes.tables_bytes, dtype=torch.uint8, device=self.device)
@@ -237,8 +259,13 @@ class Context:
             init_out = np.ascontiguousarray(init_out, dtype=np.float32)
             assert init_out.shape == (V, d)
         h = C.c_void_p()
-        _check(lib().tensair_init(C.byref(self.cfg), C.byref(bufs), _np_ptr(counts), _np_ptr(init_in),
-                                  _np_ptr(init_out), C.byref(h)), "tensair_init")
+        if self.world_replicas == W and first_replica == 0:
+            _check(lib().tensair_init(C.byref(self.cfg), C.byref(bufs), _np_ptr(counts), _np_ptr(init_in),
+                                      _np_ptr(init_out), C.byref(h)), "tensair_init")
+        else:
+            _check(lib().tensair_init_sharded(C.byref(self.cfg), C.byref(bufs), _np_ptr(counts), _np_ptr(init_in),
+                                              _np_ptr(init_out), first_replica, self.world_replicas, C.byref(h)),
+                   "tensair_init_sharded")
         self._h = h
         self._keep = []
 
@@ -299,6 +326,33 @@ class Context:
     def tensair_drain(self) -> int:
         n = C.c_uint32(0)
         _check(lib().tensair_drain(self._h, C.byref(n)), "tensair_drain", self._h)
+        return int(n.value)
+
+    # -- messages between processes (sharded jobs)
+    def tensair_message_buffers(self, sender, batch_index):
+        """(ids, delta): int32 / float32 CUDA tensors that ARE the pool slot of the message of (global sender,
+        batch_index), at full capacity ([max_rows] and [max_rows * row_stride])."""
+        v = MsgView()
+        _check(lib().tensair_message_buffers(self._h, sender, batch_index, C.byref(v)), "tensair_message_buffers", self._h)
+        ids = self.pool[v.ids_offset:v.ids_offset + 4 * v.max_rows].view(self.torch.int32)
+        delta = self.pool[v.delta_offset:v.delta_offset + 4 * v.max_rows * v.row_stride].view(self.torch.float32)
+        assert ids.data_ptr() == v.ids and delta.data_ptr() == v.delta
+        return ids, delta
+
+    def tensair_message_rows(self, replica, batch_index):
+        """(rows, input rows) of a local replica's message.  Synchronises."""
+        n, n_in = C.c_uint32(0), C.c_uint32(0)
+        _check(lib().tensair_message_rows(self._h, replica, batch_index, C.byref(n), C.byref(n_in)),
+               "tensair_message_rows", self._h)
+        return int(n.value), int(n_in.value)
+
+    def tensair_commit_message(self, sender, batch_index, n_rows, n_in_rows):
+        _check(lib().tensair_commit_message(self._h, sender, batch_index, n_rows, n_in_rows), "tensair_commit_message",
+               self._h)
+
+    def tensair_shadow_apply(self, receiver, step, drain=False) -> int:
+        n = C.c_uint32(0)
+        _check(lib().tensair_shadow_apply(self._h, receiver, step, int(drain), C.byref(n)), "tensair_shadow_apply", self._h)
         return int(n.value)
 
     def tensair_update_sampler(self):

@@ -86,6 +86,31 @@ cudaError_t launch_bucket_index(const Launcher& L, const MsgHeader* hdr, const u
     return cudaGetLastError();
 }
 
+// The same index for a message whose rows arrived from another process: the row counts come from the host and
+// are written into the slot's header here, so that the message reads like one built in place.
+__global__ void __launch_bounds__(256)
+k_index_received(MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids, uint32_t* __restrict__ bucket_start,
+                 uint32_t n_buckets, uint32_t n_rows, uint32_t n_in_rows) {
+    const uint32_t b = blockIdx.x * blockDim.x + threadIdx.x;
+    if (b == 0) *hdr = MsgHeader{n_rows, n_in_rows, 0u, 0u};
+    if (b > n_buckets) return;
+    const uint64_t key = (uint64_t)b << kBucketShift;
+    uint32_t lo = 0, hi = n_rows;
+    while (lo < hi) {
+        const uint32_t mid = (lo + hi) >> 1;
+        if ((uint64_t)__ldg(ids + mid) < key) lo = mid + 1; else hi = mid;
+    }
+    bucket_start[b] = lo;
+}
+
+cudaError_t launch_index_received(const Launcher& L, MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
+                                  uint32_t V, uint32_t n_rows, uint32_t n_in_rows) {
+    const uint32_t nb = bucket_count(V);
+    Timed timed(L, K_BUCKET_INDEX);
+    k_index_received<<<(nb + 1 + 255) / 256, 256, 0, L.stream>>>(hdr, ids, bucket_start, nb, n_rows, n_in_rows);
+    return cudaGetLastError();
+}
+
 // Several messages, one pass.  A block owns an id range (a few buckets in a grid-stride loop); for each
 // message in order its warps take the message's rows in that range; a block-wide barrier separates the
 // messages, so a row touched by two of them gets its additions in message order.  Table rows are read

@@ -45,6 +45,10 @@ struct tensair_ctx {
     uint8_t* pool;
     uint8_t* scratch;
     tensair::Schedule* sched = nullptr;
+    // Replicas of the whole job and the global id of local replica 0.  One process holding every replica has
+    // world_W == cfg.W and first == 0; in a sharded job cfg.W counts the replicas whose tables live here.
+    uint32_t world_W = 0, first = 0;
+    uint32_t gid(uint32_t local) const { return first + local; }
     std::vector<uint32_t> buffered;        // per replica: gradient messages computed and not yet sent (maxGradBuffer > 1)
     uint32_t last_n = 0, last_pairs = 0;
     bool have_last = false;

@@ -160,6 +160,9 @@ cudaError_t launch_cosine_difference(const Launcher& L, const float* rows, const
 // bucket_start[b] = first row of the message with id >= b << kBucketShift, for b in [0, bucket_count(V)].
 cudaError_t launch_bucket_index(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
                                 uint32_t V);
+// The index of a message received from another process; also writes the slot's header from the given counts.
+cudaError_t launch_index_received(const Launcher& L, MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
+                                  uint32_t V, uint32_t n_rows, uint32_t n_in_rows);
 // Same, restricted to the message's input rows when input_rows_only != 0.
 cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
                               float* table, const Shape& s, int input_rows_only);

@@ -87,9 +87,10 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
     unsigned char* ws = g_scratch_address[c.device];
     auto in_ws = [ws](uint64_t off) { return ws + off; };
 
-    const int rc = ctx->sched->on_train(replica, batch_index);
+    const uint32_t me = ctx->gid(replica);   // the replica's id among all replicas of the job
+    const int rc = ctx->sched->on_train(me, batch_index);
     if (rc != TENSAIR_OK) return rc;
-    const uint32_t slot = ctx->sched->slot_of(replica, batch_index);
+    const uint32_t slot = ctx->sched->slot_of(me, batch_index);
     const uint32_t pairs = n_tokens >= 2 ? pair_count(n_tokens, c.window) : 0;
     const uint32_t n_items = pairs ? 2 * n_tokens + pairs * (c.k + 1) : 0;
     uint32_t* err = ctx->at<uint32_t>(cv.err);
@@ -105,8 +106,8 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
 
     // the array keeps what the previous call left: the list counters must start at zero
     TENSAIR_CUDA(ctx, cudaMemsetAsync(long_counters, 0, 8, ctx->stream));
-    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tokens_dev, n_tokens, c.V, err, nullptr, nullptr, nullptr, c.W, replica, c.seed));
-    TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tokens_dev, n_tokens, ctx->shape, replica, (uint32_t)batch_index, c.seed,
+    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tokens_dev, n_tokens, c.V, err, nullptr, nullptr, nullptr, ctx->world_W, me, c.seed));
+    TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tokens_dev, n_tokens, ctx->shape, me, (uint32_t)batch_index, c.seed,
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows), items_a,
                                      ctx->at<unsigned long long>(cv.counts), err, nullptr));
     if (n_items) {

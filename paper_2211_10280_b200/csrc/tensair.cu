@@ -120,15 +120,16 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
     // maxGradBuffer = 1: the batch's message is built in its send slot and filed at once.  Otherwise it is built
     // in a buffer slot of the replica, and after every m-th batch the m buffered messages are summed into a send slot.
     const uint32_t m_buf = c.max_grad_buffer;
-    const uint32_t send_slot = ctx->sched->slot_of(replica, batch_index);
+    const uint32_t me = ctx->gid(replica);   // the replica's id among all replicas of the job
+    const uint32_t send_slot = ctx->sched->slot_of(me, batch_index);
     const bool sends = m_buf == 1 || ctx->buffered[replica] + 1 == m_buf;
     if (sends && m_buf > 1 && ctx->sched->slot_busy(send_slot)) return TENSAIR_EPENDING;
     if (m_buf == 1) {
-        const int rc = ctx->sched->on_train(replica, batch_index);
+        const int rc = ctx->sched->on_train(me, batch_index);
         if (rc != TENSAIR_OK) return rc;
     }
     const uint32_t slot = m_buf == 1 ? send_slot
-                                     : c.W * (c.max_delay + 1) + replica * m_buf + ctx->buffered[replica];
+                                     : ctx->world_W * (c.max_delay + 1) + replica * m_buf + ctx->buffered[replica];
     const uint32_t pairs = n >= 2 ? pair_count(n, c.window) : 0;
     const uint32_t contrib = pairs * (c.k + 1);
     const uint32_t n_items = pairs ? 2 * n + contrib : 0;
@@ -141,8 +142,8 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
     uint8_t* owner = routed ? ctx->at<uint8_t>(cv.owner) : nullptr;
     uint32_t* owned = routed ? ctx->at<uint32_t>(cv.owned) : nullptr;
     uint32_t* n_owned = routed ? ctx->at<uint32_t>(cv.n_owned) : nullptr;
-    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err, owner, owned, n_owned, c.W, replica, c.seed));
-    TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tok_dev, n, ctx->shape, routed ? 0u : replica, (uint32_t)batch_index, c.seed,
+    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err, owner, owned, n_owned, ctx->world_W, me, c.seed));
+    TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tok_dev, n, ctx->shape, routed ? 0u : me, (uint32_t)batch_index, c.seed,
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows),
                                      ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err, owner));
     if (n_items) {
@@ -202,7 +203,7 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
             MergeInputs in;
             in.count = m_buf;
             for (uint32_t b = 0; b < m_buf; ++b) {
-                const uint32_t bs = c.W * (c.max_delay + 1) + replica * m_buf + b;
+                const uint32_t bs = ctx->world_W * (c.max_delay + 1) + replica * m_buf + b;
                 in.ids[b] = ctx->slot_ids(bs);
                 in.delta[b] = ctx->slot_delta(bs);
                 in.buckets[b] = ctx->slot_buckets(bs);
@@ -210,7 +211,7 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
             TENSAIR_CUDA(ctx, launch_merge(ctx->L, in, ctx->slot_hdr(send_slot), ctx->slot_buckets(send_slot),
                                            ctx->slot_ids(send_slot), ctx->slot_delta(send_slot),
                                            ctx->at<uint32_t>(cv.merge_counts), ctx->shape));
-            const int rc = ctx->sched->on_train(replica, batch_index);
+            const int rc = ctx->sched->on_train(me, batch_index);
             if (rc != TENSAIR_OK) return rc;
             ctx->buffered[replica] = 0;
         }
@@ -278,14 +279,19 @@ int copy_rows(tensair_ctx* ctx, uint32_t replica, int which, uint32_t row0, uint
 extern "C" {
 
 int tensair_workspace_bytes(const tensair_config* cfg, tensair_sizes* out) {
+    return tensair_workspace_bytes_sharded(cfg, cfg ? cfg->W : 0, out);
+}
+
+int tensair_workspace_bytes_sharded(const tensair_config* cfg, uint32_t world_W, tensair_sizes* out) {
     const int rc = validate_config(cfg);
-    if (rc != TENSAIR_OK || !out) return TENSAIR_EINVAL;
+    if (rc != TENSAIR_OK || !out || world_W < cfg->W || world_W > 256) return TENSAIR_EINVAL;
     Carve cv;
     carve(*cfg, cv);
     out->row_stride = cv.stride;
     out->tables_bytes = (uint64_t)cfg->W * 2 * cfg->V * cv.stride * 4;
-    // one slot per message in flight, plus (maxGradBuffer > 1) the buffered messages of every replica
-    out->pool_bytes = ((uint64_t)cfg->W * (cfg->max_delay + 1) +
+    // one slot per message in flight of every replica of the job, plus (maxGradBuffer > 1) the buffered messages
+    // of the replicas that live here
+    out->pool_bytes = ((uint64_t)world_W * (cfg->max_delay + 1) +
                        (cfg->max_grad_buffer > 1 ? (uint64_t)cfg->W * cfg->max_grad_buffer : 0)) * cv.slot_bytes;
     out->scratch_bytes = cv.total;
     out->max_pairs = cv.max_pairs;
@@ -296,9 +302,16 @@ int tensair_workspace_bytes(const tensair_config* cfg, tensair_sizes* out) {
 
 int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const uint64_t* counts_host,
                  const float* init_in_host, const float* init_out_host, tensair_ctx** out) {
+    return tensair_init_sharded(cfg, bufs, counts_host, init_in_host, init_out_host, 0, cfg ? cfg->W : 0, out);
+}
+
+int tensair_init_sharded(const tensair_config* cfg, const tensair_buffers* bufs, const uint64_t* counts_host,
+                         const float* init_in_host, const float* init_out_host, uint32_t first_replica,
+                         uint32_t world_W, tensair_ctx** out) {
     tensair_sizes sz;
-    if (!out || !bufs || tensair_workspace_bytes(cfg, &sz) != TENSAIR_OK) return TENSAIR_EINVAL;
+    if (!out || !bufs || tensair_workspace_bytes_sharded(cfg, world_W, &sz) != TENSAIR_OK) return TENSAIR_EINVAL;
     *out = nullptr;
+    if ((uint64_t)first_replica + cfg->W > world_W) return TENSAIR_EINVAL;
     if (!bufs->tables || !bufs->pool || !bufs->scratch) return TENSAIR_EINVAL;
     if (((uintptr_t)bufs->tables | (uintptr_t)bufs->pool | (uintptr_t)bufs->scratch) & 255) return TENSAIR_EINVAL;
     if (bufs->tables_bytes < sz.tables_bytes || bufs->pool_bytes < sz.pool_bytes || bufs->scratch_bytes < sz.scratch_bytes)
@@ -310,6 +323,8 @@ int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const u
     tensair_ctx* ctx = new (std::nothrow) tensair_ctx();
     if (!ctx) return TENSAIR_ENOMEM;
     ctx->cfg = *cfg;
+    ctx->world_W = world_W;
+    ctx->first = first_replica;
     carve(*cfg, ctx->cv);
     ctx->shape = Shape{cfg->V, cfg->d, cfg->d / 4, ctx->cv.stride, cfg->window, cfg->k, cfg->k + 1};
     ctx->stream = (cudaStream_t)bufs->stream;
@@ -330,7 +345,7 @@ int tensair_init(const tensair_config* cfg, const tensair_buffers* bufs, const u
     if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount, &ctx->prof};
     if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
-    ctx->sched = new Schedule(cfg->W, cfg->max_delay, cfg->seed);
+    ctx->sched = new Schedule(world_W, cfg->max_delay, cfg->seed);
     ctx->buffered.assign(cfg->W, 0);
     // The second stream carries small latency-bound kernels that run beside a long one on the caller's
     // stream; the highest priority lets their blocks in as soon as a slot is free.
@@ -427,7 +442,7 @@ int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint64_t step, ui
     if (!ctx || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return TENSAIR_ECUDA;
-    const std::vector<Due> due = ctx->sched->take_due(replica, step, false);
+    const std::vector<Due> due = ctx->sched->take_due(ctx->gid(replica), step, false);
     if (n_applied) *n_applied = (uint32_t)due.size();
     return apply_due(ctx, replica, due);
 }
@@ -438,12 +453,67 @@ int tensair_drain(tensair_ctx* ctx, uint32_t* n_applied) {
     if (!guard.ok) return TENSAIR_ECUDA;
     uint32_t total = 0;
     for (uint32_t r = 0; r < ctx->cfg.W; ++r) {
-        const std::vector<Due> due = ctx->sched->take_due(r, 0, true);
+        const std::vector<Due> due = ctx->sched->take_due(ctx->gid(r), 0, true);
         total += (uint32_t)due.size();
         const int rc = apply_due(ctx, r, due);
         if (rc != TENSAIR_OK) return rc;
     }
+    // the replicas held by other processes drain there; only their bookkeeping is kept here
+    for (uint32_t g = 0; g < ctx->world_W; ++g)
+        if (g < ctx->first || g >= ctx->first + ctx->cfg.W) ctx->sched->take_due(g, 0, true);
     if (n_applied) *n_applied = total;
+    return TENSAIR_OK;
+}
+
+int tensair_message_buffers(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, tensair_msg_view* out) {
+    if (!ctx || !out || sender >= ctx->world_W || batch_index >= (1ull << 32)) return TENSAIR_EINVAL;
+    const uint32_t slot = ctx->sched->slot_of(sender, batch_index);
+    const bool local = sender >= ctx->first && sender < ctx->first + ctx->cfg.W;
+    // a local message must be the one held; a remote one is about to be received, so its slot must be free
+    if (local ? !ctx->sched->slot_holds(slot, batch_index) : ctx->sched->slot_busy(slot))
+        return local ? TENSAIR_ENOTFOUND : TENSAIR_EPENDING;
+    out->ids = ctx->slot_ids(slot);
+    out->delta = ctx->slot_delta(slot);
+    out->max_rows = ctx->cv.max_rows;
+    out->row_stride = ctx->cv.stride;
+    out->ids_offset = (uint64_t)slot * ctx->cv.slot_bytes + ctx->cv.ids_off;
+    out->delta_offset = (uint64_t)slot * ctx->cv.slot_bytes + ctx->cv.delta_off;
+    return TENSAIR_OK;
+}
+
+int tensair_message_rows(tensair_ctx* ctx, uint32_t replica, uint64_t batch_index, uint32_t* n_rows, uint32_t* n_in_rows) {
+    if (!ctx || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const uint32_t slot = ctx->sched->slot_of(ctx->gid(replica), batch_index);
+    if (!ctx->sched->slot_holds(slot, batch_index)) return TENSAIR_ENOTFOUND;
+    TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->hdr, ctx->slot_hdr(slot), sizeof(MsgHeader), cudaMemcpyDeviceToHost, ctx->stream));
+    const int st = collect(ctx);
+    if (st != TENSAIR_OK) return st;
+    if (n_rows) *n_rows = ctx->stage->hdr.n_rows;
+    if (n_in_rows) *n_in_rows = ctx->stage->hdr.n_in_rows;
+    return TENSAIR_OK;
+}
+
+int tensair_commit_message(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, uint32_t n_rows, uint32_t n_in_rows) {
+    if (!ctx || sender >= ctx->world_W || batch_index >= (1ull << 32) || n_in_rows > n_rows || n_rows > ctx->cv.max_rows)
+        return TENSAIR_EINVAL;
+    if (sender >= ctx->first && sender < ctx->first + ctx->cfg.W) return TENSAIR_EINVAL;   // local messages file themselves
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const int rc = ctx->sched->on_train(sender, batch_index);
+    if (rc != TENSAIR_OK) return rc;
+    const uint32_t slot = ctx->sched->slot_of(sender, batch_index);
+    TENSAIR_CUDA(ctx, launch_index_received(ctx->L, ctx->slot_hdr(slot), ctx->slot_ids(slot), ctx->slot_buckets(slot),
+                                            ctx->cfg.V, n_rows, n_in_rows));
+    return TENSAIR_OK;
+}
+
+int tensair_shadow_apply(tensair_ctx* ctx, uint32_t receiver, uint64_t step, int drain, uint32_t* n_applied) {
+    if (!ctx || receiver >= ctx->world_W) return TENSAIR_EINVAL;
+    if (receiver >= ctx->first && receiver < ctx->first + ctx->cfg.W) return TENSAIR_EINVAL;   // that one is applied for real
+    const std::vector<Due> due = ctx->sched->take_due(receiver, step, drain != 0);
+    if (n_applied) *n_applied = (uint32_t)due.size();
     return TENSAIR_OK;
 }
 
@@ -550,7 +620,7 @@ int tensair_read_scalars(tensair_ctx* ctx, double* host_g) {
 
 int tensair_read_message(tensair_ctx* ctx, uint32_t replica, uint64_t batch_index, uint32_t* n_rows,
                          uint32_t* host_ids, float* host_delta) {
-    if (!ctx || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
+    if (!ctx || replica >= ctx->world_W) return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return TENSAIR_ECUDA;
     const uint32_t slot = ctx->sched->slot_of(replica, batch_index);
@@ -586,7 +656,7 @@ int tensair_read_sampler(tensair_ctx* ctx, uint32_t* thresh, uint32_t* alias, ui
 
 int tensair_read_delivery_log(tensair_ctx* ctx, uint32_t replica, uint64_t max_records, tensair_delivery* out, uint64_t* n) {
     if (!ctx || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
-    const std::vector<tensair_delivery>& lg = ctx->sched->log(replica);
+    const std::vector<tensair_delivery>& lg = ctx->sched->log(ctx->gid(replica));
     if (n) *n = lg.size();
     for (uint64_t i = 0; i < lg.size() && i < max_records && out; ++i) out[i] = lg[i];
     return TENSAIR_OK;
@@ -594,7 +664,7 @@ int tensair_read_delivery_log(tensair_ctx* ctx, uint32_t replica, uint64_t max_r
 
 int tensair_pending(tensair_ctx* ctx, uint32_t replica, uint64_t* n) {
     if (!ctx || !n || replica >= ctx->cfg.W) return TENSAIR_EINVAL;
-    *n = ctx->sched->pending(replica);
+    *n = ctx->sched->pending(ctx->gid(replica));
     return TENSAIR_OK;
 }
 
