@@ -151,6 +151,111 @@ def rank_streams(wl: synth.Workload, rank: int, batches: int):
 
 
 # ------------------------------------------------------------------------------------------------
+def run_sharded(args):
+    """`--sharded`: the workload's W replicas spread over the ranks (W / N per GPU), every message broadcast into
+    every rank's pool over NCCL (paper_2211_10280_b200/exchange.py).  The job computes what the one-GPU job
+    computes, so the total work is fixed as N grows ("strong")."""
+    import torch
+    import torch.distributed as dist
+
+    from paper_2211_10280_b200 import binding as B
+    from paper_2211_10280_b200.exchange import ShardedReplicas
+
+    rank = int(os.environ.get("RANK", "0"))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
+    local = int(os.environ.get("LOCAL_RANK", "0"))
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py needs a CUDA device: the SGNS path has no CPU implementation")
+    torch.cuda.set_device(local)
+    if world > 1:
+        dist.init_process_group("nccl", device_id=torch.device("cuda", local))
+    wl = pick_workload(args.workload, args.override)
+    if wl.W % world or wl.routed or wl.max_grad_buffer != 1:
+        raise SystemExit(f"--sharded needs a workload whose {wl.W} replicas divide over {world} ranks, unrouted, maxGradBuffer 1")
+    Wl = wl.W // world
+    K, Wm = args.steps, max(args.warmup, 3)
+    total_steps = 2 * (Wm + K)
+    toks_all, counts = rank_streams(wl, 0, total_steps)          # the one-GPU job's streams; this rank takes its replicas'
+    toks_np = np.ascontiguousarray(toks_all[:, rank * Wl:(rank + 1) * Wl])
+    ctx = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=Wl, lr=wl.lr, max_delay=wl.max_delay,
+                    seed=wl.seed, counts=counts, device=local, reduction=wl.reduction, world_replicas=wl.W,
+                    first_replica=rank * Wl)
+    grp = ShardedReplicas(ctx, rank, world, Wl, dist if world > 1 else None, count_device="cuda")
+    toks_dev = torch.from_numpy(toks_np).cuda()
+    toks_pin = torch.from_numpy(toks_np).pin_memory()
+
+    def step(t, host=False):
+        if wl.drift_every and t and t % wl.drift_every == 0:
+            ctx.tensair_update_sampler()
+        for r in range(Wl):
+            if host:
+                ctx.tensair_train_batch_host(r, toks_pin[t, r], t, want_loss=True)
+            else:
+                ctx.tensair_train_batch(r, toks_dev[t, r], t)
+        grp.exchange(t)
+        grp.apply(t)
+
+    def barrier():
+        torch.cuda.synchronize()
+        if world > 1:
+            dist.barrier()
+        torch.cuda.synchronize()
+
+    def timed(first, host):
+        ev0, ev1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        barrier()
+        wall0 = time.time()
+        ev0.record()
+        for t in range(first, first + K):
+            step(t, host=host)
+        ev1.record()
+        barrier()
+        ms = ev0.elapsed_time(ev1)
+        return (max_over_ranks(ms, dist, "cuda") if world > 1 else ms), wall0, time.time()
+
+    uuid = str(torch.cuda.get_device_properties(local).uuid)
+    sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
+    t = 0
+    for _ in range(Wm):
+        step(t)
+        t += 1
+    sampler.start()
+    time.sleep(0.3)
+    launches0, sent0 = ctx.tensair_kernel_launches(), grp.bytes_sent
+    ms_dev, wall0, wall1 = timed(t, host=False)
+    launches, sent = ctx.tensair_kernel_launches() - launches0, grp.bytes_sent - sent0
+    sampler.stop()
+    t += K
+    for _ in range(Wm):
+        step(t, host=True)
+        t += 1
+    ms_e2e, _, _ = timed(t, host=True)
+    if ctx.tensair_sync() != B.OK:
+        raise SystemExit("the device reported a bad token during the benchmark")
+    P = wl.pairs_per_batch
+    out = {
+        "metric": METRIC, "value": wl.W * P * K / (ms_dev * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
+        "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+        "dtype": "f64", "data": "synthetic",
+        "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
+                   "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
+                   "pairs_per_batch": P, "storage": "f32",
+                   "l2": "inputs larger than L2 (tables %.1f GB per GPU)" % (ctx.sizes.tables_bytes / 1e9),
+                   "parallelism": f"{Wl} of {wl.W} replicas per GPU, every message broadcast into every GPU's pool"},
+        "e2e": {"value": wl.W * P * K / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e / K,
+                "h2d_bytes_per_step": Wl * wl.batch * 4, "d2h_bytes_per_step": Wl * (8 + 16 + 4)},
+        "gpu_launches": int(launches),
+        "exchange": {"bytes_sent_per_step_per_gpu": int(sent / K), "transport": "NCCL broadcast per message" if world > 1 else "none (one rank)"},
+        "clocks": sampler.summary(wall0, wall1),
+    }
+    ctx.close()
+    if world > 1:
+        dist.barrier()
+        dist.destroy_process_group()
+    if rank == 0:
+        print(json.dumps(out))
+
+
 def run_ours(args):
     import torch
     import torch.distributed as dist
@@ -499,9 +604,13 @@ def main():
     ap.add_argument("--log-applies", default="", help="write one JSON line per apply call (bytes to move) to this file")
     ap.add_argument("--sweep", action="store_true", help="run the 32-point throughput sweep instead (one line per point)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--sharded", action="store_true",
+                    help="spread the workload's replicas over the ranks and exchange their messages (strong scaling)")
     args = ap.parse_args()
     if args.sweep:
         run_sweep(args)
+    elif args.sharded and args.impl == "ours":
+        run_sharded(args)
     elif args.impl == "reference":
         run_reference(args)
     else:

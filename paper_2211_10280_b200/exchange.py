@@ -37,11 +37,11 @@ class ShardedReplicas:
         this process's pool and files them.  Collective: every process calls it for every step."""
         import torch
 
-        mine = [self.port.tensair_message_rows(r, step) for r in range(self.local)]
         if self.world_size == 1:
             return
         if self.dist is None:
             raise RuntimeError("exchange() between processes needs torch.distributed")
+        mine = [self.port.tensair_message_rows(r, step) for r in range(self.local)]
         counts = torch.tensor(mine, dtype=torch.int64, device=self.count_device).reshape(self.local, 2)
         gathered = [torch.empty_like(counts) for _ in range(self.world_size)]
         self.dist.all_gather(gathered, counts, group=self.group)
