@@ -304,8 +304,11 @@ def run_ours(args):
                 n_rows[(i, t)] = (inf.n_rows, inf.n_in_rows)
             if info or args.log_applies:
                 msg_ids[(i, t)] = ctx.tensair_read_message_ids(i, t)
-        for j in range(wl.W):
-            ctx.tensair_apply_messages(j, t)
+        if args.apply_per_replica:
+            for j in range(wl.W):
+                ctx.tensair_apply_messages(j, t)
+        else:
+            ctx.tensair_apply_step(t)                         # all replicas' due messages in one pass
 
     def barrier():
         torch.cuda.synchronize()
@@ -409,6 +412,24 @@ def run_ours(args):
     }
     if fused_bytes:
         algo["apply_fused"] = float(np.mean(fused_bytes))
+    # one pass for all receivers of a step: every delta row of the distinct messages read once, and per receiver
+    # every row of the union of its messages' id sets read and written once
+    per_step = {}
+    for (j, at), members in groups.items():
+        per_step.setdefault(at, {})[j] = members
+    step_pass_bytes, step_pass_log = [], []
+    for at, per_j in sorted(per_step.items()):
+        distinct = sorted({m for ms in per_j.values() for m in ms})
+        if sum(len(ms) for ms in per_j.values()) < 2 or any(msg_ids.get(m) is None for m in distinct):
+            continue
+        delta_rows = sum(msg_ids[m].size for m in distinct)
+        union_rows = sum(np.unique(np.concatenate([msg_ids[m] for m in ms])).size for ms in per_j.values())
+        step_pass_bytes.append(delta_rows * (row + 4) + union_rows * 2 * row)
+        step_pass_log.append({"step": at, "messages": len(distinct), "deliveries": sum(len(ms) for ms in per_j.values()),
+                              "kernel": "k_apply_step", "delta_rows": delta_rows, "union_rows": union_rows,
+                              "algorithmic_bytes": step_pass_bytes[-1]})
+    if step_pass_bytes:
+        algo["apply_step"] = float(np.mean(step_pass_bytes))
     if args.log_applies:
         # every apply call of the run in call order, with the bytes its launch has to move (for matching ncu captures)
         calls = {}
@@ -416,7 +437,11 @@ def run_ours(args):
             for origin, snd, due, at, _ in ctx.tensair_read_delivery_log(j).tolist():
                 calls.setdefault((at, j), []).append((snd, origin))
         with open(args.log_applies, "w") as fh:
-            for (at, j), members in sorted(calls.items()):
+            if not args.apply_per_replica:
+                # note: only the steps of the per-kernel pass (the message ids of earlier steps are not kept)
+                for rec in step_pass_log:
+                    fh.write(json.dumps(rec) + "\n")
+            for (at, j), members in sorted(calls.items()) if args.apply_per_replica else []:
                 ids = [msg_ids.get(m) for m in members]
                 if any(x is None for x in ids):
                     continue
@@ -604,6 +629,8 @@ def main():
     ap.add_argument("--log-applies", default="", help="write one JSON line per apply call (bytes to move) to this file")
     ap.add_argument("--sweep", action="store_true", help="run the 32-point throughput sweep instead (one line per point)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--apply-per-replica", action="store_true",
+                    help="apply the due messages with one tensair_apply_messages call per replica instead of tensair_apply_step")
     ap.add_argument("--sharded", action="store_true",
                     help="spread the workload's replicas over the ranks and exchange their messages (strong scaling)")
     args = ap.parse_args()

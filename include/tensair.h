@@ -284,6 +284,16 @@ TENSAIR_API int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, c
  */
 TENSAIR_API int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint64_t step, uint32_t* n_applied);
 
+/*
+ * tensair_apply_messages(replica, step) for every replica of the context, as one pass over their tables: a
+ * message due for several of them at this step is read from memory once and added to each (the replicas share
+ * one GPU's memory, so the gradient application that every Model instance repeats - Section 4.2 notes it does
+ * not shrink with the number of instances - shares its reads here).  Per replica the messages are applied in
+ * the same (origin step, sender) order, so tables and delivery logs are bit-identical to the per-replica calls.
+ * n_applied: host, nullable: deliveries made, summed over the replicas.
+ */
+TENSAIR_API int tensair_apply_step(tensair_ctx* ctx, uint64_t step, uint32_t* n_applied);
+
 /* End of a run: delivers everything still pending, per receiver in (due step, origin step, sender)
  * order, so that all replicas have applied the same gradients.  n_applied: host, nullable. */
 TENSAIR_API int tensair_drain(tensair_ctx* ctx, uint32_t* n_applied);

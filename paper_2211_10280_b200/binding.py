@@ -81,6 +81,7 @@ SYMBOLS = {
     "tensair_route": (_int, [_u64, _u32, _u32, _vp]),
     "tensair_train_batch_static": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
     "tensair_apply_messages": (_int, [_vp, _u32, _u64, _P(_u32)]),
+    "tensair_apply_step": (_int, [_vp, _u64, _P(_u32)]),
     "tensair_drain": (_int, [_vp, _P(_u32)]),
     "tensair_update_sampler": (_int, [_vp]),
     "tensair_sync": (_int, [_vp]),
@@ -321,6 +322,12 @@ class Context:
     def tensair_apply_messages(self, replica, step) -> int:
         n = C.c_uint32(0)
         _check(lib().tensair_apply_messages(self._h, replica, step, C.byref(n)), "tensair_apply_messages", self._h)
+        return int(n.value)
+
+    def tensair_apply_step(self, step) -> int:
+        """tensair_apply_messages for every replica of the context in one pass; returns the deliveries made."""
+        n = C.c_uint32(0)
+        _check(lib().tensair_apply_step(self._h, step, C.byref(n)), "tensair_apply_step", self._h)
         return int(n.value)
 
     def tensair_drain(self) -> int:

@@ -169,6 +169,104 @@ cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float*
     return cudaGetLastError();
 }
 
+// All receivers, one pass, no ordering barriers.  A message carries the set of receivers it is due for.  A block
+// owns a bucket (16 consecutive row ids).  It first notes, per message, which of the 16 ids the message holds
+// (a 16-bit mask; ids ascend, so the row of id j is the bucket's first row plus the number of mask bits below j).
+// Then a warp takes one (id, receiver) pair at a time: it fetches the receiver's table row once, adds the delta
+// rows of the messages that hold the id and are due for that receiver, in message order, and stores the row
+// once.  The sums are the ones a message-after-message application makes (fp32 additions in the same order);
+// a delta row needed by several receivers comes from memory once and from the cache afterwards.
+static_assert(kBucketShift == 4, "the step kernel maps a bucket onto half a warp");
+constexpr int kStepThreads = 128;
+template <int NV>
+__global__ void __launch_bounds__(kStepThreads)
+k_apply_step(StepMessages f, uint32_t n_receivers, float4* __restrict__ tables, size_t replica4, uint32_t d4,
+             uint32_t stride4, uint32_t n_buckets) {
+    // two copies, used by alternate buckets: a warp may note the next bucket while another still works on this one
+    __shared__ uint32_t first_row[2][kMaxStepMessages];
+    __shared__ uint32_t held[2][kMaxStepMessages];
+    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
+    constexpr uint32_t kWarps = kStepThreads / 32;
+    const uint32_t half = lane >> 4, j_mine = lane & 15;
+    const uint32_t half_mask = 0xFFFFu << (16 * half);
+    uint32_t turn = 0;
+    for (uint32_t b = blockIdx.x; b < n_buckets; b += gridDim.x, turn ^= 1u) {
+        // which ids of the bucket each message holds: half a warp per message
+        for (uint32_t k0 = 2 * wid; k0 < f.count; k0 += 2 * kWarps) {
+            const uint32_t k = k0 + half;
+            uint32_t beg = 0, bit = 0;
+            if (k < f.count) {
+                beg = __ldg(f.buckets[k] + b);
+                const uint32_t end = __ldg(f.buckets[k] + b + 1);
+                if (beg + j_mine < end) bit = 1u << (__ldg(f.ids[k] + beg + j_mine) & 15u);
+            }
+            const uint32_t mask = __reduce_or_sync(half_mask, bit);
+            if (k < f.count && j_mine == 0) { first_row[turn][k] = beg; held[turn][k] = mask; }
+        }
+        __syncthreads();
+        const uint32_t set_mine = lane < f.count ? f.receivers[lane] : 0u;
+        const uint32_t held_mine = lane < f.count ? held[turn][lane] : 0u;
+        for (uint32_t task = wid; task < 16u * n_receivers; task += kWarps) {
+            const uint32_t j = task / n_receivers, rcv = task - j * n_receivers;
+            // messages (lane = message index, so in message order) that hold id j and are due for this receiver
+            uint32_t todo = __ballot_sync(0xFFFFFFFFu, ((held_mine >> j) & 1u) && ((set_mine >> rcv) & 1u));
+            if (!todo) continue;
+            const uint32_t id = (b << kBucketShift) + j;
+            float4* dst = tables + (size_t)rcv * replica4 + (size_t)id * stride4;
+            float4 r[NV], a[NV];
+            uint32_t k = (uint32_t)__ffs((int)todo) - 1u;
+            todo &= todo - 1;
+            const float4* __restrict__ src = reinterpret_cast<const float4*>(f.delta[k]) +
+                (size_t)(first_row[turn][k] + __popc(held[turn][k] & ((1u << j) - 1u))) * stride4;
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const uint32_t e = lane + 32 * i;
+                if (e < d4) {
+                    r[i] = __ldcg(dst + e);
+                    a[i] = __ldg(src + e);
+                }
+            }
+            for (;;) {
+#pragma unroll
+                for (int i = 0; i < NV; ++i) { r[i].x += a[i].x; r[i].y += a[i].y; r[i].z += a[i].z; r[i].w += a[i].w; }
+                if (!todo) break;
+                k = (uint32_t)__ffs((int)todo) - 1u;
+                todo &= todo - 1;
+                src = reinterpret_cast<const float4*>(f.delta[k]) +
+                      (size_t)(first_row[turn][k] + __popc(held[turn][k] & ((1u << j) - 1u))) * stride4;
+#pragma unroll
+                for (int i = 0; i < NV; ++i) {
+                    const uint32_t e = lane + 32 * i;
+                    if (e < d4) a[i] = __ldg(src + e);
+                }
+            }
+#pragma unroll
+            for (int i = 0; i < NV; ++i) {
+                const uint32_t e = lane + 32 * i;
+                if (e < d4) dst[e] = r[i];
+            }
+        }
+    }
+}
+
+cudaError_t launch_apply_step(const Launcher& L, const StepMessages& f, uint32_t n_receivers, float* tables,
+                              size_t replica_floats, const Shape& s) {
+    const uint32_t stride4 = s.stride / 4;
+    float4* t4 = reinterpret_cast<float4*>(tables);
+    const uint32_t nb = bucket_count(s.V);
+    uint32_t blocks = (uint32_t)(L.sms * grid_shape().fused_blocks_per_sm);
+    if (blocks > nb) blocks = nb;
+    Timed timed(L, K_APPLY_STEP);
+#define TENSAIR_STEP(NV) k_apply_step<NV><<<blocks, kStepThreads, 0, L.stream>>>(f, n_receivers, t4, replica_floats / 4, s.d4, stride4, nb)
+    if (s.d4 <= 32) TENSAIR_STEP(1);
+    else if (s.d4 <= 64) TENSAIR_STEP(2);
+    else if (s.d4 <= 96) TENSAIR_STEP(3);
+    else if (s.d4 <= 128) TENSAIR_STEP(4);
+    else TENSAIR_STEP(8);
+#undef TENSAIR_STEP
+    return cudaGetLastError();
+}
+
 // One warp per row: dot product and both squared norms in fp64, combined by shuffles.
 __global__ void __launch_bounds__(256)
 k_cosine_difference(const float* __restrict__ rows, const float* __restrict__ snap, float* __restrict__ out,

@@ -9,13 +9,15 @@ namespace tensair {
 enum KernelKind {
     K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
     K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
-    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_ALIAS_BUILD, K_HEADS_LONG, K_KINDS
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_ALIAS_BUILD, K_HEADS_LONG,
+    K_APPLY_STEP, K_KINDS
 };
 inline const char* kernel_name(int kind) {
     static const char* const names[K_KINDS] = {
         "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
         "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
-        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted", "alias_build", "heads_long_rows"};
+        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted", "alias_build", "heads_long_rows",
+        "apply_step"};
     return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
 }
 
@@ -133,6 +135,19 @@ struct FusedMessages {
     const uint32_t* buckets[kMaxFused];
 };
 cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float* table, const Shape& s);
+// Everything due in one step, for all receivers of the context, in one pass: the messages in (origin step,
+// sender) order, each with the set of receivers it is due for.  Every (row, receiver) pair is fetched once,
+// receives the deltas of its messages in message order and is stored once.
+constexpr int kMaxStepMessages = 32;
+struct StepMessages {
+    uint32_t count;
+    const uint32_t* ids[kMaxStepMessages];
+    const float* delta[kMaxStepMessages];
+    const uint32_t* buckets[kMaxStepMessages];
+    uint32_t receivers[kMaxStepMessages];   // bit r set: add to the table of local replica r
+};
+cudaError_t launch_apply_step(const Launcher& L, const StepMessages& f, uint32_t n_receivers, float* tables,
+                              size_t replica_floats, const Shape& s);
 // merge.cu: the sum of up to kMaxMerge buffered messages (each with its bucket index) into one message.
 constexpr int kMaxMerge = 8;
 struct MergeInputs {

@@ -447,6 +447,49 @@ int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint64_t step, ui
     return apply_due(ctx, replica, due);
 }
 
+int tensair_apply_step(tensair_ctx* ctx, uint64_t step, uint32_t* n_applied) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const uint32_t W = ctx->cfg.W;
+    std::vector<std::vector<Due>> due(W);
+    uint32_t total = 0;
+    for (uint32_t r = 0; r < W; ++r) {
+        due[r] = ctx->sched->take_due(ctx->gid(r), step, false);
+        total += (uint32_t)due[r].size();
+    }
+    if (n_applied) *n_applied = total;
+    // the distinct messages among them, in (origin step, sender) order, each with its receivers
+    struct Msg { uint64_t origin; uint32_t sender, slot, receivers; };
+    std::vector<Msg> msgs;
+    for (uint32_t r = 0; r < W && r < 32; ++r)
+        for (const Due& d : due[r]) {
+            auto it = std::find_if(msgs.begin(), msgs.end(), [&](const Msg& m) { return m.slot == d.slot; });
+            if (it == msgs.end()) msgs.push_back(Msg{d.origin, d.sender, d.slot, 1u << r});
+            else it->receivers |= 1u << r;
+        }
+    std::sort(msgs.begin(), msgs.end(), [](const Msg& a, const Msg& b) {
+        return a.origin != b.origin ? a.origin < b.origin : a.sender < b.sender;
+    });
+    if (!grid_shape().fuse_apply || W > 32 || msgs.size() > (size_t)kMaxStepMessages || total < 2) {
+        for (uint32_t r = 0; r < W; ++r) {
+            const int rc = apply_due(ctx, r, due[r]);
+            if (rc != TENSAIR_OK) return rc;
+        }
+        return TENSAIR_OK;
+    }
+    StepMessages f;
+    f.count = (uint32_t)msgs.size();
+    for (size_t i = 0; i < msgs.size(); ++i) {
+        f.ids[i] = ctx->slot_ids(msgs[i].slot);
+        f.delta[i] = ctx->slot_delta(msgs[i].slot);
+        f.buckets[i] = ctx->slot_buckets(msgs[i].slot);
+        f.receivers[i] = msgs[i].receivers;
+    }
+    TENSAIR_CUDA(ctx, launch_apply_step(ctx->L, f, W, ctx->tables, (size_t)2 * ctx->cfg.V * ctx->cv.stride, ctx->shape));
+    return TENSAIR_OK;
+}
+
 int tensair_drain(tensair_ctx* ctx, uint32_t* n_applied) {
     if (!ctx) return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);

@@ -616,6 +616,34 @@ def test_fused_and_one_by_one_application_are_bit_identical(torch):
         assert np.array_equal(a.view(np.uint32), b.view(np.uint32))
 
 
+@pytest.mark.parametrize("W,d,max_delay", [(5, 40, 2), (8, 300, 3), (2, 8, 0)])
+def test_one_pass_for_all_receivers_equals_the_per_receiver_calls(torch, W, d, max_delay):
+    """tensair_apply_step against tensair_apply_messages per replica: tables and delivery logs bit for bit, and
+    both against the oracle's delivery order."""
+    wl = synth.scaled(synth.LARGE_DRIFT, V=30_000, d=d, batch=1024, W=W, k=6, drift_every=0, max_delay=max_delay,
+                      stream_seeds=tuple(range(30, 30 + W)))
+    streams = synth.all_streams(wl, 7)
+    counts = synth.stream_counts(streams, wl.V)
+    o, one_pass = make_pair(wl, counts=counts)
+    _, per_receiver = make_pair(wl, counts=counts)
+    for t in range(7):
+        for i in range(wl.W):
+            assert o.train_batch(i, streams[i][t], t)[0] == 0
+            one_pass.tensair_train_batch(i, dev(torch, streams[i][t]), t)
+            per_receiver.tensair_train_batch(i, dev(torch, streams[i][t]), t)
+        n = sum(per_receiver.tensair_apply_messages(j, t) for j in range(wl.W))
+        assert one_pass.tensair_apply_step(t) == n == sum(o.apply_messages(j, t) for j in range(wl.W))
+        assert one_pass.tensair_apply_step(t) == 0          # a second call for the step applies nothing
+    assert one_pass.tensair_drain() == per_receiver.tensair_drain() == o.drain()
+    for j in range(wl.W):
+        log = one_pass.tensair_read_delivery_log(j)
+        assert np.array_equal(log, per_receiver.tensair_read_delivery_log(j)) and np.array_equal(log, o.delivery_log(j))
+        for which in (0, 1):
+            a, b = one_pass.tensair_read_embeddings(j, which), per_receiver.tensair_read_embeddings(j, which)
+            assert np.array_equal(a.view(np.uint32), b.view(np.uint32)), (j, which)
+        compare_tables(o, one_pass, j, TOL_200)
+
+
 def test_full_size_drift_workload_with_sampler_rebuild(torch):
     """V = 1M, d = 300, batch 16384, k = 15, W = 8, delay <= 2, Zipf 1.1 with a permuted vocabulary: two steps,
     the sampler rebuilt from the running counts in between, everything against the oracle."""
