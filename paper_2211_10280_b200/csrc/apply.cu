@@ -111,64 +111,6 @@ cudaError_t launch_index_received(const Launcher& L, MsgHeader* hdr, const uint3
     return cudaGetLastError();
 }
 
-// Several messages, one pass.  A block owns an id range (a few buckets in a grid-stride loop); for each
-// message in order its warps take the message's rows in that range; a block-wide barrier separates the
-// messages, so a row touched by two of them gets its additions in message order.  Table rows are read
-// with L1 bypassed (another warp of the block may just have written them).
-constexpr int kFusedThreads = 128;
-template <int NV>
-__global__ void __launch_bounds__(kFusedThreads)
-k_apply_fused(FusedMessages f, float4* __restrict__ table, uint32_t d4, uint32_t stride4, uint32_t n_buckets) {
-    const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    constexpr uint32_t kWarps = kFusedThreads / 32;
-    for (uint32_t b = blockIdx.x; b < n_buckets; b += gridDim.x) {
-        for (uint32_t k = 0; k < f.count; ++k) {
-            const uint32_t beg = __ldg(f.buckets[k] + b), end = __ldg(f.buckets[k] + b + 1);
-            const float4* __restrict__ delta = reinterpret_cast<const float4*>(f.delta[k]);
-            for (uint32_t m = beg + wid; m < end; m += kWarps) {
-                const uint32_t id = __ldg(f.ids[k] + m);
-                const float4* __restrict__ src = delta + (size_t)m * stride4;
-                float4* dst = table + (size_t)id * stride4;
-                float4 a[NV], r[NV];
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const uint32_t e = lane + 32 * i;
-                    if (e < d4) {
-                        a[i] = __ldg(src + e);
-                        r[i] = __ldcg(dst + e);
-                    }
-                }
-#pragma unroll
-                for (int i = 0; i < NV; ++i) {
-                    const uint32_t e = lane + 32 * i;
-                    if (e < d4) {
-                        r[i].x += a[i].x; r[i].y += a[i].y; r[i].z += a[i].z; r[i].w += a[i].w;
-                        dst[e] = r[i];
-                    }
-                }
-            }
-            __syncthreads();
-        }
-    }
-}
-
-cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float* table, const Shape& s) {
-    const uint32_t stride4 = s.stride / 4;
-    float4* t4 = reinterpret_cast<float4*>(table);
-    const uint32_t nb = bucket_count(s.V);
-    uint32_t blocks = (uint32_t)(L.sms * grid_shape().fused_blocks_per_sm);
-    if (blocks > nb) blocks = nb;
-    Timed timed(L, K_APPLY_FUSED);
-#define TENSAIR_FUSED(NV) k_apply_fused<NV><<<blocks, kFusedThreads, 0, L.stream>>>(f, t4, s.d4, stride4, nb)
-    if (s.d4 <= 32) TENSAIR_FUSED(1);
-    else if (s.d4 <= 64) TENSAIR_FUSED(2);
-    else if (s.d4 <= 96) TENSAIR_FUSED(3);
-    else if (s.d4 <= 128) TENSAIR_FUSED(4);
-    else TENSAIR_FUSED(8);
-#undef TENSAIR_FUSED
-    return cudaGetLastError();
-}
-
 // All receivers, one pass, no ordering barriers.  A message carries the set of receivers it is due for.  A block
 // owns a bucket (16 consecutive row ids).  It first notes, per message, which of the 16 ids the message holds
 // (a 16-bit mask; ids ascend, so the row of id j is the bucket's first row plus the number of mask bits below j).
@@ -250,13 +192,13 @@ k_apply_step(StepMessages f, uint32_t n_receivers, float4* __restrict__ tables, 
 }
 
 cudaError_t launch_apply_step(const Launcher& L, const StepMessages& f, uint32_t n_receivers, float* tables,
-                              size_t replica_floats, const Shape& s) {
+                              size_t replica_floats, const Shape& s, int kind) {
     const uint32_t stride4 = s.stride / 4;
     float4* t4 = reinterpret_cast<float4*>(tables);
     const uint32_t nb = bucket_count(s.V);
     uint32_t blocks = (uint32_t)(L.sms * grid_shape().fused_blocks_per_sm);
     if (blocks > nb) blocks = nb;
-    Timed timed(L, K_APPLY_STEP);
+    Timed timed(L, kind);
 #define TENSAIR_STEP(NV) k_apply_step<NV><<<blocks, kStepThreads, 0, L.stream>>>(f, n_receivers, t4, replica_floats / 4, s.d4, stride4, nb)
     if (s.d4 <= 32) TENSAIR_STEP(1);
     else if (s.d4 <= 64) TENSAIR_STEP(2);

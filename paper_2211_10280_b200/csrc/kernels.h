@@ -125,16 +125,6 @@ cudaError_t launch_reduce_long_rows(const Launcher& L, const Rec* terms, const u
 // apply.cu
 cudaError_t launch_apply(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, const float* delta,
                          float* table, const Shape& s);
-// Several messages for one receiver in one pass: applied id range by id range, message after message within
-// a range, so every table row sees its deltas in message order and is fetched from memory once.
-constexpr int kMaxFused = 8;
-struct FusedMessages {
-    uint32_t count;
-    const uint32_t* ids[kMaxFused];
-    const float* delta[kMaxFused];
-    const uint32_t* buckets[kMaxFused];
-};
-cudaError_t launch_apply_fused(const Launcher& L, const FusedMessages& f, float* table, const Shape& s);
 // Everything due in one step, for all receivers of the context, in one pass: the messages in (origin step,
 // sender) order, each with the set of receivers it is due for.  Every (row, receiver) pair is fetched once,
 // receives the deltas of its messages in message order and is stored once.
@@ -146,8 +136,9 @@ struct StepMessages {
     const uint32_t* buckets[kMaxStepMessages];
     uint32_t receivers[kMaxStepMessages];   // bit r set: add to the table of local replica r
 };
+// kind: K_APPLY_STEP, or K_APPLY_FUSED when the pass serves one receiver (tables = that receiver's table).
 cudaError_t launch_apply_step(const Launcher& L, const StepMessages& f, uint32_t n_receivers, float* tables,
-                              size_t replica_floats, const Shape& s);
+                              size_t replica_floats, const Shape& s, int kind);
 // merge.cu: the sum of up to kMaxMerge buffered messages (each with its bucket index) into one message.
 constexpr int kMaxMerge = 8;
 struct MergeInputs {

@@ -237,24 +237,26 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
 }
 
 int apply_due(tensair_ctx* ctx, uint32_t receiver, const std::vector<Due>& due) {
-    // Messages are applied in the order given; up to kMaxFused of them share one pass over the table.
+    // Messages are applied in the order given; up to kMaxStepMessages of them share one pass over the table.
     size_t at = 0;
+    const size_t replica_floats = (size_t)2 * ctx->cfg.V * ctx->cv.stride;
     while (at < due.size()) {
-        const size_t k = grid_shape().fuse_apply ? std::min(due.size() - at, (size_t)kMaxFused) : 1;
+        const size_t k = grid_shape().fuse_apply ? std::min(due.size() - at, (size_t)kMaxStepMessages) : 1;
         if (k == 1) {
             const Due& d = due[at];
             TENSAIR_CUDA(ctx, launch_apply(ctx->L, ctx->slot_hdr(d.slot), ctx->slot_ids(d.slot), ctx->slot_delta(d.slot),
                                            ctx->table_of(receiver), ctx->shape));
         } else {
-            FusedMessages f;
+            StepMessages f;
             f.count = (uint32_t)k;
             for (size_t i = 0; i < k; ++i) {
                 const uint32_t slot = due[at + i].slot;
                 f.ids[i] = ctx->slot_ids(slot);
                 f.delta[i] = ctx->slot_delta(slot);
                 f.buckets[i] = ctx->slot_buckets(slot);
+                f.receivers[i] = 1u;
             }
-            TENSAIR_CUDA(ctx, launch_apply_fused(ctx->L, f, ctx->table_of(receiver), ctx->shape));
+            TENSAIR_CUDA(ctx, launch_apply_step(ctx->L, f, 1, ctx->table_of(receiver), replica_floats, ctx->shape, K_APPLY_FUSED));
         }
         at += k;
     }
@@ -486,7 +488,7 @@ int tensair_apply_step(tensair_ctx* ctx, uint64_t step, uint32_t* n_applied) {
         f.buckets[i] = ctx->slot_buckets(msgs[i].slot);
         f.receivers[i] = msgs[i].receivers;
     }
-    TENSAIR_CUDA(ctx, launch_apply_step(ctx->L, f, W, ctx->tables, (size_t)2 * ctx->cfg.V * ctx->cv.stride, ctx->shape));
+    TENSAIR_CUDA(ctx, launch_apply_step(ctx->L, f, W, ctx->tables, (size_t)2 * ctx->cfg.V * ctx->cv.stride, ctx->shape, K_APPLY_STEP));
     return TENSAIR_OK;
 }
 
