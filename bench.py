@@ -43,9 +43,9 @@ FALLBACK_HBM_GBS = 6650.0
 # the ncu captures summarised under profiles/ on a reduced case; the apply kernels are pure streams over the rows
 # of their messages, so traffic grows in proportion to the algorithmic bytes of a launch.  Only valid for the
 # source file the capture ran (checked by its SHA-256), null otherwise.
-NCU_TRAFFIC = {"apply_fused": {"traffic_per_algorithmic_byte": 0.996, "source": "paper_2211_10280_b200/csrc/apply.cu",
-                               "sha256": "68c94b2b3562f04ec06ec7ab85632d6640ba520cbf1c509e65fdade149f06ed0",
-                               "profile": "profiles/k_apply_fused_small_case_V250k_W4.md"}}
+NCU_TRAFFIC = {"apply_step": {"traffic_per_algorithmic_byte": 1.026, "source": "paper_2211_10280_b200/csrc/apply.cu",
+                              "sha256": "0fbd0c9d1aa90b2ff98518c7af8f160f2efc609bc9c97a02da3bcbe088d29569",
+                              "profile": "profiles/k_apply_step_small_case_V250k_W4.md"}}
 
 
 def ncu_traffic(kernel: str, algorithmic_bytes: float):
@@ -417,7 +417,7 @@ def run_ours(args):
     per_step = {}
     for (j, at), members in groups.items():
         per_step.setdefault(at, {})[j] = members
-    step_pass_bytes, step_pass_log = [], []
+    step_pass_bytes = []
     for at, per_j in sorted(per_step.items()):
         distinct = sorted({m for ms in per_j.values() for m in ms})
         if sum(len(ms) for ms in per_j.values()) < 2 or any(msg_ids.get(m) is None for m in distinct):
@@ -425,31 +425,33 @@ def run_ours(args):
         delta_rows = sum(msg_ids[m].size for m in distinct)
         union_rows = sum(np.unique(np.concatenate([msg_ids[m] for m in ms])).size for ms in per_j.values())
         step_pass_bytes.append(delta_rows * (row + 4) + union_rows * 2 * row)
-        step_pass_log.append({"step": at, "messages": len(distinct), "deliveries": sum(len(ms) for ms in per_j.values()),
-                              "kernel": "k_apply_step", "delta_rows": delta_rows, "union_rows": union_rows,
-                              "algorithmic_bytes": step_pass_bytes[-1]})
     if step_pass_bytes:
         algo["apply_step"] = float(np.mean(step_pass_bytes))
     if args.log_applies:
-        # every apply call of the run in call order, with the bytes its launch has to move (for matching ncu captures)
+        # every apply launch of the run in call order, with the bytes it has to move (for matching ncu captures)
         calls = {}
         for j in range(wl.W):
             for origin, snd, due, at, _ in ctx.tensair_read_delivery_log(j).tolist():
-                calls.setdefault((at, j), []).append((snd, origin))
+                calls.setdefault(at, {}).setdefault(j, []).append((snd, origin))
         with open(args.log_applies, "w") as fh:
-            if not args.apply_per_replica:
-                # note: only the steps of the per-kernel pass (the message ids of earlier steps are not kept)
-                for rec in step_pass_log:
-                    fh.write(json.dumps(rec) + "\n")
-            for (at, j), members in sorted(calls.items()) if args.apply_per_replica else []:
-                ids = [msg_ids.get(m) for m in members]
-                if any(x is None for x in ids):
+            for at, per_j in sorted(calls.items()):
+                if any(msg_ids.get(m) is None for ms in per_j.values() for m in ms):
                     continue
-                union = np.unique(np.concatenate(ids)).size
-                nbytes = sum(x.size for x in ids) * (row + 4) + union * 2 * row
-                fh.write(json.dumps({"step": at, "receiver": j, "messages": len(members), "kernel":
-                                     "k_apply_fused" if len(members) > 1 else "k_apply", "delta_rows": sum(x.size for x in ids),
-                                     "union_rows": union, "algorithmic_bytes": nbytes}) + "\n")
+                if args.apply_per_replica:
+                    for j, members in sorted(per_j.items()):
+                        ids = [msg_ids[m] for m in members]
+                        union = np.unique(np.concatenate(ids)).size
+                        fh.write(json.dumps({"step": at, "receiver": j, "messages": len(members), "kernel":
+                                             "k_apply_step (one receiver)" if len(members) > 1 else "k_apply",
+                                             "delta_rows": sum(x.size for x in ids), "union_rows": union,
+                                             "algorithmic_bytes": sum(x.size for x in ids) * (row + 4) + union * 2 * row}) + "\n")
+                else:
+                    distinct = sorted({m for ms in per_j.values() for m in ms})
+                    delta_rows = sum(msg_ids[m].size for m in distinct)
+                    union_rows = sum(np.unique(np.concatenate([msg_ids[m] for m in ms])).size for ms in per_j.values())
+                    fh.write(json.dumps({"step": at, "messages": len(distinct), "deliveries": sum(len(ms) for ms in per_j.values()),
+                                         "kernel": "k_apply_step", "delta_rows": delta_rows, "union_rows": union_rows,
+                                         "algorithmic_bytes": delta_rows * (row + 4) + union_rows * 2 * row}) + "\n")
     tot_ms = sum(v[1] for v in prof.values()) or 1.0
     kernels = {}
     for name, (cnt, ms) in prof.items():

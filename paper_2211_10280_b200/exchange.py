@@ -12,7 +12,7 @@ one-process result bit for bit.
 
 Only plumbing lives here (torch.distributed calls and the order of the library calls); the arithmetic is
 the library's.  `port` is a binding.Context created with world_replicas / first_replica, or anything with
-the same six methods (the CPU tests use a stand-in that needs no GPU).
+the same calls (the CPU tests use a stand-in that needs no GPU).
 """
 from __future__ import annotations
 
@@ -65,11 +65,9 @@ class ShardedReplicas:
     def apply(self, step: int) -> int:
         """Gradient application of what is due at `step`: for real on the replicas held here, as book-keeping
         for the others.  Returns the messages applied to local replicas."""
-        applied = 0
+        applied = self.port.tensair_apply_step(step)          # all local replicas in one pass over their tables
         for g in range(self.world_replicas):
-            if self.first <= g < self.first + self.local:
-                applied += self.port.tensair_apply_messages(g - self.first, step)
-            else:
+            if not self.first <= g < self.first + self.local:
                 self.port.tensair_shadow_apply(g, step, False)
         return applied
 

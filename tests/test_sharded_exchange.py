@@ -1,6 +1,6 @@
 """The message exchange between processes (paper_2211_10280_b200/exchange.py) on CPU: two and three gloo ranks.
 
-No GPU here, so the context is replaced by a stand-in with the same six calls: its pool slots are CPU
+No GPU here, so the context is replaced by a stand-in with the same calls: its pool slots are CPU
 tensors, its "training" writes a message whose content is a function of (sender, step), and its delivery
 schedule is the library's own host-side schedule (tensair_schedule_*).  Checked per rank: every message that
 is applied carries the sender's content (it arrived whole, before it was due, and was not overwritten before
@@ -93,6 +93,9 @@ class Port:
         for rec in due:
             self._check(self.first + r, rec)
         return len(due)
+
+    def tensair_apply_step(self, step):
+        return sum(self.tensair_apply_messages(r, step) for r in range(LOCAL))
 
     def tensair_shadow_apply(self, g, step, drain):
         return len(self.sched.take_due(g, step, drain))
