@@ -27,7 +27,10 @@
  * Layouts
  *   - Tables: replica r owns 2*V rows of row_stride floats, input (centre-word) rows [0,V) followed
  *     by output (context-word) rows [V,2V); replicas are consecutive.  Only the first d floats of a
- *     row are meaningful.  A "row id" in [0,2V) names a row of this unified table.
+ *     row are meaningful.  A "row id" in [0,2V) names a row of this unified table.  Table entries must be
+ *     finite: the kernels widen fp32 to fp64 by a bit manipulation that is exact for every finite value
+ *     (subnormals and zeros included) but reads an infinity or a NaN as a finite number, so a table that has
+ *     diverged to non-finite values gives unspecified (finite or not) results instead of propagating NaNs.
  *   - Sparse gradient message (the payload of Algorithm 1's send_gradients; Section 4 notes that a
  *     word-embedding mini-batch changes few of the model's variables, so only touched rows travel):
  *     a row count n, n strictly ascending row ids, n delta rows (already scaled by -lr).  Applying
@@ -287,8 +290,8 @@ TENSAIR_API int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint6
 /*
  * tensair_apply_messages(replica, step) for every replica of the context, as one pass over their tables: a
  * message due for several of them at this step is read from memory once and added to each (the replicas share
- * one GPU's memory, so the gradient application that every Model instance repeats - Section 4.2 notes it does
- * not shrink with the number of instances - shares its reads here).  Per replica the messages are applied in
+ * one GPU's memory, so the gradient application that every Model instance repeats - Section 4.2 notes that it is
+ * not distributed - shares its reads here).  Per replica the messages are applied in
  * the same (origin step, sender) order, so tables and delivery logs are bit-identical to the per-replica calls.
  * n_applied: host, nullable: deliveries made, summed over the replicas.
  */
