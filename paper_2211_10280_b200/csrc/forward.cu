@@ -61,8 +61,9 @@ constexpr int kFwdWarps = 2;       // warps per block
 //   3. evaluates sigmoid and loss for all rows at once (one row per lane pair instead of one per warp),
 //   4. re-reads the staged rows and adds g * u to the centre gradient kept in registers.
 // The partial centre gradient of the side is written once; nothing is shared between warps.
-// NV: float4 slices per lane.  CR: rows reduced together (16 or 8); 32 / CR lanes share a row's scalar.
-template <int NV, int CR>
+// NV: float4 slices per lane.  CR: rows reduced together (a power of two); 32 / CR lanes share a row's scalar.
+// NR <= CR: rows of a whole chunk (the loops without predicates run over exactly NR staged rows).
+template <int NV, int CR, int NR = CR>
 __global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, uint32_t stride4, uint32_t w,
           uint32_t k, uint32_t chunk_rows, uint32_t warp_stage4, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
@@ -134,24 +135,24 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                 // A chunk whose CR rows are all live takes loops without predicates, which the compiler is free to
                 // interleave: a lane whose slice lies past the row's end reads whatever the buffer holds there
                 // (finite once widened) against a centre value of zero.
-                const bool full = live == (CR == 32 ? 0xFFFFFFFFu : (1u << CR) - 1u);
+                const bool full = live == (NR == 32 ? 0xFFFFFFFFu : (1u << NR) - 1u);
                 double xp[CR];
                 if (full) {
 #pragma unroll
-                    for (int j = 0; j < CR; ++j) xp[j] = 0.0;
+                    for (int j = 0; j < CR; ++j) xp[j] = 0.0;   // rows NR .. CR-1 stay zero
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
-                        float4 f[CR];
+                        float4 f[NR];
 #pragma unroll
-                        for (int j = 0; j < CR; ++j) f[j] = stage[(size_t)j * stride4 + lane + 32 * i];
+                        for (int j = 0; j < NR; ++j) f[j] = stage[(size_t)j * stride4 + lane + 32 * i];
 #pragma unroll
-                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].x), v[i][0], xp[j]);
+                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].x), v[i][0], xp[j]);
 #pragma unroll
-                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].y), v[i][1], xp[j]);
+                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].y), v[i][1], xp[j]);
 #pragma unroll
-                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].z), v[i][2], xp[j]);
+                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].z), v[i][2], xp[j]);
 #pragma unroll
-                        for (int j = 0; j < CR; ++j) xp[j] = fma(widen_down(f[j].w), v[i][3], xp[j]);
+                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].w), v[i][3], xp[j]);
                     }
                 } else {
 #pragma unroll
@@ -201,13 +202,13 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                 if (writer && jr < nr) rec[cbase + j0 + jr] = Rec{g, centre, 0u};
                 // 4. centre gradient: acc += g_j * u_j
                 if (full) {
-                    double gw[CR];
+                    double gw[NR];
 #pragma unroll
-                    for (int j = 0; j < CR; ++j) gw[j] = __shfl_sync(0xFFFFFFFFu, g, LPR * j) * kWidenUp;   // exact: |g| <= 1
+                    for (int j = 0; j < NR; ++j) gw[j] = __shfl_sync(0xFFFFFFFFu, g, LPR * j) * kWidenUp;   // exact: |g| <= 1
 #pragma unroll
                     for (int i = 0; i < NV; ++i) {
 #pragma unroll
-                        for (int j = 0; j < CR; ++j) {
+                        for (int j = 0; j < NR; ++j) {
                             const float4 f = stage[(size_t)j * stride4 + lane + 32 * i];
                             acc[i][0] = fma(gw[j], widen_down(f.x), acc[i][0]);
                             acc[i][1] = fma(gw[j], widen_down(f.y), acc[i][1]);
@@ -272,10 +273,17 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     int blocks_per_sm = g_forward_blocks > 0 ? g_forward_blocks : (cr == 16 ? 5 : cr == 8 ? 8 : 10);
     // rows staged per chunk: as many of the cr as fit the shared memory share of one block
     uint32_t chunk_rows = s.K1 < (uint32_t)cr ? s.K1 : (uint32_t)cr;
-    const size_t budget = (size_t)216 * 1024 / blocks_per_sm - 1024;
     // a warp's buffer ends with padding up to slice 32 * NV of its last row (see the kernel)
     const uint32_t nv = s.d4 <= 32 ? 1 : s.d4 <= 64 ? 2 : s.d4 <= 96 ? 3 : s.d4 <= 128 ? 4 : 8;
     const size_t pad = 32u * nv * 16 > row ? 32u * nv * 16 - row : 0;
+    // Whole chunks first: the loops without predicates need all cr rows staged, and they are worth more than
+    // resident blocks (measured at d = 512: 6 blocks of whole chunks 0.89 ms, 8 blocks of 6-row chunks 1.15 ms).
+    auto fits = [&](uint32_t rows_, int blocks_) {
+        return (size_t)kFwdWarps * (rows_ * row + pad) + kFwdWarps * 8 <= (size_t)216 * 1024 / blocks_ - 1024;
+    };
+    if (g_forward_blocks <= 0)
+        while (blocks_per_sm > 2 && !fits(chunk_rows, blocks_per_sm)) --blocks_per_sm;
+    const size_t budget = (size_t)216 * 1024 / blocks_per_sm - 1024;
     while (chunk_rows > 1 && (size_t)kFwdWarps * (chunk_rows * row + pad) + kFwdWarps * 8 > budget) --chunk_rows;
     const uint32_t warp_stage4 = (uint32_t)((chunk_rows * row + pad) / 16);
     const size_t smem = (size_t)kFwdWarps * warp_stage4 * 16 + kFwdWarps * 8;
@@ -286,20 +294,22 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     const uint32_t resident = (uint32_t)(L.sms * blocks_per_sm);
     if (blocks > resident) blocks = resident;
     Timed timed(L, K_FORWARD);
-#define TENSAIR_FWD(NV, CR)                                                                                     \
+#define TENSAIR_FWD(NV, CR)  TENSAIR_FWD_NR(NV, CR, CR)
+#define TENSAIR_FWD_NR(NV, CR, NR)                                                                                  \
     do {                                                                                                        \
-        static bool attr_set = false;                                                                           \
+        static bool attr_set = false;                                                                        \
         if (!attr_set) {                                                                                        \
-            cudaFuncSetAttribute(k_forward<NV, CR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);   \
-            cudaFuncSetAttribute(k_forward<NV, CR>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);       \
+            cudaFuncSetAttribute(k_forward<NV, CR, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);   \
+            cudaFuncSetAttribute(k_forward<NV, CR, NR>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);       \
             attr_set = true;                                                                                    \
         }                                                                                                       \
-        k_forward<NV, CR><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,     \
+        k_forward<NV, CR, NR><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,     \
                                                                       chunk_rows, warp_stage4, t4, rows, rec,  \
                                                                       gin_pos,                                 \
                                                                       loss_pos, err, owned, n_owned);                  \
     } while (0)
-#define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)
+    // k = 5 (six rows per pair) is common enough to have whole chunks of its own
+#define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8 && chunk_rows == 6) TENSAIR_FWD_NR(NV, 8, 6); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)
     if (s.d4 <= 32) TENSAIR_FWD_NV(1);
     else if (s.d4 <= 64) TENSAIR_FWD_NV(2);
     else if (s.d4 <= 96) TENSAIR_FWD_NV(3);
@@ -307,6 +317,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     else TENSAIR_FWD_NV(8);
 #undef TENSAIR_FWD_NV
 #undef TENSAIR_FWD
+#undef TENSAIR_FWD_NR
     return cudaGetLastError();
 }
 
