@@ -52,6 +52,11 @@ __device__ inline SigmoidLoss sigmoid_loss(double x) {
 }
 
 constexpr int kFwdWarps = 2;       // warps per block
+// The radix sort of a batch runs on a second stream beside this kernel; its scatter kernel needs 256 threads x 64
+// registers on a multiprocessor to get in at all.  The forward grid leaves that many registers free: measured
+// with 120 registers per thread, 8 resident blocks (no room: the sort ends up behind the forward kernel) 5.79 ms
+// per step, 6 blocks (room for one sort block) 5.57 ms although the forward kernel itself takes 0.40 instead of 0.31 ms.
+constexpr int kRegistersLeftForTheSort = 256 * 64;
 
 // One warp per side of a centre position (grid-stride), no block-level cooperation.  For every pair of
 // its side the warp stages the pair's 1 + k output rows into its own shared-memory buffer with one
@@ -109,13 +114,23 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
         const uint32_t hi = q + w < n ? q + w : n - 1;
         const uint32_t c_beg = side ? q + 1 : lo, c_end = side ? hi + 1 : q;
         uint32_t p = pair_offset(q, n, w) + (side ? q - lo : 0u);
+        // Row ids of a pair (lane l holds row l when a pair has at most 32 rows) and its context token are fetched
+        // one pair ahead, so that a chunk's copies do not wait for a load of their addresses first.
+        const bool ids_in_lanes = K1 <= 32;
+        uint32_t ids_next = ids_in_lanes && lane < K1 && c_beg < c_end ? __ldg(rows + p * K1 + lane) : 0u;
+        uint32_t ctx_next = c_beg < c_end ? (uint32_t)tok[c_beg] : 0u;
         for (uint32_t c = c_beg; c < c_end && !failed; ++c) {
-            const uint32_t ctx = (uint32_t)tok[c];
+            const uint32_t ctx = ctx_next, ids_pair = ids_next;
             const uint32_t cbase = p * K1;
             ++p;
+            if (c + 1 < c_end) {
+                if (ids_in_lanes && lane < K1) ids_next = __ldg(rows + p * K1 + lane);
+                ctx_next = (uint32_t)tok[c + 1];
+            }
             for (uint32_t j0 = 0; j0 < K1 && !failed; j0 += chunk_rows) {
                 const uint32_t nr = K1 - j0 < chunk_rows ? K1 - j0 : chunk_rows;
-                const uint32_t rid = lane < nr ? __ldg(rows + cbase + j0 + lane) : 0u;
+                uint32_t rid = __shfl_sync(0xFFFFFFFFu, ids_pair, (j0 + lane) & 31u);
+                if (!ids_in_lanes) rid = lane < nr ? __ldg(rows + cbase + j0 + lane) : 0u;
                 const bool mine = lane < nr && (j0 + lane == 0 || rid != ctx);
                 const uint32_t live = __ballot_sync(0xFFFFFFFFu, mine);
                 // stage the live rows: the buffer was last read by this warp, so order those reads first
@@ -296,17 +311,24 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     Timed timed(L, K_FORWARD);
 #define TENSAIR_FWD(NV, CR)  TENSAIR_FWD_NR(NV, CR, CR)
 #define TENSAIR_FWD_NR(NV, CR, NR)                                                                                  \
-    do {                                                                                                        \
-        static bool attr_set = false;                                                                        \
-        if (!attr_set) {                                                                                        \
+    do {                                                                                                            \
+        static bool attr_set = false;                                                                               \
+        static int room_for = 0;                                                                                    \
+        if (!attr_set) {                                                                                            \
             cudaFuncSetAttribute(k_forward<NV, CR, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);   \
             cudaFuncSetAttribute(k_forward<NV, CR, NR>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);       \
-            attr_set = true;                                                                                    \
-        }                                                                                                       \
-        k_forward<NV, CR, NR><<<blocks, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,     \
-                                                                      chunk_rows, warp_stage4, t4, rows, rec,  \
-                                                                      gin_pos,                                 \
-                                                                      loss_pos, err, owned, n_owned);                  \
+            cudaFuncAttributes fa;                                                                                  \
+            if (cudaFuncGetAttributes(&fa, k_forward<NV, CR, NR>) == cudaSuccess && fa.numRegs > 0)                 \
+                room_for = (65536 - kRegistersLeftForTheSort) / (fa.numRegs * kFwdWarps * 32);                      \
+            attr_set = true;                                                                                        \
+        }                                                                                                           \
+        uint32_t grid = blocks;                                                                                     \
+        if (g_forward_blocks <= 0 && grid_shape().overlap_sort && room_for >= 1 &&                                  \
+            grid > (uint32_t)(L.sms * room_for))                                                                    \
+            grid = (uint32_t)(L.sms * room_for);                                                                    \
+        k_forward<NV, CR, NR><<<grid, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,       \
+                                                                        chunk_rows, warp_stage4, t4, rows, rec,     \
+                                                                        gin_pos, loss_pos, err, owned, n_owned);    \
     } while (0)
     // k = 5 (six rows per pair) is common enough to have whole chunks of its own
 #define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8 && chunk_rows == 6) TENSAIR_FWD_NR(NV, 8, 6); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)
