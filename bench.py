@@ -473,9 +473,19 @@ def run_ours(args):
                 "avg_ms": kernels[dom]["avg_ms"], "share_of_device_time": kernels[dom]["share"]}
     own = U * row + U * (row + 4) + U * (row + 4 + 2 * row)
     # remote part: every message applied in the per-kernel pass, per-message model (delta read, row read, row write)
-    remote_per_step = len(applied) / Kp * U_applied * (row + 4 + 2 * row) if applied else 0.0
+    # remote part, two models: what the launches really have to move (the one-pass apply reads a delta row once however
+    # many receivers it is due for, and a table row once however many messages touch it), and the per-message model
+    # (delta read, row read, row write for every delivery) that a message-by-message application would move
+    per_message_model = len(applied) / Kp * U_applied * (row + 4 + 2 * row) if applied else 0.0
+    if args.apply_per_replica:
+        moved = (sum(fused_bytes) + sum(msg_ids[ms[0]].size * (3 * row + 4) for ms in groups.values()
+                                        if len(ms) == 1 and msg_ids.get(ms[0]) is not None)) / Kp
+    else:
+        moved = sum(step_pass_bytes) / Kp
+    remote_per_step = moved if moved else per_message_model
     step_bytes = wl.W * own + remote_per_step
     step_gbs = step_bytes / (ms_dev * 1e-3 / K) / 1e9
+    model_gbs = (wl.W * own + per_message_model) / (ms_dev * 1e-3 / K) / 1e9
 
     out = {
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
@@ -492,7 +502,8 @@ def run_ours(args):
         "clocks": sampler.summary(wall0, wall1),
         "roofline": roofline,
         "step_hbm": {"algorithmic_bytes_per_step": int(step_bytes), "gbs": round(step_gbs, 1),
-                     "frac_of_peak": round(step_gbs / peak, 4), "rows_per_message": int(U)},
+                     "frac_of_peak": round(step_gbs / peak, 4), "rows_per_message": int(U),
+                     "per_message_model_gbs": round(model_gbs, 1)},
         "kernels": kernels,
     }
     if rebuild:

@@ -58,6 +58,29 @@ constexpr int kFwdWarps = 2;       // warps per block
 // per step, 6 blocks (room for one sort block) 5.57 ms although the forward kernel itself takes 0.40 instead of 0.31 ms.
 constexpr int kRegistersLeftForTheSort = 256 * 64;
 
+// A slice of VW consecutive floats of a row (VW = 4: one 16-byte load, VW = 2: one 8-byte load).
+template <int VW> struct Slice;
+template <> struct Slice<4> {
+    static __device__ inline void load(const float* p, float (&a)[4]) {
+        const float4 t = *reinterpret_cast<const float4*>(p);
+        a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
+    }
+    static __device__ inline void load_global(const float* p, float (&a)[4]) {
+        const float4 t = __ldg(reinterpret_cast<const float4*>(p));
+        a[0] = t.x; a[1] = t.y; a[2] = t.z; a[3] = t.w;
+    }
+};
+template <> struct Slice<2> {
+    static __device__ inline void load(const float* p, float (&a)[2]) {
+        const float2 t = *reinterpret_cast<const float2*>(p);
+        a[0] = t.x; a[1] = t.y;
+    }
+    static __device__ inline void load_global(const float* p, float (&a)[2]) {
+        const float2 t = __ldg(reinterpret_cast<const float2*>(p));
+        a[0] = t.x; a[1] = t.y;
+    }
+};
+
 // One warp per side of a centre position (grid-stride), no block-level cooperation.  For every pair of
 // its side the warp stages the pair's 1 + k output rows into its own shared-memory buffer with one
 // bulk asynchronous copy per row (all in flight together, completion counted by an mbarrier), then
@@ -66,28 +89,31 @@ constexpr int kRegistersLeftForTheSort = 256 * 64;
 //   3. evaluates sigmoid and loss for all rows at once (one row per lane pair instead of one per warp),
 //   4. re-reads the staged rows and adds g * u to the centre gradient kept in registers.
 // The partial centre gradient of the side is written once; nothing is shared between warps.
-// NV: float4 slices per lane.  CR: rows reduced together (a power of two); 32 / CR lanes share a row's scalar.
+// A lane holds NV slices of VW floats of a row: slice lane + 32 * i.  VW is 4 unless 2 leaves fewer lanes idle
+// (d = 300: 75 slices of 4 take three rounds of 32 lanes, 150 slices of 2 take five rounds of half the width).
+// CR: rows reduced together (a power of two); 32 / CR lanes share a row's scalar.
 // NR <= CR: rows of a whole chunk (the loops without predicates run over exactly NR staged rows).
-template <int NV, int CR, int NR = CR>
+template <int NV, int CR, int NR, int VW>
 __global__ void __launch_bounds__(kFwdWarps * 32)
-k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, uint32_t stride4, uint32_t w,
-          uint32_t k, uint32_t chunk_rows, uint32_t warp_stage4, const float4* __restrict__ table, const uint32_t* __restrict__ rows,
+k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d, uint32_t stride, uint32_t w,
+          uint32_t k, uint32_t chunk_rows, uint32_t warp_stage, const float* __restrict__ table, const uint32_t* __restrict__ rows,
           Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err,
           const uint32_t* __restrict__ owned, const uint32_t* __restrict__ n_owned) {
     if (*err) return;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
-    // warp_stage4 float4 per warp: chunk_rows rows plus padding, so that slice lane + 32 * i (i < NV) of every
+    // warp_stage floats per warp: chunk_rows rows plus padding, so that slice lane + 32 * i (i < NV) of every
     // staged row is inside the buffer whatever the lane
-    float4* stage = reinterpret_cast<float4*>(smem_raw) + (size_t)wib * warp_stage4;
-    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)kFwdWarps * warp_stage4 * sizeof(float4)) + wib;
+    float* stage = reinterpret_cast<float*>(smem_raw) + (size_t)wib * warp_stage;
+    uint64_t* bar = reinterpret_cast<uint64_t*>(smem_raw + (size_t)kFwdWarps * warp_stage * sizeof(float)) + wib;
     if (lane == 0) mbar_init(bar, 1);
     __syncwarp();
     uint32_t parity = 0;
     bool failed = false;
     const uint32_t K1 = k + 1;
-    const uint32_t row_bytes = d4 * 16;
-    const float4* __restrict__ tout = table + (size_t)V * stride4;
+    const uint32_t row_bytes = d * 4;
+    const uint32_t dv = d / VW;                               // slices of a row
+    const float* __restrict__ tout = table + (size_t)V * stride;
     const uint32_t warp = blockIdx.x * kFwdWarps + wib, nwarps = gridDim.x * kFwdWarps;
 
     // A unit of work is one side of a centre position: the pairs with the context to its left, or to its
@@ -98,16 +124,18 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
         const uint32_t q = owned ? owned[at >> 1] : (at >> 1);
         const uint32_t side = at & 1u;
         const uint32_t centre = (uint32_t)tok[q];
-        const float4* __restrict__ vin = table + (size_t)centre * stride4;
-        double v[NV][4], acc[NV][4];
+        const float* __restrict__ vin = table + (size_t)centre * stride;
+        double v[NV][VW], acc[NV][VW];
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             const uint32_t e = lane + 32 * i;
-            const float4 f = e < d4 ? __ldg(vin + e) : make_float4(0.f, 0.f, 0.f, 0.f);
+            float f[VW];
+#pragma unroll
+            for (int c = 0; c < VW; ++c) f[c] = 0.f;
+            if (e < dv) Slice<VW>::load_global(vin + e * VW, f);
             // the centre row carries the factor 2^896 that the staged rows lack (widen_down)
-            v[i][0] = (double)f.x * kWidenUp; v[i][1] = (double)f.y * kWidenUp;
-            v[i][2] = (double)f.z * kWidenUp; v[i][3] = (double)f.w * kWidenUp;
-            acc[i][0] = acc[i][1] = acc[i][2] = acc[i][3] = 0.0;
+#pragma unroll
+            for (int c = 0; c < VW; ++c) { v[i][c] = (double)f[c] * kWidenUp; acc[i][c] = 0.0; }
         }
         double loss = 0.0;
         const uint32_t lo = q > w ? q - w : 0;
@@ -138,7 +166,7 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                 __syncwarp();
                 if (lane == 0) mbar_arrive_expect_tx(bar, __popc(live) * row_bytes);
                 __syncwarp();
-                if (mine) bulk_copy_g2s(stage + (size_t)lane * stride4, tout + (size_t)rid * stride4, row_bytes, bar);
+                if (mine) bulk_copy_g2s(stage + (size_t)lane * stride, tout + (size_t)rid * stride, row_bytes, bar);
                 if (__any_sync(0xFFFFFFFFu, !mbar_wait_bounded(bar, parity))) {
                     failed = true;
                     mbar_wait_bounded(bar, parity);   // give copies still in flight one more chance to land
@@ -147,43 +175,37 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                 parity ^= 1;
 
                 // 1. partial dot products of the staged rows
-                // A chunk whose CR rows are all live takes loops without predicates, which the compiler is free to
+                // A chunk whose NR rows are all live takes loops without predicates, which the compiler is free to
                 // interleave: a lane whose slice lies past the row's end reads whatever the buffer holds there
                 // (finite once widened) against a centre value of zero.
                 const bool full = live == (NR == 32 ? 0xFFFFFFFFu : (1u << NR) - 1u);
                 double xp[CR];
+#pragma unroll
+                for (int j = 0; j < CR; ++j) xp[j] = 0.0;   // rows NR .. CR-1 of a whole chunk stay zero
                 if (full) {
 #pragma unroll
-                    for (int j = 0; j < CR; ++j) xp[j] = 0.0;   // rows NR .. CR-1 stay zero
-#pragma unroll
                     for (int i = 0; i < NV; ++i) {
-                        float4 f[NR];
+                        float f[NR][VW];
 #pragma unroll
-                        for (int j = 0; j < NR; ++j) f[j] = stage[(size_t)j * stride4 + lane + 32 * i];
+                        for (int j = 0; j < NR; ++j) Slice<VW>::load(stage + (size_t)j * stride + (lane + 32 * i) * VW, f[j]);
 #pragma unroll
-                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].x), v[i][0], xp[j]);
+                        for (int c = 0; c < VW; ++c)
 #pragma unroll
-                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].y), v[i][1], xp[j]);
-#pragma unroll
-                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].z), v[i][2], xp[j]);
-#pragma unroll
-                        for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j].w), v[i][3], xp[j]);
+                            for (int j = 0; j < NR; ++j) xp[j] = fma(widen_down(f[j][c]), v[i][c], xp[j]);
                     }
                 } else {
 #pragma unroll
                     for (int j = 0; j < CR; ++j) {
-                        xp[j] = 0.0;
                         if ((live >> j) & 1u) {
-                            const float4* __restrict__ u = stage + (size_t)j * stride4;
+                            const float* __restrict__ u = stage + (size_t)j * stride;
 #pragma unroll
                             for (int i = 0; i < NV; ++i) {
                                 const uint32_t e = lane + 32 * i;
-                                if (e < d4) {
-                                    const float4 f = u[e];
-                                    xp[j] = fma(widen_down(f.x), v[i][0], xp[j]);
-                                    xp[j] = fma(widen_down(f.y), v[i][1], xp[j]);
-                                    xp[j] = fma(widen_down(f.z), v[i][2], xp[j]);
-                                    xp[j] = fma(widen_down(f.w), v[i][3], xp[j]);
+                                if (e < dv) {
+                                    float f[VW];
+                                    Slice<VW>::load(u + e * VW, f);
+#pragma unroll
+                                    for (int c = 0; c < VW; ++c) xp[j] = fma(widen_down(f[c]), v[i][c], xp[j]);
                                 }
                             }
                         }
@@ -224,11 +246,10 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                     for (int i = 0; i < NV; ++i) {
 #pragma unroll
                         for (int j = 0; j < NR; ++j) {
-                            const float4 f = stage[(size_t)j * stride4 + lane + 32 * i];
-                            acc[i][0] = fma(gw[j], widen_down(f.x), acc[i][0]);
-                            acc[i][1] = fma(gw[j], widen_down(f.y), acc[i][1]);
-                            acc[i][2] = fma(gw[j], widen_down(f.z), acc[i][2]);
-                            acc[i][3] = fma(gw[j], widen_down(f.w), acc[i][3]);
+                            float f[VW];
+                            Slice<VW>::load(stage + (size_t)j * stride + (lane + 32 * i) * VW, f);
+#pragma unroll
+                            for (int c = 0; c < VW; ++c) acc[i][c] = fma(gw[j], widen_down(f[c]), acc[i][c]);
                         }
                     }
                 } else {
@@ -236,16 +257,15 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
                     for (int j = 0; j < CR; ++j) {
                         const double gj = __shfl_sync(0xFFFFFFFFu, g, LPR * j) * kWidenUp;
                         if ((live >> j) & 1u) {
-                            const float4* __restrict__ u = stage + (size_t)j * stride4;
+                            const float* __restrict__ u = stage + (size_t)j * stride;
 #pragma unroll
                             for (int i = 0; i < NV; ++i) {
                                 const uint32_t e = lane + 32 * i;
-                                if (e < d4) {
-                                    const float4 f = u[e];
-                                    acc[i][0] = fma(gj, widen_down(f.x), acc[i][0]);
-                                    acc[i][1] = fma(gj, widen_down(f.y), acc[i][1]);
-                                    acc[i][2] = fma(gj, widen_down(f.z), acc[i][2]);
-                                    acc[i][3] = fma(gj, widen_down(f.w), acc[i][3]);
+                                if (e < dv) {
+                                    float f[VW];
+                                    Slice<VW>::load(u + e * VW, f);
+#pragma unroll
+                                    for (int c = 0; c < VW; ++c) acc[i][c] = fma(gj, widen_down(f[c]), acc[i][c]);
                                 }
                             }
                         }
@@ -254,13 +274,13 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d4, 
             }
         }
         if (failed) break;
-        double2* out = reinterpret_cast<double2*>(gin_pos + (size_t)(2 * q + side) * stride4 * 4);
+        double2* out = reinterpret_cast<double2*>(gin_pos + (size_t)(2 * q + side) * stride);
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
             const uint32_t e = lane + 32 * i;
-            if (e < d4) {
-                out[2 * e] = make_double2(acc[i][0], acc[i][1]);
-                out[2 * e + 1] = make_double2(acc[i][2], acc[i][3]);
+            if (e < dv) {
+#pragma unroll
+                for (int c = 0; c < VW; c += 2) out[(e * VW + c) / 2] = make_double2(acc[i][c], acc[i][c + 1]);
             }
         }
 #pragma unroll
@@ -288,9 +308,13 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     int blocks_per_sm = g_forward_blocks > 0 ? g_forward_blocks : (cr == 16 ? 5 : cr == 8 ? 8 : 10);
     // rows staged per chunk: as many of the cr as fit the shared memory share of one block
     uint32_t chunk_rows = s.K1 < (uint32_t)cr ? s.K1 : (uint32_t)cr;
-    // a warp's buffer ends with padding up to slice 32 * NV of its last row (see the kernel)
-    const uint32_t nv = s.d4 <= 32 ? 1 : s.d4 <= 64 ? 2 : s.d4 <= 96 ? 3 : s.d4 <= 128 ? 4 : 8;
-    const size_t pad = 32u * nv * 16 > row ? 32u * nv * 16 - row : 0;
+    // Slices of 2 floats where they leave fewer lanes idle than slices of 4 (an odd number of rounds of 64 floats,
+    // up to 7 of them); nv = rounds of 32 lanes.
+    const uint32_t rounds2 = (s.d / 2 + 31) / 32, rounds4 = (s.d4 + 31) / 32;
+    const int vw = rounds2 * 2 < rounds4 * 4 && rounds2 <= 7 ? 2 : 4;
+    const uint32_t nv = vw == 2 ? rounds2 : (rounds4 <= 4 ? rounds4 : 8);
+    // a warp's buffer ends with padding up to slice 32 * nv of its last row (see the kernel)
+    const size_t pad = 32u * nv * vw * 4 > row ? 32u * nv * vw * 4 - row : 0;
     // Whole chunks first: the loops without predicates need all cr rows staged, and they are worth more than
     // resident blocks (measured at d = 512: 6 blocks of whole chunks 0.89 ms, 8 blocks of 6-row chunks 1.15 ms).
     auto fits = [&](uint32_t rows_, int blocks_) {
@@ -300,25 +324,22 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
         while (blocks_per_sm > 2 && !fits(chunk_rows, blocks_per_sm)) --blocks_per_sm;
     const size_t budget = (size_t)216 * 1024 / blocks_per_sm - 1024;
     while (chunk_rows > 1 && (size_t)kFwdWarps * (chunk_rows * row + pad) + kFwdWarps * 8 > budget) --chunk_rows;
-    const uint32_t warp_stage4 = (uint32_t)((chunk_rows * row + pad) / 16);
-    const size_t smem = (size_t)kFwdWarps * warp_stage4 * 16 + kFwdWarps * 8;
+    const uint32_t warp_stage = (uint32_t)((chunk_rows * row + pad) / 4);
+    const size_t smem = (size_t)kFwdWarps * warp_stage * 4 + kFwdWarps * 8;
     if (smem > 200 * 1024) return cudaErrorInvalidConfiguration;
-    const uint32_t stride4 = s.stride / 4;
-    const float4* t4 = reinterpret_cast<const float4*>(table);
     uint32_t blocks = (2 * n + kFwdWarps - 1) / kFwdWarps;
     const uint32_t resident = (uint32_t)(L.sms * blocks_per_sm);
     if (blocks > resident) blocks = resident;
     Timed timed(L, K_FORWARD);
-#define TENSAIR_FWD(NV, CR)  TENSAIR_FWD_NR(NV, CR, CR)
-#define TENSAIR_FWD_NR(NV, CR, NR)                                                                                  \
+#define TENSAIR_FWD(NV, CR, NR, VW)                                                                                 \
     do {                                                                                                            \
         static bool attr_set = false;                                                                               \
         static int room_for = 0;                                                                                    \
         if (!attr_set) {                                                                                            \
-            cudaFuncSetAttribute(k_forward<NV, CR, NR>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024);   \
-            cudaFuncSetAttribute(k_forward<NV, CR, NR>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);       \
+            cudaFuncSetAttribute(k_forward<NV, CR, NR, VW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); \
+            cudaFuncSetAttribute(k_forward<NV, CR, NR, VW>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);   \
             cudaFuncAttributes fa;                                                                                  \
-            if (cudaFuncGetAttributes(&fa, k_forward<NV, CR, NR>) == cudaSuccess && fa.numRegs > 0)                 \
+            if (cudaFuncGetAttributes(&fa, k_forward<NV, CR, NR, VW>) == cudaSuccess && fa.numRegs > 0)             \
                 room_for = (65536 - kRegistersLeftForTheSort) / (fa.numRegs * kFwdWarps * 32);                      \
             attr_set = true;                                                                                        \
         }                                                                                                           \
@@ -326,20 +347,33 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
         if (g_forward_blocks <= 0 && grid_shape().overlap_sort && room_for >= 1 &&                                  \
             grid > (uint32_t)(L.sms * room_for))                                                                    \
             grid = (uint32_t)(L.sms * room_for);                                                                    \
-        k_forward<NV, CR, NR><<<grid, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d4, stride4, s.w, s.k,       \
-                                                                        chunk_rows, warp_stage4, t4, rows, rec,     \
-                                                                        gin_pos, loss_pos, err, owned, n_owned);    \
+        k_forward<NV, CR, NR, VW><<<grid, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d, s.stride, s.w, s.k,   \
+                                                                            chunk_rows, warp_stage, table, rows,    \
+                                                                            rec, gin_pos, loss_pos, err, owned,     \
+                                                                            n_owned);                               \
     } while (0)
     // k = 5 (six rows per pair) is common enough to have whole chunks of its own
-#define TENSAIR_FWD_NV(NV) do { if (cr == 16) TENSAIR_FWD(NV, 16); else if (cr == 8 && chunk_rows == 6) TENSAIR_FWD_NR(NV, 8, 6); else if (cr == 8) TENSAIR_FWD(NV, 8); else TENSAIR_FWD(NV, 4); } while (0)
-    if (s.d4 <= 32) TENSAIR_FWD_NV(1);
-    else if (s.d4 <= 64) TENSAIR_FWD_NV(2);
-    else if (s.d4 <= 96) TENSAIR_FWD_NV(3);
-    else if (s.d4 <= 128) TENSAIR_FWD_NV(4);
-    else TENSAIR_FWD_NV(8);
-#undef TENSAIR_FWD_NV
+#define TENSAIR_FWD_ROWS(NV, VW)                                                     \
+    do {                                                                             \
+        if (cr == 16) TENSAIR_FWD(NV, 16, 16, VW);                                   \
+        else if (cr == 8 && chunk_rows == 6) TENSAIR_FWD(NV, 8, 6, VW);              \
+        else if (cr == 8) TENSAIR_FWD(NV, 8, 8, VW);                                 \
+        else TENSAIR_FWD(NV, 4, 4, VW);                                              \
+    } while (0)
+    if (vw == 2) {
+        if (nv == 1) TENSAIR_FWD_ROWS(1, 2);
+        else if (nv == 3) TENSAIR_FWD_ROWS(3, 2);
+        else if (nv == 5) TENSAIR_FWD_ROWS(5, 2);
+        else TENSAIR_FWD_ROWS(7, 2);
+    } else {
+        if (nv == 1) TENSAIR_FWD_ROWS(1, 4);
+        else if (nv == 2) TENSAIR_FWD_ROWS(2, 4);
+        else if (nv == 3) TENSAIR_FWD_ROWS(3, 4);
+        else if (nv == 4) TENSAIR_FWD_ROWS(4, 4);
+        else TENSAIR_FWD_ROWS(8, 4);
+    }
+#undef TENSAIR_FWD_ROWS
 #undef TENSAIR_FWD
-#undef TENSAIR_FWD_NR
     return cudaGetLastError();
 }
 
