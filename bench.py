@@ -9,8 +9,8 @@ applies the messages that are due.  The default workload is the V = 1M, d = 300,
 
 One JSON line is printed by rank 0.  `value` is measured with the batches already in device memory;
 `e2e` is the same metric through tensair_train_batch_host with the batches in pinned host memory and
-the loss and message header read back every call.  `roofline` describes the kernel with the largest
-share of device time, timed with CUDA events inside the library in a separate pass.  `cpu_baseline`
+every replica's loss copied back (tensair_read_loss_async) and read after the step's one synchronisation.
+`roofline` describes the kernel with the largest share of device time, timed with CUDA events inside the library in a separate pass.  `cpu_baseline`
 is the CPU oracle timed on a bounded sample of the same workload on this host's cores.
 
 `--impl reference` times the CPU oracle alone (the only "reference" there is: the paper ships no code).
@@ -183,17 +183,21 @@ def run_sharded(args):
     grp = ShardedReplicas(ctx, rank, world, Wl, dist if world > 1 else None, count_device="cuda")
     toks_dev = torch.from_numpy(toks_np).cuda()
     toks_pin = torch.from_numpy(toks_np).pin_memory()
+    losses_pin = torch.zeros(Wl, dtype=torch.float64).pin_memory()
 
     def step(t, host=False):
         if wl.drift_every and t and t % wl.drift_every == 0:
             ctx.tensair_update_sampler()
         for r in range(Wl):
             if host:
-                ctx.tensair_train_batch_host(r, toks_pin[t, r], t, want_loss=True)
+                ctx.tensair_train_batch_host(r, toks_pin[t, r], t)
+                ctx.tensair_read_loss_async(losses_pin.data_ptr() + 8 * r)
             else:
                 ctx.tensair_train_batch(r, toks_dev[t, r], t)
         grp.exchange(t)
         grp.apply(t)
+        if host and ctx.tensair_sync() != B.OK:      # the step's one synchronisation: the losses are in losses_pin now
+            raise SystemExit("the device reported a bad token during the benchmark")
 
     def barrier():
         torch.cuda.synchronize()
@@ -243,7 +247,7 @@ def run_sharded(args):
                    "l2": "inputs larger than L2 (tables %.1f GB per GPU)" % (ctx.sizes.tables_bytes / 1e9),
                    "parallelism": f"{Wl} of {wl.W} replicas per GPU, every message broadcast into every GPU's pool"},
         "e2e": {"value": wl.W * P * K / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e / K,
-                "h2d_bytes_per_step": Wl * wl.batch * 4, "d2h_bytes_per_step": Wl * (8 + 16 + 4)},
+                "h2d_bytes_per_step": Wl * wl.batch * 4, "d2h_bytes_per_step": Wl * 8 + 4},
         "gpu_launches": int(launches),
         "exchange": {"bytes_sent_per_step_per_gpu": int(sent / K), "transport": "NCCL broadcast per message" if world > 1 else "none (one rank)"},
         "clocks": sampler.summary(wall0, wall1),
@@ -284,6 +288,8 @@ def run_ours(args):
                     max_grad_buffer=wl.max_grad_buffer)
     toks_dev = torch.from_numpy(toks_np).cuda()
     toks_pin = torch.from_numpy(toks_np).pin_memory()
+    losses_pin = torch.zeros(wl.W, dtype=torch.float64).pin_memory()
+    step_losses = []
     n_rows = {}
 
     msg_ids = {}
@@ -297,7 +303,9 @@ def run_ours(args):
                 _, inf = ctx.tensair_train_batch_routed(i, shared if host else toks_dev[t, 0], t, want_loss=host,
                                                         want_info=host or info)
             elif host:
-                _, inf = ctx.tensair_train_batch_host(i, toks_pin[t, i], t, want_loss=True, want_info=True)
+                # the loss of every replica travels back asynchronously; the step ends with one synchronisation
+                _, inf = ctx.tensair_train_batch_host(i, toks_pin[t, i], t)
+                ctx.tensair_read_loss_async(losses_pin.data_ptr() + 8 * i)
             else:
                 _, inf = ctx.tensair_train_batch(i, toks_dev[t, i], t, want_info=info)
             if inf is not None:
@@ -309,6 +317,10 @@ def run_ours(args):
                 ctx.tensair_apply_messages(j, t)
         else:
             ctx.tensair_apply_step(t)                         # all replicas' due messages in one pass
+        if host and not wl.routed:
+            if ctx.tensair_sync() != B.OK:
+                raise SystemExit("the device reported a bad token during the benchmark")
+            step_losses.append(float(losses_pin.sum()))
 
     def barrier():
         torch.cuda.synchronize()
@@ -497,7 +509,7 @@ def run_ours(args):
                    "pairs_per_batch": P, "storage": "f32", "l2": "inputs larger than L2 (tables %.1f GB)" %
                    (ctx.sizes.tables_bytes / 1e9), "parallelism": f"{world} independent replica groups"},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / K,
-                "h2d_bytes_per_step": (1 if wl.routed else wl.W) * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4)},
+                "h2d_bytes_per_step": (1 if wl.routed else wl.W) * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4) if wl.routed else wl.W * 8 + 4},
         "gpu_launches": int(launches),
         "clocks": sampler.summary(wall0, wall1),
         "roofline": roofline,

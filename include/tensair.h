@@ -308,6 +308,12 @@ TENSAIR_API int tensair_drain(tensair_ctx* ctx, uint32_t* n_applied);
  * and the call synchronises.) */
 TENSAIR_API int tensair_update_sampler(tensair_ctx* ctx);
 
+/* The loss of the most recent tensair_train_batch* call without waiting for it: enqueues, on the context's
+ * stream, a copy of the batch loss (sum of the pair losses) into host_dst (host, double; pinned memory for the
+ * copy to be asynchronous).  The value is there once the stream has passed the copy, e.g. after tensair_sync;
+ * one synchronisation per step can so serve the losses of all replicas.  host_dst must stay valid until then. */
+TENSAIR_API int tensair_read_loss_async(tensair_ctx* ctx, double* host_dst);
+
 /* Waits for the stream; returns and clears a pending TENSAIR_EBADTOKEN. */
 TENSAIR_API int tensair_sync(tensair_ctx* ctx);
 

@@ -84,6 +84,7 @@ SYMBOLS = {
     "tensair_apply_step": (_int, [_vp, _u64, _P(_u32)]),
     "tensair_drain": (_int, [_vp, _P(_u32)]),
     "tensair_update_sampler": (_int, [_vp]),
+    "tensair_read_loss_async": (_int, [_vp, _vp]),
     "tensair_sync": (_int, [_vp]),
     "tensair_read_embeddings": (_int, [_vp, _u32, _int, _u32, _u32, _vp]),
     "tensair_write_embeddings": (_int, [_vp, _u32, _int, _u32, _u32, _vp]),
@@ -364,6 +365,10 @@ class Context:
 
     def tensair_update_sampler(self):
         _check(lib().tensair_update_sampler(self._h), "tensair_update_sampler", self._h)
+
+    def tensair_read_loss_async(self, host_ptr: int):
+        """Enqueues the copy of the last batch loss into the (pinned) host double at address host_ptr."""
+        _check(lib().tensair_read_loss_async(self._h, host_ptr), "tensair_read_loss_async", self._h)
 
     def tensair_sync(self) -> int:
         """Returns the status (OK or EBADTOKEN) instead of raising."""

@@ -578,6 +578,14 @@ int tensair_update_sampler(tensair_ctx* ctx) {
     return upload_sampler(ctx, counts.data());
 }
 
+int tensair_read_loss_async(tensair_ctx* ctx, double* host_dst) {
+    if (!ctx || !host_dst || !ctx->have_last) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    TENSAIR_CUDA(ctx, cudaMemcpyAsync(host_dst, ctx->at<double>(ctx->cv.loss), 8, cudaMemcpyDeviceToHost, ctx->stream));
+    return TENSAIR_OK;
+}
+
 int tensair_sync(tensair_ctx* ctx) {
     if (!ctx) return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);

@@ -75,6 +75,13 @@ ONE_BATCH = [
     ("w16_k2", synth.scaled(synth.TINY, V=3000, d=64, window=16, k=2, batch=600), True),
     ("V2_every_other_negative_dropped", synth.scaled(synth.TINY, V=2, d=8, window=2, k=3, batch=50), True),
     ("k40_d100", synth.scaled(synth.TINY, V=4000, d=100, window=2, k=40, batch=200, reduction=1), True),
+    # every width class of the forward kernel: slices of 2 floats in 3 and 7 rounds, slices of 4 in 2 and 3 rounds,
+    # with whole 8-row chunks (k = 7, 15), whole 6-row chunks (k = 5) and ragged ones (k = 9)
+    ("d192_k7", synth.scaled(synth.TINY, V=3000, d=192, window=3, k=7, batch=300, reduction=1), True),
+    ("d448_k5", synth.scaled(synth.TINY, V=3000, d=448, window=2, k=5, batch=300, reduction=1), True),
+    ("d256_k15", synth.scaled(synth.TINY, V=3000, d=256, window=2, k=15, batch=300, reduction=1), True),
+    ("d384_k9", synth.scaled(synth.TINY, V=3000, d=384, window=2, k=9, batch=300, reduction=1), True),
+    ("d36_stride40", synth.scaled(synth.TINY, V=3000, d=36, window=2, k=15, batch=300, reduction=1), True),
 ]
 
 
@@ -212,6 +219,23 @@ def test_host_and_device_entry_points_agree_bit_for_bit(torch):
     for which in (0, 1):
         assert np.array_equal(g1.tensair_read_embeddings(0, which).view(np.uint32),
                               g2.tensair_read_embeddings(0, which).view(np.uint32))
+
+
+def test_loss_read_back_without_waiting_equals_the_blocking_read(torch):
+    wl = synth.scaled(synth.MID, V=20_000, batch=1024, W=2, stream_seeds=(1, 2), batches=3)
+    streams = synth.all_streams(wl, 3)
+    _, g = make_pair(wl, counts=synth.stream_counts(streams, wl.V))
+    _, h = make_pair(wl, counts=synth.stream_counts(streams, wl.V))
+    pinned = torch.zeros(2 * 3, dtype=torch.float64).pin_memory()
+    want = []
+    for t in range(3):
+        for i in range(2):
+            want.append(g.tensair_train_batch(i, dev(torch, streams[i][t]), t, want_loss=True)[0])
+            h.tensair_train_batch(i, dev(torch, streams[i][t]), t)
+            h.tensair_read_loss_async(pinned.data_ptr() + 8 * (2 * t + i))
+        assert g.tensair_apply_step(t) == h.tensair_apply_step(t)
+    assert h.tensair_sync() == 0
+    assert pinned.tolist() == want
 
 
 def test_runs_are_bit_reproducible(torch):
