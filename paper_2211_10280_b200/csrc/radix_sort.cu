@@ -60,8 +60,8 @@ k_scan_digits(uint32_t* __restrict__ hist, uint32_t tiles, uint32_t* __restrict_
 // Stable scatter.  Warp w of a block owns the consecutive items [w*512, (w+1)*512) of the tile and
 // walks them 32 at a time; lanes with the same digit are ranked by lane order within a round and
 // rounds are ranked by their order, so the rank of an item among equal digits follows input order.
-// At most 64 registers per thread: a block then fits beside the resident blocks of the forward kernel, which the
-// sort runs next to (8 blocks of 64 threads and 96 registers leave 16 K registers per multiprocessor).
+// At most 64 registers per thread: a block of 256 threads then needs 16 K registers of a multiprocessor, which the
+// forward kernel, beside which the sort runs, leaves free when it sizes its grid.
 __global__ void __launch_bounds__(kSortThreads, 4)
 k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_t n, uint32_t shift,
                 const uint32_t* __restrict__ hist, uint32_t tiles, const uint32_t* __restrict__ totals) {
