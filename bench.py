@@ -124,6 +124,29 @@ def max_over_ranks(ms: float, dist, device) -> float:
     return float(x.item())
 
 
+MIN_TIMED_SECONDS = 2.0     # a K-step region is repeated until this much has been timed; the median region is reported
+MAX_REPEATS = 40
+
+
+def config_of(wl: synth.Workload, world: int, parallelism: str) -> dict:
+    """The `config` object of the JSON line: the same keys, from the workload alone, in both arms."""
+    stride = -(-wl.d // 8) * 8
+    return {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
+            "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
+            "max_grad_buffer": wl.max_grad_buffer,
+            "routing": "hash of the centre word, one batch shared by the replicas" if wl.routed else "one substream per replica",
+            "pairs_per_batch": wl.pairs_per_batch, "storage": "f32",
+            "l2": "inputs larger than L2 (tables %.1f GB)" % (wl.W * 2 * wl.V * stride * 4 / 1e9),
+            "parallelism": parallelism}
+
+
+def repeats_for(ms_one_region: float) -> int:
+    """How many K-step regions to time so that at least MIN_TIMED_SECONDS are covered."""
+    if ms_one_region <= 0:
+        return 1
+    return max(1, min(MAX_REPEATS, int(-(-MIN_TIMED_SECONDS * 1e3 // ms_one_region))))
+
+
 def pick_workload(name: str, override: str = "") -> synth.Workload:
     """A named workload, optionally with fields replaced (`--override V=250000,W=2`: reduced cases for profiling)."""
     if name not in synth.WORKLOADS:
@@ -140,6 +163,15 @@ def pick_workload(name: str, override: str = "") -> synth.Workload:
     return wl
 
 
+def stream_batches(wl: synth.Workload) -> int:
+    """Batches of the workload's stream kept for a run (the steps cycle through them): the whole stream up to 512,
+    a whole number of drift epochs when the workload drifts."""
+    nb = min(wl.batches, 512)
+    if wl.drift_every and nb > wl.drift_every:
+        nb -= nb % wl.drift_every
+    return nb
+
+
 def rank_streams(wl: synth.Workload, rank: int, batches: int):
     """Token batches [batches, W, B] of this rank and the unigram counts of its whole stream."""
     wl_r = synth.scaled(wl, stream_seeds=tuple(s + 1000 * rank for s in wl.stream_seeds))
@@ -151,10 +183,19 @@ def rank_streams(wl: synth.Workload, rank: int, batches: int):
 
 
 # ------------------------------------------------------------------------------------------------
+def sharded_workload(wl: synth.Workload, world: int):
+    """The workload as N processes run it: its W replicas spread evenly when N divides W (the one-GPU job, total work
+    fixed: "strong"); otherwise one replica per GPU, W = N, the stream seeds continued (work per GPU fixed apart from
+    the messages to apply, which grow with N: "weak")."""
+    if wl.W % world == 0:
+        return wl, wl.W // world, "strong"
+    seeds = tuple(wl.stream_seeds[0] + i for i in range(world))
+    return synth.scaled(wl, name=f"{wl.name}[W={world}]", W=world, stream_seeds=seeds), 1, "weak"
+
+
 def run_sharded(args):
-    """`--sharded`: the workload's W replicas spread over the ranks (W / N per GPU), every message broadcast into
-    every rank's pool over NCCL (paper_2211_10280_b200/exchange.py).  The job computes what the one-GPU job
-    computes, so the total work is fixed as N grows ("strong")."""
+    """The paper's placement: the replicas spread over the ranks, one group per GPU, every message broadcast into
+    every rank's pool over NCCL on a communication stream (paper_2211_10280_b200/exchange.py)."""
     import torch
     import torch.distributed as dist
 
@@ -168,14 +209,15 @@ def run_sharded(args):
         raise SystemExit("bench.py needs a CUDA device: the SGNS path has no CPU implementation")
     torch.cuda.set_device(local)
     if world > 1:
+        os.environ.setdefault("NCCL_DEBUG", "INFO")      # the communicator log shows the ranks and the transport
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     wl = pick_workload(args.workload, args.override)
-    if wl.W % world or wl.routed or wl.max_grad_buffer != 1:
-        raise SystemExit(f"--sharded needs a workload whose {wl.W} replicas divide over {world} ranks, unrouted, maxGradBuffer 1")
-    Wl = wl.W // world
+    if wl.routed or wl.max_grad_buffer != 1:
+        raise SystemExit("the sharded placement needs an unrouted workload with maxGradBuffer 1")
+    wl, Wl, scaling = sharded_workload(wl, world)
     K, Wm = args.steps, max(args.warmup, 3)
-    total_steps = 2 * (Wm + K)
-    toks_all, counts = rank_streams(wl, 0, total_steps)          # the one-GPU job's streams; this rank takes its replicas'
+    nb = stream_batches(wl)
+    toks_all, counts = rank_streams(wl, 0, nb)                   # the one-process job's streams; this rank takes its replicas'
     toks_np = np.ascontiguousarray(toks_all[:, rank * Wl:(rank + 1) * Wl])
     ctx = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=Wl, lr=wl.lr, max_delay=wl.max_delay,
                     seed=wl.seed, counts=counts, device=local, reduction=wl.reduction, world_replicas=wl.W,
@@ -186,18 +228,19 @@ def run_sharded(args):
     losses_pin = torch.zeros(Wl, dtype=torch.float64).pin_memory()
 
     def step(t, host=False):
+        b = t % nb
         if wl.drift_every and t and t % wl.drift_every == 0:
             ctx.tensair_update_sampler()
         for r in range(Wl):
             if host:
-                ctx.tensair_train_batch_host(r, toks_pin[t, r], t)
+                ctx.tensair_train_batch_host(r, toks_pin[b, r], t)
                 ctx.tensair_read_loss_async(losses_pin.data_ptr() + 8 * r)
             else:
-                ctx.tensair_train_batch(r, toks_dev[t, r], t)
-        grp.exchange(t)
-        grp.apply(t)
+                ctx.tensair_train_batch(r, toks_dev[b, r], t)
+        grp.exchange(t)                                          # transfers start on the communication stream
+        grp.apply(t)                                             # waits only for what is due here at step t
         if host and ctx.tensair_sync() != B.OK:      # the step's one synchronisation: the losses are in losses_pin now
-            raise SystemExit("the device reported a bad token during the benchmark")
+            raise SystemExit("the device reported an error during the benchmark: " + ctx.tensair_last_error())
 
     def barrier():
         torch.cuda.synchronize()
@@ -217,6 +260,19 @@ def run_sharded(args):
         ms = ev0.elapsed_time(ev1)
         return (max_over_ranks(ms, dist, "cuda") if world > 1 else ms), wall0, time.time()
 
+    def timed_regions(first, host):
+        ms0, wall0, wall1 = timed(first, host)
+        first += K
+        regions = [ms0]
+        reps = repeats_for(ms0)
+        if world > 1:
+            reps = int(max_over_ranks(float(reps), dist, "cuda"))
+        for _ in range(reps - 1):
+            ms, _, wall1 = timed(first, host)
+            first += K
+            regions.append(ms)
+        return statistics.median(regions), regions, wall0, wall1, first
+
     uuid = str(torch.cuda.get_device_properties(local).uuid)
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
     t = 0
@@ -226,30 +282,35 @@ def run_sharded(args):
     sampler.start()
     time.sleep(0.3)
     launches0, sent0 = ctx.tensair_kernel_launches(), grp.bytes_sent
-    ms_dev, wall0, wall1 = timed(t, host=False)
-    launches, sent = ctx.tensair_kernel_launches() - launches0, grp.bytes_sent - sent0
+    ms_dev, regions_dev, wall0, wall1, t = timed_regions(t, host=False)
+    launches = (ctx.tensair_kernel_launches() - launches0) // len(regions_dev)
+    sent = (grp.bytes_sent - sent0) / (len(regions_dev) * K)
     sampler.stop()
-    t += K
     for _ in range(Wm):
         step(t, host=True)
         t += 1
-    ms_e2e, _, _ = timed(t, host=True)
+    ms_e2e, regions_e2e, _, _, t = timed_regions(t, host=True)
     if ctx.tensair_sync() != B.OK:
-        raise SystemExit("the device reported a bad token during the benchmark")
+        raise SystemExit("the device reported an error during the benchmark: " + ctx.tensair_last_error())
     P = wl.pairs_per_batch
+    placement = (f"{Wl} of {wl.W} replicas per GPU, every message broadcast into every GPU's pool on a communication stream"
+                 if world > 1 else f"all {wl.W} replicas on one GPU (sharded code path, nothing to exchange)")
     out = {
         "metric": METRIC, "value": wl.W * P * K / (ms_dev * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
-        "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "strong", "vs_baseline": None,
+        "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": scaling, "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
-                   "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
-                   "pairs_per_batch": P, "storage": "f32",
-                   "l2": "inputs larger than L2 (tables %.1f GB per GPU)" % (ctx.sizes.tables_bytes / 1e9),
-                   "parallelism": f"{Wl} of {wl.W} replicas per GPU, every message broadcast into every GPU's pool"},
-        "e2e": {"value": wl.W * P * K / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e / K,
+        "config": config_of(wl, world, placement),
+        "timing": {"regions": len(regions_dev), "steps_per_region": K, "reported": "median region",
+                   "ms_per_step_min": round(min(regions_dev) / K, 5), "ms_per_step_max": round(max(regions_dev) / K, 5),
+                   "timed_seconds": round(sum(regions_dev) / 1e3, 3)},
+        "e2e": {"value": wl.W * P * K / (ms_e2e * 1e-3), "unit": UNIT, "ms_per_step": ms_e2e / K, "regions": len(regions_e2e),
                 "h2d_bytes_per_step": Wl * wl.batch * 4, "d2h_bytes_per_step": Wl * 8 + 4},
         "gpu_launches": int(launches),
-        "exchange": {"bytes_sent_per_step_per_gpu": int(sent / K), "transport": "NCCL broadcast per message" if world > 1 else "none (one rank)"},
+        "exchange": {"bytes_sent_per_step_per_gpu": int(sent),
+                     "transport": "NCCL broadcast per message on a communication stream" if world > 1 else "none (one rank)",
+                     "received_bytes_waited_for_at_their_own_step": int(grp.bytes_waited_at_own_step),
+                     "received_bytes_that_travelled_during_later_batches": int(grp.bytes_waited_later),
+                     "hidden_share": round(grp.hidden_share(), 4)},
         "clocks": sampler.summary(wall0, wall1),
     }
     ctx.close()
@@ -279,8 +340,8 @@ def run_ours(args):
         B.tensair_tune(item.split("=")[0], int(item.split("=")[1]))
     K, Wm = args.steps, max(args.warmup, 3)
     Kp = min(K, 8)                                          # steps of the per-kernel timing pass
-    total_steps = 2 * (Wm + K) + Kp + wl.max_delay
-    toks_np, counts = rank_streams(wl, rank, total_steps)
+    nb = stream_batches(wl)                                 # batches held; step t trains batch t mod nb
+    toks_np, counts = rank_streams(wl, rank, nb)
     P = wl.pairs_per_batch
 
     ctx = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=wl.W, lr=wl.lr,
@@ -297,17 +358,18 @@ def run_ours(args):
     def step(t, host=False, info=False):
         if wl.drift_every and t and t % wl.drift_every == 0:
             ctx.tensair_update_sampler()                      # passive drift adaptation: the sampler follows the stream
-        shared = toks_pin[t, 0].to("cuda", non_blocking=True) if (wl.routed and host) else None
+        b = t % nb
+        shared = toks_pin[b, 0].to("cuda", non_blocking=True) if (wl.routed and host) else None
         for i in range(wl.W):
             if wl.routed:       # one batch for all replicas, split by the hash of the centre word
-                _, inf = ctx.tensair_train_batch_routed(i, shared if host else toks_dev[t, 0], t, want_loss=host,
+                _, inf = ctx.tensair_train_batch_routed(i, shared if host else toks_dev[b, 0], t, want_loss=host,
                                                         want_info=host or info)
             elif host:
                 # the loss of every replica travels back asynchronously; the step ends with one synchronisation
-                _, inf = ctx.tensair_train_batch_host(i, toks_pin[t, i], t)
+                _, inf = ctx.tensair_train_batch_host(i, toks_pin[b, i], t)
                 ctx.tensair_read_loss_async(losses_pin.data_ptr() + 8 * i)
             else:
-                _, inf = ctx.tensair_train_batch(i, toks_dev[t, i], t, want_info=info)
+                _, inf = ctx.tensair_train_batch(i, toks_dev[b, i], t, want_info=info)
             if inf is not None:
                 n_rows[(i, t)] = (inf.n_rows, inf.n_in_rows)
             if info or args.log_applies:
@@ -343,6 +405,21 @@ def run_ours(args):
             ms = max_over_ranks(ms, dist, "cuda")
         return ms, wall0, wall1
 
+    def timed_regions(first, host):
+        """K-step regions back to back until MIN_TIMED_SECONDS are covered: (median ms of a region, all of them,
+        wall-clock bounds, the step after the last)."""
+        ms0, wall0, wall1 = timed(first, host)
+        first += K
+        regions = [ms0]
+        reps = repeats_for(ms0)
+        if world > 1:                                        # every rank must time the same number of regions
+            reps = int(max_over_ranks(float(reps), dist, "cuda"))
+        for _ in range(reps - 1):
+            ms, _, wall1 = timed(first, host)
+            first += K
+            regions.append(ms)
+        return statistics.median(regions), regions, wall0, wall1, first
+
     uuid = str(torch.cuda.get_device_properties(local).uuid)
     sampler = ClockSampler(uuid if uuid.startswith("GPU-") else "GPU-" + uuid)
     t = 0
@@ -352,15 +429,13 @@ def run_ours(args):
     sampler.start()
     time.sleep(0.3)
     launches0 = ctx.tensair_kernel_launches()
-    ms_dev, wall0, wall1 = timed(t, host=False)
-    launches = ctx.tensair_kernel_launches() - launches0
+    ms_dev, regions_dev, wall0, wall1, t = timed_regions(t, host=False)
+    launches = (ctx.tensair_kernel_launches() - launches0) // len(regions_dev)
     sampler.stop()
-    t += K
     for _ in range(Wm):
         step(t, host=True)
         t += 1
-    ms_e2e, _, _ = timed(t, host=True)
-    t += K
+    ms_e2e, regions_e2e, _, _, t = timed_regions(t, host=True)
 
     # per-kernel pass: CUDA events around every launch, on the library's stream
     for _ in range(wl.max_delay):                            # so that every message applied below has its ids on record
@@ -503,12 +578,11 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
-                   "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
-                   "max_grad_buffer": wl.max_grad_buffer, "routing": "hash of the centre word, one batch shared by the replicas" if wl.routed else "one substream per replica",
-                   "pairs_per_batch": P, "storage": "f32", "l2": "inputs larger than L2 (tables %.1f GB)" %
-                   (ctx.sizes.tables_bytes / 1e9), "parallelism": f"{world} independent replica groups"},
-        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / K,
+        "config": config_of(wl, world, f"{world} independent replica group{'s' if world > 1 else ''}, no exchange between them"),
+        "timing": {"regions": len(regions_dev), "steps_per_region": K, "reported": "median region",
+                   "ms_per_step_min": round(min(regions_dev) / K, 5), "ms_per_step_max": round(max(regions_dev) / K, 5),
+                   "timed_seconds": round(sum(regions_dev) / 1e3, 3)},
+        "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / K, "regions": len(regions_e2e),
                 "h2d_bytes_per_step": (1 if wl.routed else wl.W) * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4) if wl.routed else wl.W * 8 + 4},
         "gpu_launches": int(launches),
         "clocks": sampler.summary(wall0, wall1),
@@ -567,6 +641,8 @@ def run_reference(args):
     import oracle
 
     wl = pick_workload(args.workload, args.override)
+    if world > 1 and not args.replicas_only:
+        wl = sharded_workload(wl, world)[0]                 # the workload the N-rank arm runs
     K, Wm = args.steps, args.warmup
     total = Wm + K
     toks_np, counts = rank_streams(wl, 0, -(-total // wl.W) + 1)
@@ -592,9 +668,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": Wm, "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
-                   "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
-                   "pairs_per_batch": wl.pairs_per_batch},
+        "config": config_of(wl, world, "CPU oracle on rank 0's host cores, all replicas in one process"),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
@@ -628,18 +702,39 @@ def run_sweep(args):
         ev1.record()
         torch.cuda.synchronize()
         ms = ev0.elapsed_time(ev1) / steps
+        launches = ctx.tensair_kernel_launches()
         _, info = ctx.tensair_train_batch(0, toks[3 + steps], 3 + steps, want_info=True)
+        launches = ctx.tensair_kernel_launches() - launches
         U = float(np.mean(rows + [info.n_rows]))
         row = 4 * wl.d
         own = U * row + U * (row + 4) + U * (row + 4 + 2 * row)
-        print(json.dumps({"workload": wl.name, "d": wl.d, "batch": wl.batch, "k": wl.k, "pairs_per_batch": wl.pairs_per_batch,
-                          "rows_per_message": int(U), "ms_per_batch": round(ms, 4),
-                          "pairs_per_s": wl.pairs_per_batch / (ms * 1e-3), "algorithmic_gbs": round(own / (ms * 1e-3) / 1e9, 1),
-                          "frac_of_peak": round(own / (ms * 1e-3) / 1e9 / peak, 4), "peak": f"{peak} GB/s of {peak_kind}"}),
-              flush=True)
+        # nominal model: every contribution's row fetched once by the gradient calculation and its centre row once by
+        # the row sums (what the kernels request from L2; the distinct rows are what must come from DRAM)
+        nominal = 2.0 * wl.pairs_per_batch * (wl.k + 1) * row + U * (row + 4) + U * 2 * row
+        line = {"workload": wl.name, "d": wl.d, "batch": wl.batch, "k": wl.k, "pairs_per_batch": wl.pairs_per_batch,
+                "rows_per_message": int(U), "ms_per_batch": round(ms, 4), "launches_per_batch": int(launches),
+                "pairs_per_s": wl.pairs_per_batch / (ms * 1e-3), "algorithmic_gbs": round(own / (ms * 1e-3) / 1e9, 1),
+                "frac_of_peak": round(own / (ms * 1e-3) / 1e9 / peak, 4), "peak": f"{peak} GB/s of {peak_kind}",
+                "nominal_gbs": round(nominal / (ms * 1e-3) / 1e9, 1)}
+        if not args.no_cpu_baseline:
+            line["cpu_baseline"] = cpu_baseline(wl, stream[:, None, :], counts, steps=3)
+        print(json.dumps(line), flush=True)
         ctx.close()
         del ctx, toks
         torch.cuda.empty_cache()
+
+
+def launch_ranks(n: int, argv) -> int:
+    """Runs this script as n ranks on one node under torch.distributed.run (rendezvous on 127.0.0.1, a free port)."""
+    import socket
+
+    with socket.socket() as sock:
+        sock.bind(("127.0.0.1", 0))
+        port = sock.getsockname()[1]
+    env = dict(os.environ, MASTER_ADDR="127.0.0.1")
+    cmd = [sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={n}",
+           "--master-addr", "127.0.0.1", "--master-port", str(port), str(Path(__file__).resolve()), *argv]
+    return subprocess.call(cmd, env=env)
 
 
 def main():
@@ -657,14 +752,20 @@ def main():
     ap.add_argument("--apply-per-replica", action="store_true",
                     help="apply the due messages with one tensair_apply_messages call per replica instead of tensair_apply_step")
     ap.add_argument("--sharded", action="store_true",
-                    help="spread the workload's replicas over the ranks and exchange their messages (strong scaling)")
+                    help="the paper's placement: replicas spread over the ranks, messages exchanged (the default with --gpus > 1)")
+    ap.add_argument("--replicas-only", action="store_true",
+                    help="with --gpus > 1: N independent copies of the one-GPU job instead of the sharded placement")
     args = ap.parse_args()
+    if args.gpus > 1 and "RANK" not in os.environ:
+        # not started by a launcher: start the N ranks here, one per GPU, and hand on their exit status
+        sys.exit(launch_ranks(args.gpus, sys.argv[1:]))
+    world = int(os.environ.get("WORLD_SIZE", "1"))
     if args.sweep:
         run_sweep(args)
-    elif args.sharded and args.impl == "ours":
-        run_sharded(args)
     elif args.impl == "reference":
         run_reference(args)
+    elif args.sharded or (world > 1 and not args.replicas_only):
+        run_sharded(args)
     else:
         run_ours(args)
 

@@ -65,7 +65,11 @@ enum {
     TENSAIR_ECUDA = -3,     /* a CUDA call failed; see tensair_last_error */
     TENSAIR_EBADTOKEN = -4, /* a batch held a token id outside [0,V) */
     TENSAIR_EPENDING = -5,  /* a message slot still has undelivered recipients */
-    TENSAIR_ENOTFOUND = -6  /* the requested message is no longer held */
+    TENSAIR_ENOTFOUND = -6, /* the requested message is no longer held */
+    TENSAIR_ETIMEOUT = -7,  /* a bounded wait inside a kernel ran out (a warp's own bulk copies did not land);
+                               the batch it belonged to is incomplete */
+    TENSAIR_EBOUNDS = -8    /* an index checked on the device was outside its array (checked builds), or a merged
+                               message outgrew its slot; the access was skipped, nothing was written out of place */
 };
 
 /* Model, batch and exchange shape (Algorithm 1's constructor arguments plus the SGNS shape). */
@@ -91,7 +95,9 @@ typedef struct tensair_sizes {
     uint64_t scratch_bytes;   /* sort buffers, gradient scalars, partial sums, sampler table, counts */
     uint32_t row_stride;      /* the stride the library will use */
     uint32_t max_pairs;       /* pairs of a full batch: 2*w*batch - w*(w+1) when batch > w */
-    uint32_t max_rows;        /* most rows a message can have */
+    uint32_t max_rows;        /* most rows a sent message can have (the capacity of a pool slot): distinct input rows
+                                 <= min(m * batch, V) plus distinct output rows <= min(m * contributions, V),
+                                 m = max_grad_buffer */
     uint32_t reserved;
 } tensair_sizes;
 
@@ -155,7 +161,8 @@ TENSAIR_API int tensair_init(const tensair_config* cfg, const tensair_buffers* b
  *     tensair_message_buffers names (any transport: an NCCL broadcast or all-gather straight into the pool),
  *     tensair_commit_message each, then tensair_apply_messages for the local replicas and tensair_shadow_apply
  *     for the others.
- * tensair_workspace_bytes_sharded sizes the pool for world_W senders.  max_grad_buffer must be 1.
+ * tensair_workspace_bytes_sharded sizes the pool for world_W senders.  With world_W > cfg->W max_grad_buffer
+ * must be 1 (TENSAIR_EINVAL otherwise): buffered gradients are merged only inside one process.
  * world_W == cfg->W and first_replica == 0 is tensair_init.
  */
 TENSAIR_API int tensair_workspace_bytes_sharded(const tensair_config* cfg, uint32_t world_W, tensair_sizes* out);
@@ -171,6 +178,8 @@ typedef struct tensair_msg_view {
     uint32_t row_stride;      /* floats between consecutive delta rows */
     uint64_t ids_offset;      /* byte offsets of the two arrays in the pool buffer given at init */
     uint64_t delta_offset;
+    uint64_t header_offset;   /* byte offset of the slot's header: uint32 n_rows, uint32 n_in_rows (written on the
+                                 device by the kernels that build the message; valid once the stream passed them) */
 } tensair_msg_view;
 /*
  * The "wire" of send_gradients (Algorithm 1) between processes.  Host-only, no synchronisation.
@@ -192,6 +201,17 @@ TENSAIR_API int tensair_message_rows(tensair_ctx* ctx, uint32_t replica, uint64_
  */
 TENSAIR_API int tensair_commit_message(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, uint32_t n_rows,
                                        uint32_t n_in_rows);
+/*
+ * The same with the header write and the bucket index enqueued on `stream` (a cudaStream_t of the context's device;
+ * NULL = the context's stream) instead of the context's stream: for a caller that receives messages on a
+ * communication stream of its own while the context's stream keeps training (Section 3.1: a Model goes on computing
+ * while gradients arrive).  The entry in the delivery schedule is made at once, on the host, so the order of
+ * these calls relative to the train and apply calls is what fixes delivery order and staleness, as before.  The
+ * caller orders the streams: `stream` must have received the rows before this call, and the context's stream must
+ * wait for `stream` (an event recorded after this call) before the first apply call at which the message is due.
+ */
+TENSAIR_API int tensair_commit_message_on(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, uint32_t n_rows,
+                                          uint32_t n_in_rows, void* stream);
 /*
  * Book-keeping of a REMOTE receiver: marks what is due for it at `step` (or everything, drain != 0) as applied,
  * which the process holding that replica does for real.  Keeps slot reuse and the staleness of Section 3.1
@@ -258,17 +278,25 @@ TENSAIR_API int tensair_route(uint64_t seed, uint32_t W, uint32_t token, uint32_
  * handed its tables and message pool by a host application with a fixed memory plan, or a service
  * thread that must stay out of the allocator.  (The paper has no counterpart: this is an addition of
  * this library.)  Arguments, results, error codes and the filing of the message are those of
- * tensair_train_batch, and the result is bit-identical to it.  The difference: the per-batch working
- * memory (sort buffers, segment lists, partial sums) is not taken from the scratch buffer given at
- * tensair_init but from a fixed 32 MiB array inside the library image, which every GPU that loads the
- * library reserves until the process exits.  The call allocates nothing on the device, neither
- * directly nor through a library.
+ * tensair_train_batch, and the result is bit-identical to it.  The difference: part of the per-batch
+ * working memory is not taken from the scratch buffer given at tensair_init but from a fixed 32 MiB
+ * array inside the library image, which every GPU that loads the library reserves until the process
+ * exits.  Taken from the array: the two sort buffers, the sorted terms, the partial centre gradients and
+ * losses per position, the radix histograms, the segment starts, the long-row lists and their chunk
+ * partials.  Still in the context's scratch (it exists anyway, tensair_init needed it): the error word,
+ * the loss, the running counts, the sampler table, the per-contribution row ids and gradient scalars.
+ * The call allocates nothing on the device, neither directly nor through a library.
  *   - Only for max_grad_buffer = 1 (TENSAIR_EINVAL otherwise).
  *   - TENSAIR_ENOMEM (with the sizes in tensair_last_error) when the context's configuration needs
- *     more per-batch memory than the array holds; roughly batch * 2 * window * (k+1) * 32 bytes plus
- *     batch * row_stride * 8 bytes must stay below 32 MiB.
+ *     more of that memory than the array holds.  With I = 2 * batch + pairs * (k+1) sort items
+ *     (pairs = 2 * window * batch - window * (window+1)) the need is about
+ *       I * (8 + 8 + 16)  +  2 * batch * row_stride * 8  +  (I / 32 + 2) * row_stride * 8  +  I / 4  bytes
+ *     (sort buffers and terms; partial centre gradients, two per position; chunk partials; lists and
+ *     histograms): e.g. V = 20,000, d = 64, window 5, k = 5, batch 1,024 needs 4 MiB; batch 8,192 at
+ *     d = 300, k = 15 needs 180 MiB and is refused.
  *   - The first call on a device looks up the array's device address (once per device, with that device
- *     current).  Make that first call before any stream capture begins.
+ *     current, under a lock, so first calls from several threads are safe).  Make that first call before
+ *     any stream capture begins.
  *   - All calls, from all contexts of the process on one GPU, share the one array.  It keeps the last
  *     call's contents; the call clears what it needs to be zero itself.  Two calls that may overlap on
  *     the GPU (contexts on different streams) race on it: serialise them.
@@ -314,7 +342,8 @@ TENSAIR_API int tensair_update_sampler(tensair_ctx* ctx);
  * one synchronisation per step can so serve the losses of all replicas.  host_dst must stay valid until then. */
 TENSAIR_API int tensair_read_loss_async(tensair_ctx* ctx, double* host_dst);
 
-/* Waits for the stream; returns and clears a pending TENSAIR_EBADTOKEN. */
+/* Waits for the stream; returns and clears a pending device-side error: TENSAIR_EBADTOKEN, TENSAIR_ETIMEOUT or
+ * TENSAIR_EBOUNDS (the gravest of those raised; tensair_last_error names all). */
 TENSAIR_API int tensair_sync(tensair_ctx* ctx);
 
 /* Copies rows [row0, row0+nrows) of a replica's input (which=0) or output (which=1) table into
@@ -396,6 +425,18 @@ TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensa
 
 TENSAIR_API const char* tensair_strerror(int code);
 TENSAIR_API const char* tensair_last_error(const tensair_ctx* ctx);
+
+/* The device-side error word.  Kernels never trap: one that meets bad input or gives up a bounded wait sets a bit
+ * of a sticky word in the scratch buffer and skips its work; the next synchronising call turns the word into a code.
+ *   bit 0 (1)  a token id outside [0,V)                          -> TENSAIR_EBADTOKEN
+ *   bit 1 (2)  a wait for a warp's own bulk copies ran out        -> TENSAIR_ETIMEOUT
+ *   bit 2 (4)  checked build: an index outside its array         -> TENSAIR_EBOUNDS
+ *   bit 3 (8)  a merged message outgrew its slot                  -> TENSAIR_EBOUNDS
+ * tensair_error_of_flags gives the code a value of the word stands for (host only, no context needed).
+ * tensair_raise_error_flags ORs bits into a context's word from the host, as a kernel would have: a hook for testing
+ * a caller's error handling without making a GPU misbehave.  Synchronises. */
+TENSAIR_API int tensair_error_of_flags(uint32_t flags);
+TENSAIR_API int tensair_raise_error_flags(tensair_ctx* ctx, uint32_t flags);
 
 /* ---- host-only pieces, usable without a GPU ---- */
 

@@ -15,7 +15,7 @@ _HERE = Path(__file__).resolve().parent
 LIB_PATH = _HERE / "libtensair.so"
 
 SUM, MEAN = 0, 1
-OK, EINVAL, ENOMEM, ECUDA, EBADTOKEN, EPENDING, ENOTFOUND = 0, -1, -2, -3, -4, -5, -6
+OK, EINVAL, ENOMEM, ECUDA, EBADTOKEN, EPENDING, ENOTFOUND, ETIMEOUT, EBOUNDS = 0, -1, -2, -3, -4, -5, -6, -7, -8
 
 
 class Config(C.Structure):
@@ -44,7 +44,7 @@ class MsgInfo(C.Structure):
 
 class MsgView(C.Structure):
     _fields_ = [("ids", C.c_void_p), ("delta", C.c_void_p), ("max_rows", C.c_uint32), ("row_stride", C.c_uint32),
-                ("ids_offset", C.c_uint64), ("delta_offset", C.c_uint64)]
+                ("ids_offset", C.c_uint64), ("delta_offset", C.c_uint64), ("header_offset", C.c_uint64)]
 
 
 class Delivery(C.Structure):
@@ -73,6 +73,7 @@ SYMBOLS = {
     "tensair_message_buffers": (_int, [_vp, _u32, _u64, _P(MsgView)]),
     "tensair_message_rows": (_int, [_vp, _u32, _u64, _P(_u32), _P(_u32)]),
     "tensair_commit_message": (_int, [_vp, _u32, _u64, _u32, _u32]),
+    "tensair_commit_message_on": (_int, [_vp, _u32, _u64, _u32, _u32, _vp]),
     "tensair_shadow_apply": (_int, [_vp, _u32, _u64, _int, _P(_u32)]),
     "tensair_destroy": (None, [_vp]),
     "tensair_train_batch": (_int, [_vp, _u32, _vp, _u32, _u64, _P(C.c_double), _P(MsgInfo)]),
@@ -103,6 +104,8 @@ SYMBOLS = {
     "tensair_profile_read": (_int, [_vp, _u32, _vp, _P(_u32)]),
     "tensair_strerror": (C.c_char_p, [_int]),
     "tensair_last_error": (C.c_char_p, [_vp]),
+    "tensair_error_of_flags": (_int, [_u32]),
+    "tensair_raise_error_flags": (_int, [_vp, _u32]),
     "tensair_build_alias_host": (_int, [_vp, _u32, _vp, _vp]),
     "tensair_philox4x32_10": (None, [_P(_u32), _P(_u32), _P(_u32)]),
     "tensair_delay": (_u32, [_u64, _u32, _u64, _u32, _u32]),
@@ -173,6 +176,10 @@ def tensair_philox4x32_10(counter, key):
     o = (C.c_uint32 * 4)()
     lib().tensair_philox4x32_10(c, k, o)
     return [int(x) for x in o]
+
+
+def tensair_error_of_flags(flags: int) -> int:
+    return int(lib().tensair_error_of_flags(flags))
 
 
 def tensair_tune(name: str, value: int):
@@ -354,9 +361,18 @@ class Context:
                "tensair_message_rows", self._h)
         return int(n.value), int(n_in.value)
 
-    def tensair_commit_message(self, sender, batch_index, n_rows, n_in_rows):
-        _check(lib().tensair_commit_message(self._h, sender, batch_index, n_rows, n_in_rows), "tensair_commit_message",
-               self._h)
+    def tensair_message_header(self, sender, batch_index):
+        """int32 CUDA tensor [2] that IS the head of the slot's header: (rows, input rows) of the message, as the
+        kernels that built it left them (valid once the stream has passed them)."""
+        v = MsgView()
+        _check(lib().tensair_message_buffers(self._h, sender, batch_index, C.byref(v)), "tensair_message_buffers", self._h)
+        return self.pool[v.header_offset:v.header_offset + 8].view(self.torch.int32)
+
+    def tensair_commit_message(self, sender, batch_index, n_rows, n_in_rows, stream=None):
+        """stream: a torch.cuda.Stream on which the slot's header and index are written (default: the context's)."""
+        _check(lib().tensair_commit_message_on(self._h, sender, batch_index, n_rows, n_in_rows,
+                                               stream.cuda_stream if stream is not None else None),
+               "tensair_commit_message_on", self._h)
 
     def tensair_shadow_apply(self, receiver, step, drain=False) -> int:
         n = C.c_uint32(0)
@@ -371,8 +387,14 @@ class Context:
         _check(lib().tensair_read_loss_async(self._h, host_ptr), "tensair_read_loss_async", self._h)
 
     def tensair_sync(self) -> int:
-        """Returns the status (OK or EBADTOKEN) instead of raising."""
+        """Returns the status (OK, EBADTOKEN, ETIMEOUT or EBOUNDS) instead of raising."""
         return int(lib().tensair_sync(self._h))
+
+    def tensair_raise_error_flags(self, flags: int):
+        _check(lib().tensair_raise_error_flags(self._h, flags), "tensair_raise_error_flags", self._h)
+
+    def tensair_last_error(self) -> str:
+        return lib().tensair_last_error(self._h).decode()
 
     def tensair_read_embeddings(self, replica, which, row0=0, nrows=None) -> np.ndarray:
         nrows = self.cfg.V - row0 if nrows is None else nrows

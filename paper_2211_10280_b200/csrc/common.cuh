@@ -72,6 +72,12 @@ __device__ inline double widen_down(float f) {
 }
 constexpr double kWidenUp = 0x1p896;   // widen_down(f) * kWidenUp == (double)f
 
+// Bits of the device error word (sticky until a synchronising call reads and clears it).
+constexpr uint32_t kErrBadToken = 1u;   // a batch held a token id outside [0,V)
+constexpr uint32_t kErrTimeout = 2u;    // a bounded wait for a warp's own bulk copies ran out
+constexpr uint32_t kErrBounds = 4u;     // checked build: an index left its array; the access was skipped
+constexpr uint32_t kErrOverflow = 8u;   // a merged message had more rows than its slot holds; the rest was dropped
+
 struct Shape {
     uint32_t V, d, d4, stride, w, k, K1;
 };

@@ -18,7 +18,9 @@ struct Carve {
     uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, terms, gin_pos, loss_pos, hist,
         tile_counts, seg_start, long_rows, chunk_items, partials, merge_counts, topk, owner, owned, n_owned, alias_state, alias_work, total;
     uint64_t slot_bytes, bucket_off, ids_off, delta_off;
-    uint32_t stride, max_pairs, max_contrib, max_items, max_rows, max_long, max_chunks;
+    uint32_t stride, max_pairs, max_contrib, max_items, max_long, max_chunks;
+    uint32_t max_rows;    // most rows the message of ONE batch can have (bounds the per-batch lists)
+    uint32_t slot_rows;   // rows a message slot holds: max_rows, or the union of maxGradBuffer buffered messages
 };
 
 inline uint32_t bits_for(uint32_t x) {   // bits needed to represent x
@@ -69,8 +71,10 @@ namespace tensair {
 
 // Records the CUDA error text on the context and returns TENSAIR_ECUDA.
 int fail(tensair_ctx* ctx, cudaError_t e, const char* what);
-// Waits for the stream, then reads and clears the device error flag.
+// Waits for the stream, then reads and clears the device error word.
 int collect(tensair_ctx* ctx);
+// The code and text that a value of the device error word stands for.
+int error_of_flags(uint32_t flags, std::string* text);
 
 #define TENSAIR_CUDA(ctx, call)                                    \
     do {                                                           \

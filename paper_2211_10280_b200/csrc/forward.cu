@@ -287,7 +287,7 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d, u
         for (int o = 16; o > 0; o >>= 1) loss += __shfl_xor_sync(0xFFFFFFFFu, loss, o);
         if (lane == 0) loss_pos[2 * q + side] = loss;
     }
-    if (failed && lane == 0) atomicOr(err, 2u);
+    if (failed && lane == 0) atomicOr(err, kErrTimeout);
 }
 
 // Launch shape of the forward kernel: rows reduced together (8 by default: less shared memory per warp, so
@@ -303,6 +303,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err,
                            const uint32_t* owned, const uint32_t* n_owned) {
     if (n < 2) return cudaSuccess;
+    if (L.device < 0 || L.device >= kMaxDevices) return cudaErrorInvalidDevice;
     const size_t row = (size_t)s.stride * 4;
     const int cr = g_forward_rows == 4 || g_forward_rows == 8 || g_forward_rows == 16 ? g_forward_rows : 8;
     int blocks_per_sm = g_forward_blocks > 0 ? g_forward_blocks : (cr == 16 ? 5 : cr == 8 ? 8 : 10);
@@ -333,8 +334,11 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
     Timed timed(L, K_FORWARD);
 #define TENSAIR_FWD(NV, CR, NR, VW)                                                                                 \
     do {                                                                                                            \
-        static bool attr_set = false;                                                                               \
-        static int room_for = 0;                                                                                    \
+        /* function attributes belong to a device: set them once on each device that launches */                  \
+        static bool attr_set_on[kMaxDevices] = {};                                                                  \
+        static int room_for_on[kMaxDevices] = {};                                                                   \
+        bool& attr_set = attr_set_on[L.device];                                                                     \
+        int& room_for = room_for_on[L.device];                                                                      \
         if (!attr_set) {                                                                                            \
             cudaFuncSetAttribute(k_forward<NV, CR, NR, VW>, cudaFuncAttributeMaxDynamicSharedMemorySize, 200 * 1024); \
             cudaFuncSetAttribute(k_forward<NV, CR, NR, VW>, cudaFuncAttributePreferredSharedMemoryCarveout, 100);   \

@@ -40,7 +40,9 @@ struct Launcher {
     uint64_t* launches;   // incremented once per kernel launch
     int sms;              // multiprocessors of the device
     Profiler* prof;       // nullable
+    int device = 0;       // ordinal of the device the stream belongs to
 };
+constexpr int kMaxDevices = 64;   // per-device launch state (function attributes, symbol addresses) is kept up to here
 
 // Blocks per multiprocessor of the grid-stride kernels (row sums, message apply).  More blocks than
 // are resident at once let the hardware scheduler even out rows of unequal cost.
@@ -147,8 +149,9 @@ struct MergeInputs {
     const float* delta[kMaxMerge];
     const uint32_t* buckets[kMaxMerge];
 };
+// capacity: rows the output slot holds; a union with more rows raises kErrOverflow and is cut there.
 cudaError_t launch_merge(const Launcher& L, const MergeInputs& in, MsgHeader* hdr, uint32_t* bucket_start, uint32_t* ids,
-                         float* delta, uint32_t* counts, const Shape& s);
+                         float* delta, uint32_t* counts, const Shape& s, uint32_t capacity, uint32_t* err);
 // out[r] = 1 - cos(table row r, snapshot row r) for nrows rows; rows of `rows` are strided, of `snap` dense.
 // Working state of the most-drifted-rows selection, in the context's scratch.
 constexpr uint32_t kTopkMax = 4096;

@@ -29,7 +29,7 @@ k_merge_count(MergeInputs in, uint32_t n_buckets, uint32_t* __restrict__ counts)
 // One block: exclusive scan of the bucket counts into the merged message's bucket index; row count in the header.
 __global__ void __launch_bounds__(1024)
 k_merge_scan(const uint32_t* __restrict__ counts, uint32_t n_buckets, uint32_t* __restrict__ bucket_start,
-             MsgHeader* __restrict__ hdr) {
+             MsgHeader* __restrict__ hdr, uint32_t capacity, uint32_t* __restrict__ err) {
     __shared__ uint32_t warp_tot[32];
     __shared__ uint32_t carry_s;
     if (threadIdx.x == 0) carry_s = 0;
@@ -65,7 +65,10 @@ k_merge_scan(const uint32_t* __restrict__ counts, uint32_t n_buckets, uint32_t* 
     }
     if (threadIdx.x == 0) {
         bucket_start[n_buckets] = carry_s;
-        hdr->n_rows = carry_s;
+        // The slots are sized for the largest union there can be; should one still not fit, the message is cut
+        // at the slot's capacity (the write kernel skips the rows past it) and the error word says so.
+        if (carry_s > capacity) atomicOr(err, kErrOverflow);
+        hdr->n_rows = carry_s < capacity ? carry_s : capacity;
         hdr->n_items = 0;
         hdr->pad = 0;
     }
@@ -76,7 +79,7 @@ template <int NV>
 __global__ void __launch_bounds__(128)
 k_merge_write(MergeInputs in, uint32_t n_buckets, uint32_t V, const uint32_t* __restrict__ bucket_start,
               MsgHeader* __restrict__ hdr, uint32_t* __restrict__ out_ids, float4* __restrict__ out_delta, uint32_t d4,
-              uint32_t stride4) {
+              uint32_t stride4, uint32_t capacity) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
@@ -97,13 +100,14 @@ k_merge_write(MergeInputs in, uint32_t n_buckets, uint32_t V, const uint32_t* __
         const uint32_t first_id = b << kBucketShift;
         // the first output row (id >= V) marks the end of the input rows
         if (lane == 0 && V >= first_id && V < first_id + (1u << kBucketShift))
-            hdr->n_in_rows = base + __popc(all & ((1u << (V - first_id)) - 1));
+            hdr->n_in_rows = min(base + __popc(all & ((1u << (V - first_id)) - 1)), capacity);
         uint32_t rest = all;
         while (rest) {
             const uint32_t j = __ffs(rest) - 1;
             rest &= rest - 1;
             const uint32_t below = (1u << j) - 1;
             const uint32_t pos = base + __popc(all & below);
+            if (pos >= capacity) break;   // positions ascend with j: nothing further of this bucket fits either
             float4 acc[NV];
             bool have = false;
 #pragma unroll
@@ -134,7 +138,7 @@ k_merge_write(MergeInputs in, uint32_t n_buckets, uint32_t V, const uint32_t* __
 }
 
 cudaError_t launch_merge(const Launcher& L, const MergeInputs& in, MsgHeader* hdr, uint32_t* bucket_start, uint32_t* ids,
-                         float* delta, uint32_t* counts, const Shape& s) {
+                         float* delta, uint32_t* counts, const Shape& s, uint32_t capacity, uint32_t* err) {
     const uint32_t nb = bucket_count(s.V);
     const uint32_t stride4 = s.stride / 4;
     float4* d4p = reinterpret_cast<float4*>(delta);
@@ -144,13 +148,13 @@ cudaError_t launch_merge(const Launcher& L, const MergeInputs& in, MsgHeader* hd
     }
     {
         Timed timed(L, K_MERGE);
-        k_merge_scan<<<1, 1024, 0, L.stream>>>(counts, nb, bucket_start, hdr);
+        k_merge_scan<<<1, 1024, 0, L.stream>>>(counts, nb, bucket_start, hdr, capacity, err);
     }
     uint32_t blocks = (uint32_t)L.sms * 32;
     if (blocks > (nb + 3) / 4) blocks = (nb + 3) / 4;
     Timed timed(L, K_MERGE);
 #define TENSAIR_MERGE(NV) \
-    k_merge_write<NV><<<blocks, 128, 0, L.stream>>>(in, nb, s.V, bucket_start, hdr, ids, d4p, s.d4, stride4)
+    k_merge_write<NV><<<blocks, 128, 0, L.stream>>>(in, nb, s.V, bucket_start, hdr, ids, d4p, s.d4, stride4, capacity)
     if (s.d4 <= 32) TENSAIR_MERGE(1);
     else if (s.d4 <= 64) TENSAIR_MERGE(2);
     else if (s.d4 <= 96) TENSAIR_MERGE(3);

@@ -89,7 +89,7 @@ __global__ void k_validate(const int32_t* __restrict__ tok, uint32_t n, uint32_t
     const uint32_t i = blockIdx.x * blockDim.x + threadIdx.x;
     if (i < n) {
         const int32_t t = tok[i];
-        if (t < 0 || (uint32_t)t >= V) atomicOr(err, 1u);
+        if (t < 0 || (uint32_t)t >= V) atomicOr(err, kErrBadToken);
         if (owner) {
             const Philox4 r = philox4x32_10(Philox4{(uint32_t)t, 0u, 0u, kTagRoute}, key0, key1);
             const bool mine = __umulhi(r.x, W) == replica;

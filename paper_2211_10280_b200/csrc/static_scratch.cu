@@ -14,6 +14,7 @@
 // cudaGetSymbolAddress while that device is current, on the first call for that device.
 #include <cstdio>
 #include <cstring>
+#include <mutex>
 
 #include "context.h"
 
@@ -24,9 +25,9 @@ namespace {
 constexpr size_t kStaticScratchBytes = 32u << 20;   // 32 MiB per GPU
 static __device__ __align__(256) unsigned char g_static_scratch[kStaticScratchBytes];
 
-constexpr int kMaxDevices = 64;
 unsigned char* g_scratch_address[kMaxDevices];      // device address of the array, per device ordinal
 bool g_scratch_known[kMaxDevices];
+std::mutex g_scratch_lock;                          // first calls may come from several host threads
 
 // Byte offsets of the per-batch working buffers inside the array (same sizes as the context's own scratch).
 struct StaticCarve {
@@ -77,14 +78,18 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
     }
     DeviceGuard guard(c.device);
     if (!guard.ok) return TENSAIR_ECUDA;
-    if (!g_scratch_known[c.device]) {
-        // set-up, once per device, with that device current: the symbol is not a device pointer in host code
-        unsigned char* ptr = nullptr;
-        TENSAIR_CUDA(ctx, cudaGetSymbolAddress((void**)&ptr, g_static_scratch));
-        g_scratch_address[c.device] = ptr;
-        g_scratch_known[c.device] = true;
+    unsigned char* ws = nullptr;
+    {
+        std::lock_guard<std::mutex> hold(g_scratch_lock);
+        if (!g_scratch_known[c.device]) {
+            // set-up, once per device, with that device current: the symbol is not a device pointer in host code
+            unsigned char* ptr = nullptr;
+            TENSAIR_CUDA(ctx, cudaGetSymbolAddress((void**)&ptr, g_static_scratch));
+            g_scratch_address[c.device] = ptr;
+            g_scratch_known[c.device] = true;
+        }
+        ws = g_scratch_address[c.device];
     }
-    unsigned char* ws = g_scratch_address[c.device];
     auto in_ws = [ws](uint64_t off) { return ws + off; };
 
     const uint32_t me = ctx->gid(replica);   // the replica's id among all replicas of the job

@@ -26,6 +26,7 @@ int validate_config(const tensair_config* c) {
     if (c->max_delay > 64) return TENSAIR_EINVAL;
     if (c->row_stride && (c->row_stride < c->d || c->row_stride % 4)) return TENSAIR_EINVAL;
     if (!(c->lr == c->lr)) return TENSAIR_EINVAL;
+    if (c->device < 0 || c->device >= kMaxDevices) return TENSAIR_EINVAL;
     if (c->reduction > TENSAIR_MEAN) return TENSAIR_EINVAL;
     const uint64_t contrib = (uint64_t)pair_count(c->batch, c->window) * (c->k + 1);
     if (contrib + c->batch >= (1ull << 31)) return TENSAIR_EINVAL;
@@ -38,6 +39,9 @@ void carve(const tensair_config& c, Carve& k) {
     k.max_contrib = k.max_pairs * (c.k + 1);
     k.max_items = 2 * c.batch + k.max_contrib;   // two input-row items per position, then the contributions
     k.max_rows = (c.batch < c.V ? c.batch : c.V) + (k.max_contrib < c.V ? k.max_contrib : c.V);
+    // A sent message is the union of maxGradBuffer batch messages: up to m times the rows of one, capped by the tables.
+    const uint64_t m_in = (uint64_t)c.max_grad_buffer * c.batch, m_out = (uint64_t)c.max_grad_buffer * k.max_contrib;
+    k.slot_rows = (uint32_t)((m_in < c.V ? m_in : c.V) + (m_out < c.V ? m_out : c.V));
     k.max_long = k.max_items / kChunk + 1;
     k.max_chunks = 2 * (k.max_items / kChunk) + 2;
     uint64_t off = 0;
@@ -71,8 +75,8 @@ void carve(const tensair_config& c, Carve& k) {
     k.total = off;
     k.bucket_off = kHeaderBytes;
     k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
-    k.delta_off = round_up(k.ids_off + (uint64_t)k.max_rows * 4, 256);
-    k.slot_bytes = round_up(k.delta_off + (uint64_t)k.max_rows * k.stride * 4, 256);
+    k.delta_off = round_up(k.ids_off + (uint64_t)k.slot_rows * 4, 256);
+    k.slot_bytes = round_up(k.delta_off + (uint64_t)k.slot_rows * k.stride * 4, 256);
 }
 
 }  // namespace
@@ -84,14 +88,32 @@ int fail(tensair_ctx* ctx, cudaError_t e, const char* what) {
     return TENSAIR_ECUDA;
 }
 
-// Reads and clears the device error flag after a synchronisation.
+// What a value of the device error word means.  Several bits may be set; the code is that of the gravest
+// (an index out of bounds, then a wait that ran out, then bad input), the text names all of them.
+int error_of_flags(uint32_t flags, std::string* text) {
+    if (!flags) return TENSAIR_OK;
+    std::string t;
+    auto add = [&t](const char* what) { if (!t.empty()) t += "; "; t += what; };
+    if (flags & kErrBounds) add("a checked index was outside its array (the access was skipped)");
+    if (flags & kErrOverflow) add("a merged message had more rows than its slot holds");
+    if (flags & kErrTimeout) add("a wait for a warp's own asynchronous copies ran out (the batch is incomplete)");
+    if (flags & kErrBadToken) add("a batch held a token id outside [0,V)");
+    if (flags & ~(kErrBounds | kErrOverflow | kErrTimeout | kErrBadToken)) add("unknown error bits");
+    t += "; that batch and the batches after it were dropped";
+    if (text) *text = t;
+    if (flags & (kErrBounds | kErrOverflow)) return TENSAIR_EBOUNDS;
+    if (flags & kErrTimeout) return TENSAIR_ETIMEOUT;
+    if (flags & kErrBadToken) return TENSAIR_EBADTOKEN;
+    return TENSAIR_ECUDA;
+}
+
+// Reads and clears the device error word after a synchronisation.
 int collect(tensair_ctx* ctx) {
     TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->err, ctx->at<uint32_t>(ctx->cv.err), 4, cudaMemcpyDeviceToHost, ctx->stream));
     TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
     if (ctx->stage->err) {
         TENSAIR_CUDA(ctx, cudaMemsetAsync(ctx->at<uint32_t>(ctx->cv.err), 0, 4, ctx->stream));
-        ctx->last_error = "a batch held a token id outside [0,V); it and the batches after it were dropped";
-        return TENSAIR_EBADTOKEN;
+        return error_of_flags(ctx->stage->err, &ctx->last_error);
     }
     return TENSAIR_OK;
 }
@@ -210,7 +232,7 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
             }
             TENSAIR_CUDA(ctx, launch_merge(ctx->L, in, ctx->slot_hdr(send_slot), ctx->slot_buckets(send_slot),
                                            ctx->slot_ids(send_slot), ctx->slot_delta(send_slot),
-                                           ctx->at<uint32_t>(cv.merge_counts), ctx->shape));
+                                           ctx->at<uint32_t>(cv.merge_counts), ctx->shape, cv.slot_rows, err));
             const int rc = ctx->sched->on_train(me, batch_index);
             if (rc != TENSAIR_OK) return rc;
             ctx->buffered[replica] = 0;
@@ -297,7 +319,7 @@ int tensair_workspace_bytes_sharded(const tensair_config* cfg, uint32_t world_W,
                        (cfg->max_grad_buffer > 1 ? (uint64_t)cfg->W * cfg->max_grad_buffer : 0)) * cv.slot_bytes;
     out->scratch_bytes = cv.total;
     out->max_pairs = cv.max_pairs;
-    out->max_rows = cv.max_rows;
+    out->max_rows = cv.slot_rows;
     out->reserved = 0;
     return TENSAIR_OK;
 }
@@ -314,6 +336,8 @@ int tensair_init_sharded(const tensair_config* cfg, const tensair_buffers* bufs,
     if (!out || !bufs || tensair_workspace_bytes_sharded(cfg, world_W, &sz) != TENSAIR_OK) return TENSAIR_EINVAL;
     *out = nullptr;
     if ((uint64_t)first_replica + cfg->W > world_W) return TENSAIR_EINVAL;
+    // buffered gradients are merged where they were computed; a job spread over processes sends every batch
+    if (world_W > cfg->W && cfg->max_grad_buffer != 1) return TENSAIR_EINVAL;
     if (!bufs->tables || !bufs->pool || !bufs->scratch) return TENSAIR_EINVAL;
     if (((uintptr_t)bufs->tables | (uintptr_t)bufs->pool | (uintptr_t)bufs->scratch) & 255) return TENSAIR_EINVAL;
     if (bufs->tables_bytes < sz.tables_bytes || bufs->pool_bytes < sz.pool_bytes || bufs->scratch_bytes < sz.scratch_bytes)
@@ -345,7 +369,7 @@ int tensair_init_sharded(const tensair_config* cfg, const tensair_buffers* bufs,
         return code;
     };
     if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return bail(TENSAIR_ECUDA);
-    ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount, &ctx->prof};
+    ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount, &ctx->prof, cfg->device};
     if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->sched = new Schedule(world_W, cfg->max_delay, cfg->seed);
     ctx->buffered.assign(cfg->W, 0);
@@ -519,10 +543,11 @@ int tensair_message_buffers(tensair_ctx* ctx, uint32_t sender, uint64_t batch_in
         return local ? TENSAIR_ENOTFOUND : TENSAIR_EPENDING;
     out->ids = ctx->slot_ids(slot);
     out->delta = ctx->slot_delta(slot);
-    out->max_rows = ctx->cv.max_rows;
+    out->max_rows = ctx->cv.slot_rows;
     out->row_stride = ctx->cv.stride;
     out->ids_offset = (uint64_t)slot * ctx->cv.slot_bytes + ctx->cv.ids_off;
     out->delta_offset = (uint64_t)slot * ctx->cv.slot_bytes + ctx->cv.delta_off;
+    out->header_offset = (uint64_t)slot * ctx->cv.slot_bytes;
     return TENSAIR_OK;
 }
 
@@ -541,7 +566,12 @@ int tensair_message_rows(tensair_ctx* ctx, uint32_t replica, uint64_t batch_inde
 }
 
 int tensair_commit_message(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, uint32_t n_rows, uint32_t n_in_rows) {
-    if (!ctx || sender >= ctx->world_W || batch_index >= (1ull << 32) || n_in_rows > n_rows || n_rows > ctx->cv.max_rows)
+    return tensair_commit_message_on(ctx, sender, batch_index, n_rows, n_in_rows, nullptr);
+}
+
+int tensair_commit_message_on(tensair_ctx* ctx, uint32_t sender, uint64_t batch_index, uint32_t n_rows, uint32_t n_in_rows,
+                              void* stream) {
+    if (!ctx || sender >= ctx->world_W || batch_index >= (1ull << 32) || n_in_rows > n_rows || n_rows > ctx->cv.slot_rows)
         return TENSAIR_EINVAL;
     if (sender >= ctx->first && sender < ctx->first + ctx->cfg.W) return TENSAIR_EINVAL;   // local messages file themselves
     DeviceGuard guard(ctx->cfg.device);
@@ -549,7 +579,9 @@ int tensair_commit_message(tensair_ctx* ctx, uint32_t sender, uint64_t batch_ind
     const int rc = ctx->sched->on_train(sender, batch_index);
     if (rc != TENSAIR_OK) return rc;
     const uint32_t slot = ctx->sched->slot_of(sender, batch_index);
-    TENSAIR_CUDA(ctx, launch_index_received(ctx->L, ctx->slot_hdr(slot), ctx->slot_ids(slot), ctx->slot_buckets(slot),
+    Launcher L = ctx->L;
+    if (stream) L.stream = (cudaStream_t)stream;
+    TENSAIR_CUDA(ctx, launch_index_received(L, ctx->slot_hdr(slot), ctx->slot_ids(slot), ctx->slot_buckets(slot),
                                             ctx->cfg.V, n_rows, n_in_rows));
     return TENSAIR_OK;
 }
@@ -781,11 +813,28 @@ const char* tensair_strerror(int code) {
         case TENSAIR_EBADTOKEN: return "token id outside [0,V)";
         case TENSAIR_EPENDING: return "message slot still has undelivered recipients";
         case TENSAIR_ENOTFOUND: return "message no longer held";
+        case TENSAIR_ETIMEOUT: return "a bounded wait inside a kernel ran out";
+        case TENSAIR_EBOUNDS: return "an index checked on the device was outside its array";
         default: return "unknown error";
     }
 }
 
 const char* tensair_last_error(const tensair_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
+
+int tensair_error_of_flags(uint32_t flags) { return error_of_flags(flags, nullptr); }
+
+int tensair_raise_error_flags(tensair_ctx* ctx, uint32_t flags) {
+    if (!ctx) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    // the word is sticky: OR the bits in by reading it back first (a test hook, so the round trip does not matter)
+    TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->err, ctx->at<uint32_t>(ctx->cv.err), 4, cudaMemcpyDeviceToHost, ctx->stream));
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    ctx->stage->err |= flags;
+    TENSAIR_CUDA(ctx, cudaMemcpyAsync(ctx->at<uint32_t>(ctx->cv.err), &ctx->stage->err, 4, cudaMemcpyHostToDevice, ctx->stream));
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    return TENSAIR_OK;
+}
 
 int tensair_build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias) {
     if (!V || !thresh || !alias) return TENSAIR_EINVAL;

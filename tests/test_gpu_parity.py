@@ -728,3 +728,128 @@ def test_buffered_gradients_are_sent_every_mth_batch(torch, m):
         assert np.array_equal(o.delivery_log(j), log) and log.shape[0] == sends * (wl.W - 1)
         assert set((log[:, 0] % m).tolist()) == {m - 1}
         compare_tables(o, g, j, TOL_200)
+
+
+def test_merged_message_larger_than_any_one_batch_message(torch):
+    """maxGradBuffer = 8 with few contributions per batch and a large vocabulary: the union of the 8 buffered
+    messages has several times the rows any single batch can touch, so the send slot must be sized for the union."""
+    m = 8
+    wl = synth.scaled(synth.LARGE_DASGD, V=200_000, d=16, window=2, batch=64, k=3, W=2, stream_seeds=(2, 3),
+                      max_delay=1, zipf_s=0.2)
+    one_batch = wl.batch + wl.pairs_per_batch * (wl.k + 1)
+    steps = 2 * m
+    streams = synth.all_streams(wl, steps)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 22, scale=0.2)
+    o, g = make_pair(wl, counts=synth.stream_counts(streams, wl.V), init_in=t_in, init_out=t_out, max_grad_buffer=m)
+    assert g.sizes.max_rows == m * one_batch
+    largest = 0
+    for t in range(steps):
+        for i in range(wl.W):
+            assert o.train_batch(i, streams[i][t], t)[0] == 0
+            g.tensair_train_batch(i, dev(torch, streams[i][t]), t)
+            om, gm = o.read_message(i, t), g.tensair_read_message(i, t)
+            assert (om is None) == (gm is None) == (t % m != m - 1)
+            if om is not None:
+                largest = max(largest, om[0].size)
+                assert np.array_equal(om[0], gm[0])
+                assert rel_err(gm[1], om[1]) <= TOL_200
+        for j in range(wl.W):
+            assert o.apply_messages(j, t) == g.tensair_apply_messages(j, t)
+    assert largest > 3 * one_batch, (largest, one_batch)      # the case the one-batch bound would have overflowed
+    assert o.drain() == g.tensair_drain()
+    assert g.tensair_sync() == 0
+    for j in range(wl.W):
+        compare_tables(o, g, j, TOL_200)
+
+
+def test_a_wait_that_ran_out_is_not_reported_as_a_bad_token(torch):
+    """The device error word is raised from the host, as a kernel whose bounded wait gave up would raise it
+    (no GPU is made to misbehave): every cause has its own code, and reading the word clears it."""
+    from paper_2211_10280_b200 import binding as B
+
+    wl = synth.scaled(synth.TINY, V=500, d=8, batch=64)
+    g = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch)
+    assert g.tensair_sync() == B.OK
+    g.tensair_raise_error_flags(2)
+    assert g.tensair_sync() == B.ETIMEOUT and "wait" in g.tensair_last_error()
+    assert g.tensair_sync() == B.OK
+    g.tensair_raise_error_flags(1)
+    assert g.tensair_sync() == B.EBADTOKEN and "token" in g.tensair_last_error()
+    g.tensair_raise_error_flags(1)
+    g.tensair_raise_error_flags(2)
+    assert g.tensair_sync() == B.ETIMEOUT          # the graver of the two; the text names both
+    assert "token" in g.tensair_last_error() and "wait" in g.tensair_last_error()
+    g.tensair_raise_error_flags(8)
+    assert g.tensair_sync() == B.EBOUNDS
+    # a raised word drops the batches that follow until it has been read, like a bad token does
+    before = g.tensair_read_embeddings(0, 1)
+    g.tensair_raise_error_flags(2)
+    g.tensair_train_batch(0, dev(torch, synth.token_stream(wl, 0, 1)[0]), 0)
+    assert g.tensair_sync() == B.ETIMEOUT
+    assert np.array_equal(g.tensair_read_embeddings(0, 1), before)
+
+
+def test_largest_sweep_batch_matches_the_oracle(torch):
+    """One batch of the throughput sweep's largest shape (V = 1M, batch 65,536, k = 15, window 5) at d = 64:
+    10.5 M contributions, more than 2,500 sort tiles, hot rows with tens of thousands of contributions (hundreds to
+    thousands of 64-term chunks each).  Negatives and message ids bit-exact, scalars, deltas and tables within the
+    one-batch bar."""
+    wl = synth.sweep_point(64, 65536, 15)
+    stream = synth.token_stream(wl, 0, 1)
+    counts = synth.stream_counts([stream], wl.V)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 23, scale=2.0 / math.sqrt(wl.d))
+    o, g = make_pair(wl, counts=counts, init_in=t_in, init_out=t_out)
+    rc, loss_o, nrows_o = o.train_batch(0, stream[0], 0)
+    assert rc == 0
+    loss_g, info = g.tensair_train_batch(0, dev(torch, stream[0]), 0, want_loss=True, want_info=True)
+    assert info.n_pairs == wl.pairs_per_batch == 655_330
+    assert 2 * wl.batch + info.n_pairs * (wl.k + 1) > 2500 * 4096          # sort tiles of 4,096 items
+    assert info.n_rows == nrows_o
+    no, ng = o.read_negatives(), g.tensair_read_negatives()
+    assert np.array_equal(no, ng)
+    # contributions per output row: the unmasked negative draws on it plus the pairs whose context word it is
+    toks = stream[0].astype(np.int64)
+    pos = np.arange(wl.batch)
+    as_context = np.minimum(pos, wl.window) + np.minimum(wl.batch - 1 - pos, wl.window)
+    per_row = np.bincount(toks, weights=as_context, minlength=wl.V) + np.bincount(no.ravel(), minlength=wl.V)
+    assert per_row.max() > 64 * 500, per_row.max()                           # a row of more than 500 chunks
+    assert (per_row > 64).sum() > 500                                        # and hundreds of rows on the chunked path
+    go, gg = o.read_g(), g.tensair_read_scalars()
+    assert np.max(np.abs(go - gg)) <= 1e-13
+    assert loss_g == pytest.approx(loss_o, rel=1e-12)
+    compare_message(o, g, 0, 0, TOL_ONE)
+    compare_tables(o, g, 0, TOL_ONE)
+
+
+def test_subnormal_rows_and_deltas_are_added_like_the_oracle_adds_them(torch):
+    """Table entries and deltas around the smallest normal fp32 (2^-126): the additions that apply a message (the
+    local application of the output rows inside the row-sum kernel, the input rows, and the remote application) must
+    keep subnormal inputs and results as IEEE arithmetic does - the oracle's `row + delta` in fp32 - bit for bit."""
+    wl = synth.scaled(synth.TINY, V=300, d=20, window=2, k=4, batch=200, W=2, stream_seeds=(0, 1), lr=1.0, max_delay=0)
+    streams = synth.all_streams(wl, 1)
+    t_in, t_out = synth.random_tables(wl.V, wl.d, 29, scale=1.0)
+    tiny = np.float32(2.0 ** -125)
+    t_in, t_out = (t_in * tiny).astype(np.float32), (t_out * tiny).astype(np.float32)
+    sub = np.float32(2.0 ** -126)
+    assert (np.abs(t_out[t_out != 0]) < sub).mean() > 0.3 and (np.abs(t_out) >= sub).mean() > 0.3
+    o, g = make_pair(wl, counts=synth.stream_counts(streams, wl.V), init_in=t_in, init_out=t_out)
+    for i in range(wl.W):
+        assert o.train_batch(i, streams[i][0], 0)[0] == 0
+        g.tensair_train_batch(i, dev(torch, streams[i][0]), 0)
+        ids_o, delta_o = o.read_message(i, 0)
+        ids_g, delta_g = g.tensair_read_message(i, 0)
+        assert np.array_equal(ids_o, ids_g)
+        # every dot product is ~1e-74, every sigmoid 1/2 to the last bit: a delta is one rounding of an exact sum
+        assert np.array_equal(delta_o.view(np.uint32), delta_g.view(np.uint32))
+        small = np.abs(delta_o[delta_o != 0]) < sub
+        assert small.any() and not small.all()
+    for i in range(wl.W):                                # local application, output and input rows
+        for which in (0, 1):
+            assert np.array_equal(o.read_embeddings(i, which).view(np.uint32),
+                                  g.tensair_read_embeddings(i, which).view(np.uint32)), (i, which)
+    for j in range(wl.W):                                # remote application
+        assert o.apply_messages(j, 0) == g.tensair_apply_messages(j, 0) == 1
+        for which in (0, 1):
+            got = g.tensair_read_embeddings(j, which)
+            assert np.array_equal(o.read_embeddings(j, which).view(np.uint32), got.view(np.uint32)), (j, which)
+    assert (np.abs(got[got != 0]) < sub).any()

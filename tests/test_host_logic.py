@@ -228,3 +228,45 @@ def test_null_arguments_are_rejected_not_dereferenced():
     assert lib.tensair_kernel_launches(None) == 0
     assert lib.tensair_strerror(B.EPENDING).decode().startswith("message slot")
     lib.tensair_destroy(None)
+
+
+def test_device_error_word_is_decoded_bit_by_bit():
+    # bit 0 bad token, bit 1 a bounded wait that ran out, bits 2 and 3 an index or a merged message out of bounds:
+    # each has its own code, and the gravest of several wins
+    assert B.tensair_error_of_flags(0) == B.OK
+    assert B.tensair_error_of_flags(1) == B.EBADTOKEN
+    assert B.tensair_error_of_flags(2) == B.ETIMEOUT
+    assert B.tensair_error_of_flags(4) == B.EBOUNDS
+    assert B.tensair_error_of_flags(8) == B.EBOUNDS
+    assert B.tensair_error_of_flags(1 | 2) == B.ETIMEOUT
+    assert B.tensair_error_of_flags(1 | 2 | 4) == B.EBOUNDS
+    assert len({B.EBADTOKEN, B.ETIMEOUT, B.EBOUNDS, B.ECUDA}) == 4
+    assert "wait" in B.strerror(B.ETIMEOUT) and "index" in B.strerror(B.EBOUNDS)
+
+
+@pytest.mark.parametrize("m", [1, 2, 8])
+def test_message_slots_hold_the_union_of_the_buffered_messages(m):
+    # batch 256, window 5, k 5: 15,180 contributions and 256 centre words per batch, far below V, so the union of
+    # m buffered messages can have m times the rows of one
+    cfg = B.Config(V=1_000_000, d=64, window=5, k=5, batch=256, W=1, lr=0.025, max_grad_buffer=m,
+                   max_delay=0, row_stride=0, seed=0, device=0, reduction=1)
+    sz = B.tensair_workspace_bytes(cfg)
+    contrib = synth.n_pairs(256, 5) * 6
+    assert sz.max_rows == m * 256 + m * contrib
+    slots = 1 + (m if m > 1 else 0)
+    assert sz.pool_bytes >= slots * sz.max_rows * (64 * 4 + 4)
+    # capped by the tables: a message cannot have more rows than the model
+    big = B.Config(V=1000, d=64, window=5, k=5, batch=256, W=1, lr=0.025, max_grad_buffer=m,
+                   max_delay=0, row_stride=0, seed=0, device=0, reduction=1)
+    assert B.tensair_workspace_bytes(big).max_rows == min(m * 256, 1000) + 1000
+
+
+def test_sharded_job_with_buffered_gradients_is_refused():
+    cfg = B.Config(V=100, d=8, window=2, k=3, batch=16, W=1, lr=0.025, max_grad_buffer=2, max_delay=0, row_stride=0,
+                   seed=0, device=0, reduction=0)
+    sz = B.tensair_workspace_bytes_sharded(cfg, 2)
+    # the refusal comes before any buffer or device is touched: fake, aligned, large-enough buffers will do
+    bufs = B.Buffers(256, sz.tables_bytes, 256, sz.pool_bytes, 256, sz.scratch_bytes, None)
+    h = C.c_void_p()
+    assert B.lib().tensair_init_sharded(C.byref(cfg), C.byref(bufs), None, None, None, 0, 2, C.byref(h)) == B.EINVAL
+    assert not h.value

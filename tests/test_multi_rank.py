@@ -57,5 +57,36 @@ def test_reference_arm_prints_one_line_from_rank_zero(tmp_path):
     assert res.returncode == 0
     line = json.loads(res.stdout.strip().splitlines()[-1])
     assert line["impl"] == "reference" and line["unit"] == "pairs/s" and line["value"] > 0
-    assert line["config"]["workload"] == "sgns_tiny" and line["cpu_baseline"]["kind"] == "oracle"
+    assert line["config"]["workload"] == "sgns_tiny[W=2]" and line["cpu_baseline"]["kind"] == "oracle"
     assert line["e2e"]["h2d_bytes_per_step"] == 0
+
+
+def test_gpus_flag_starts_the_ranks_itself(tmp_path):
+    """`bench.py --gpus 2` with no launcher around it (no RANK in the environment) must start two ranks; with the
+    reference arm rank 0 alone works and prints the one line, which says n_gpus 2 and names the workload as two
+    ranks run it."""
+    env = {k: v for k, v in os.environ.items() if k not in ("RANK", "WORLD_SIZE", "LOCAL_RANK", "MASTER_PORT")}
+    res = subprocess.run([sys.executable, str(ROOT / "bench.py"), "--gpus", "2", "--impl", "reference", "--workload",
+                          "sgns_tiny", "--steps", "2", "--warmup", "1"], env=env, capture_output=True, text=True,
+                         timeout=600)
+    assert res.returncode == 0, res.stderr[-2000:]
+    lines = [json.loads(x) for x in res.stdout.splitlines() if x.startswith("{")]
+    assert len(lines) == 1
+    line = lines[0]
+    assert line["impl"] == "reference" and line["n_gpus"] == 2 and line["value"] > 0
+    # sgns_tiny has one replica: over two ranks it runs with one replica per rank
+    assert line["config"]["replicas"] == 2 and line["config"]["workload"] == "sgns_tiny[W=2]"
+
+
+def test_both_arms_print_the_same_config_keys():
+    import bench
+    from paper_2211_10280_b200 import synth
+
+    a = bench.config_of(synth.LARGE_DASGD, 1, "x")
+    assert {"workload", "V", "d", "window", "k", "batch", "replicas", "max_delay", "reduction", "pairs_per_batch",
+            "storage", "l2", "parallelism"} <= set(a)
+    wl8, local, scaling = bench.sharded_workload(synth.LARGE_DASGD, 8)
+    assert (wl8.W, local, scaling) == (8, 1, "weak") and wl8.stream_seeds == tuple(range(2, 10))
+    wl2, local, scaling = bench.sharded_workload(synth.LARGE_DASGD, 2)
+    assert (wl2.W, local, scaling) == (4, 2, "strong") and wl2 is synth.LARGE_DASGD
+    assert bench.repeats_for(110.0) == 19 and bench.repeats_for(5000.0) == 1 and bench.repeats_for(1.0) == bench.MAX_REPEATS

@@ -74,7 +74,7 @@ class Port:
     def tensair_message_buffers(self, g, step):
         return self.slots[self._slot(g, step)]
 
-    def tensair_commit_message(self, g, step, n, n_in):
+    def tensair_commit_message(self, g, step, n, n_in, stream=None):
         assert not (self.first <= g < self.first + LOCAL)
         assert self.sched.on_train(g, step) == B.OK, "slot still has recipients"
         self.held[self._slot(g, step)] = (g, step, n, n_in)
@@ -112,7 +112,8 @@ class Port:
 
 
 port = Port()
-grp = ShardedReplicas(port, rank, world, LOCAL, dist=dist)
+OVERLAP = int(sys.argv[3])
+grp = ShardedReplicas(port, rank, world, LOCAL, dist=dist, max_delay=D, seed=SEED, overlap=bool(OVERLAP))
 logs = {r: [] for r in range(LOCAL)}
 for t in range(STEPS):
     for r in range(LOCAL):
@@ -120,15 +121,17 @@ for t in range(STEPS):
     grp.exchange(t)
     grp.apply(t)
 grp.drain()
-out = {"rank": rank, "applied": port.applied, "sent": grp.bytes_sent, "received": grp.bytes_received}
+assert not grp._flying, "a transfer was never waited for"
+out = {"rank": rank, "applied": port.applied, "sent": grp.bytes_sent, "received": grp.bytes_received,
+       "at_own_step": grp.bytes_waited_at_own_step, "later": grp.bytes_waited_later}
 open(sys.argv[1] + f".{rank}", "w").write(json.dumps(out))
 dist.barrier()
 dist.destroy_process_group()
 """
 
 
-@pytest.mark.parametrize("world,local,port", [(2, 1, 29621), (2, 2, 29622), (3, 1, 29623)])
-def test_every_rank_applies_every_message_once_in_the_one_process_order(tmp_path, world, local, port):
+@pytest.mark.parametrize("world,local,port,overlap", [(2, 1, 29621, 1), (2, 2, 29622, 1), (3, 1, 29623, 1), (2, 1, 29624, 0)])
+def test_every_rank_applies_every_message_once_in_the_one_process_order(tmp_path, world, local, port, overlap):
     from paper_2211_10280_b200 import binding as B
 
     script = tmp_path / "worker.py"
@@ -136,7 +139,8 @@ def test_every_rank_applies_every_message_once_in_the_one_process_order(tmp_path
     out = tmp_path / "out"
     env = dict(os.environ, MASTER_ADDR="127.0.0.1")
     subprocess.check_call([sys.executable, "-m", "torch.distributed.run", "--nnodes=1", f"--nproc-per-node={world}",
-                           "--master-addr", "127.0.0.1", "--master-port", str(port), str(script), str(out), str(local)],
+                           "--master-addr", "127.0.0.1", "--master-port", str(port), str(script), str(out), str(local),
+                           str(overlap)],
                           env=env, cwd=str(ROOT), timeout=300)
     res = [json.loads(Path(f"{out}.{r}").read_text()) for r in range(world)]
     W, D, steps = world * local, 2, 9
@@ -160,3 +164,11 @@ def test_every_rank_applies_every_message_once_in_the_one_process_order(tmp_path
             assert len(got[g]) == (W - 1) * steps and len(set(got[g])) == len(got[g])
     # every byte sent is received once per other rank
     assert sum(x["sent"] for x in res) == sum(x["received"] for x in res) > 0
+    # every received byte was waited for exactly once: at its own step when it was due there, later otherwise
+    for x in res:
+        assert x["at_own_step"] + x["later"] == x["received"]
+        if overlap:
+            # delays are uniform in {0, 1, 2}: a good share of what a rank receives is not due at its own step
+            assert x["later"] > 0.2 * x["received"]
+        else:
+            assert x["later"] == 0

@@ -4,13 +4,15 @@ Such a caller (a plug-in living inside a host application's fixed memory plan, a
 of the allocator) cannot size and provide per-batch scratch; the entry point takes it from a fixed array
 inside the library.  The check: through the C ABI, on the same seeded inputs, two calls in a row must
 give what tensair_train_batch gives - same loss, same message rows, deltas and tables within the
-one-batch parity tolerance (they are in fact bit-identical).  This file sorts last on purpose, so that a
-run that stops at the first failure has already run every other test; it also passes on its own.
+one-batch parity tolerance (they are in fact bit-identical) - and what the CPU oracle gives for the same
+batches; and a call that is not the first on its device must leave the device's free memory exactly as
+it found it.  This file sorts last on purpose, so that a run that stops at the first failure has already
+run every other test; it also passes on its own.
 """
 import numpy as np
 import pytest
 
-from parity_utils import rel_err
+from parity_utils import compare_message, compare_tables, rel_err
 from paper_2211_10280_b200 import synth
 
 pytestmark = pytest.mark.gpu
@@ -34,11 +36,27 @@ def test_static_scratch_entry_point_matches_train_batch_on_two_calls_in_a_row():
     stream = synth.token_stream(wl, 0)
     counts = synth.stream_counts([stream], wl.V)
     t_in, t_out = synth.random_tables(wl.V, wl.d, 31, scale=0.25)
+    from oracle import Oracle
+
     ref, new = _context(wl, counts, t_in, t_out), _context(wl, counts, t_in, t_out)
+    orc = Oracle(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=wl.W, lr=wl.lr, max_delay=wl.max_delay,
+                 seed=wl.seed, counts=counts, init_in=t_in, init_out=t_out, reduction=wl.reduction)
     for b in range(2):
         toks = torch.from_numpy(stream[b]).cuda()
         loss_ref, info_ref = ref.tensair_train_batch(0, toks, b, want_loss=True, want_info=True)
+        torch.cuda.synchronize()
+        free_before = torch.cuda.mem_get_info()[0]
         loss_new, info_new = new.tensair_train_batch_static(0, toks, b, want_loss=True, want_info=True)
+        torch.cuda.synchronize()
+        if b > 0:       # the first call on a device may make the driver load the module that holds the array
+            assert torch.cuda.mem_get_info()[0] == free_before, "the call changed the device's free memory"
+        rc, loss_orc, rows_orc = orc.train_batch(0, stream[b], b)
+        assert rc == 0 and info_new.n_rows == rows_orc
+        assert loss_new == pytest.approx(loss_orc, rel=1e-12)
+        assert np.array_equal(new.tensair_read_negatives(), orc.read_negatives())
+        assert np.max(np.abs(new.tensair_read_scalars() - orc.read_g())) <= 1e-13
+        compare_message(orc, new, 0, b, TOL)
+        compare_tables(orc, new, 0, (b + 1) * TOL)
         assert (info_new.n_rows, info_new.n_in_rows, info_new.n_pairs) == (info_ref.n_rows, info_ref.n_in_rows, info_ref.n_pairs)
         assert loss_new == pytest.approx(loss_ref, rel=1e-12)
         assert np.array_equal(new.tensair_read_negatives(), ref.tensair_read_negatives())
