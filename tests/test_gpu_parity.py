@@ -853,3 +853,14 @@ def test_subnormal_rows_and_deltas_are_added_like_the_oracle_adds_them(torch):
             got = g.tensair_read_embeddings(j, which)
             assert np.array_equal(o.read_embeddings(j, which).view(np.uint32), got.view(np.uint32)), (j, which)
     assert (np.abs(got[got != 0]) < sub).any()
+
+
+def test_long_parity_runner_on_a_short_drifting_run(torch):
+    """tests/long_parity.py (the runner of the full-length parity runs) on a reduced drifting workload: 25 steps of
+    3 replicas across two sampler rebuilds, checked every 10 steps."""
+    import long_parity
+
+    wl = synth.scaled(synth.LARGE_DRIFT, V=8000, d=40, batch=256, W=3, k=5, drift_every=10, stream_seeds=(6, 7, 8))
+    res = long_parity.run(wl, steps=25, check_every=10)
+    assert res["sampler_rebuilds"] == 2 and [c["step"] for c in res["checks"]] == [10, 20, 25]
+    assert res["max_rel_err"] <= TOL_200 and res["after_drain"] <= TOL_200

@@ -124,3 +124,118 @@ def test_a_slot_still_to_be_applied_is_not_handed_out_for_receiving(torch):
         a.tensair_commit_message(0, 1, 0, 0)
     with pytest.raises(B.TensairError):               # a local receiver is applied for real
         a.tensair_shadow_apply(0, 0)
+
+
+class LoopbackDist:
+    """all_gather and broadcast of torch.distributed between THREADS of one process, one thread per shard, all on one
+    GPU: a transfer is a device copy enqueued on the receiver's current stream behind an event of the sender's
+    stream - what a collective between GPUs does to the streams it is enqueued on.  Every rendezvous has a time
+    limit, so a failing thread fails the test instead of stalling it."""
+
+    def __init__(self, torch, world):
+        import threading
+
+        self.torch, self.world = torch, world
+        self.barrier = threading.Barrier(world, timeout=120)
+        self.box = [None] * world
+        self.done = [None] * world
+        self.me = threading.local()
+
+    def _event(self):
+        ev = self.torch.cuda.Event()
+        ev.record()                       # on the calling thread's current stream
+        return ev
+
+    def _finish(self):
+        # nobody reuses a source tensor before every receiver's copy from it has run
+        self.done[self.me.rank] = self._event()
+        self.barrier.wait()
+        for ev in self.done:
+            self.torch.cuda.current_stream().wait_event(ev)
+        self.barrier.wait()
+
+    def all_gather(self, out, tensor, group=None):
+        self.box[self.me.rank] = (tensor, self._event())
+        self.barrier.wait()
+        for i, (src, ev) in enumerate(self.box):
+            self.torch.cuda.current_stream().wait_event(ev)
+            out[i].copy_(src)
+        self._finish()
+
+    def broadcast(self, tensor, src, group=None, async_op=False):
+        if self.me.rank == src:
+            self.box[src] = (tensor, self._event())
+        self.barrier.wait()
+        if self.me.rank != src:
+            data, ev = self.box[src]
+            self.torch.cuda.current_stream().wait_event(ev)
+            tensor.copy_(data)
+        self._finish()
+
+
+@pytest.mark.parametrize("world,local,overlap", [(2, 1, True), (2, 2, True), (4, 1, True), (2, 1, False)])
+def test_exchange_on_a_communication_stream_equals_the_one_context_job(torch, world, local, overlap):
+    """The exchange layer itself (row counts read on the device, broadcasts and the received messages' indices on a
+    communication stream, the training stream waiting only for what is due) driven by one thread per shard over a
+    loop-back transport: tables and delivery logs must equal the one-context job bit for bit, and with delays up
+    to 2 a good part of what a shard receives must not have been waited for at its own step."""
+    import threading
+
+    W = world * local
+    wl = synth.scaled(synth.LARGE_DASGD, V=30_000, d=300, batch=1024, W=W, stream_seeds=tuple(range(20, 20 + W)),
+                      max_delay=2, batches=9)
+    streams = synth.all_streams(wl, wl.batches)
+    counts = synth.stream_counts(streams, wl.V)
+    kw = dict(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, lr=wl.lr, max_delay=wl.max_delay,
+              seed=wl.seed, counts=counts, reduction=wl.reduction)
+    one = B.Context(W=W, **kw)
+    for t in range(wl.batches):
+        for g in range(W):
+            one.tensair_train_batch(g, dev(torch, streams[g][t]), t)
+        one.tensair_apply_step(t)
+    one.tensair_drain()
+
+    wire_ = LoopbackDist(torch, world)
+    results, errors = [None] * world, []
+
+    def shard(p):
+        try:
+            wire_.me.rank = p
+            stream = torch.cuda.Stream()
+            with torch.cuda.stream(stream):
+                ctx = B.Context(W=local, world_replicas=W, first_replica=p * local, stream=stream, **kw)
+                grp = ShardedReplicas(ctx, p, world, local, dist=wire_, count_device="cuda", overlap=overlap)
+                toks = [[dev(torch, streams[p * local + r][t]) for r in range(local)] for t in range(wl.batches)]
+                for t in range(wl.batches):
+                    for r in range(local):
+                        ctx.tensair_train_batch(r, toks[t][r], t)
+                    grp.exchange(t)
+                    grp.apply(t)
+                grp.drain()
+                assert ctx.tensair_sync() == B.OK and not grp._flying
+                results[p] = ([ctx.tensair_read_delivery_log(r) for r in range(local)],
+                              [[ctx.tensair_read_embeddings(r, which) for which in (0, 1)] for r in range(local)],
+                              (grp.bytes_received, grp.bytes_waited_at_own_step, grp.bytes_waited_later, grp.bytes_sent))
+                ctx.close()
+        except BaseException as e:          # noqa: BLE001 - reported by the main thread
+            errors.append((p, repr(e)))
+            wire_.barrier.abort()
+
+    threads = [threading.Thread(target=shard, args=(p,)) for p in range(world)]
+    for th in threads:
+        th.start()
+    for th in threads:
+        th.join(timeout=600)
+    assert not errors, errors
+    assert all(r is not None for r in results)
+    for p in range(world):
+        logs, tables, (received, own_step, later, sent) = results[p]
+        for r in range(local):
+            g = p * local + r
+            assert np.array_equal(logs[r], one.tensair_read_delivery_log(g)), "delivery order or staleness differs"
+            for which in (0, 1):
+                want = one.tensair_read_embeddings(g, which)
+                assert np.array_equal(tables[r][which].view(np.uint32), want.view(np.uint32)), (g, which)
+        assert own_step + later == received > 0
+        assert (later > 0.2 * received) if overlap else (later == 0)
+    assert sum(r[2][3] for r in results) == sum(r[2][0] for r in results)
