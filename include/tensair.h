@@ -434,7 +434,13 @@ TENSAIR_API const char* tensair_last_error(const tensair_ctx* ctx);
  *   bit 3 (8)  a merged message outgrew its slot                  -> TENSAIR_EBOUNDS
  * tensair_error_of_flags gives the code a value of the word stands for (host only, no context needed).
  * tensair_raise_error_flags ORs bits into a context's word from the host, as a kernel would have: a hook for testing
- * a caller's error handling without making a GPU misbehave.  Synchronises. */
+ * a caller's error handling without making a GPU misbehave.  Synchronises.
+ *
+ * Checked build: compiled with -DTENSAIR_BOUNDS (`python -m paper_2211_10280_b200.build --bounds`, which writes
+ * libtensair_checked.so beside the normal library), every index that a kernel computes from data - row ids against
+ * the table, message rows against the slot, sort positions, list and scratch offsets - is compared with its bound
+ * before use; a violation raises bit 2 and skips the access.  tensair_checked_build() says which build is loaded. */
+TENSAIR_API int tensair_checked_build(void);
 TENSAIR_API int tensair_error_of_flags(uint32_t flags);
 TENSAIR_API int tensair_raise_error_flags(tensair_ctx* ctx, uint32_t flags);
 

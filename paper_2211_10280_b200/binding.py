@@ -11,8 +11,12 @@ from typing import Optional
 
 import numpy as np
 
+import os
+
 _HERE = Path(__file__).resolve().parent
-LIB_PATH = _HERE / "libtensair.so"
+# TENSAIR_CHECKED=1 loads the checked build (every data-dependent index compared with its bound on the device)
+CHECKED = os.environ.get("TENSAIR_CHECKED", "0") == "1"
+LIB_PATH = _HERE / ("libtensair_checked.so" if CHECKED else "libtensair.so")
 
 SUM, MEAN = 0, 1
 OK, EINVAL, ENOMEM, ECUDA, EBADTOKEN, EPENDING, ENOTFOUND, ETIMEOUT, EBOUNDS = 0, -1, -2, -3, -4, -5, -6, -7, -8
@@ -105,6 +109,7 @@ SYMBOLS = {
     "tensair_strerror": (C.c_char_p, [_int]),
     "tensair_last_error": (C.c_char_p, [_vp]),
     "tensair_error_of_flags": (_int, [_u32]),
+    "tensair_checked_build": (_int, []),
     "tensair_raise_error_flags": (_int, [_vp, _u32]),
     "tensair_build_alias_host": (_int, [_vp, _u32, _vp, _vp]),
     "tensair_philox4x32_10": (None, [_P(_u32), _P(_u32), _P(_u32)]),
@@ -124,7 +129,8 @@ def lib():
     global _lib
     if _lib is None:
         if not LIB_PATH.exists():
-            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2211_10280_b200.build`")
+            raise RuntimeError(f"{LIB_PATH} is missing: build it with `python -m paper_2211_10280_b200.build"
+                               f"{' --bounds' if CHECKED else ''}`")
         L = C.CDLL(str(LIB_PATH))
         for name, (res, args) in SYMBOLS.items():
             fn = getattr(L, name)

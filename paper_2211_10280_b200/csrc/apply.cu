@@ -15,13 +15,15 @@ GridShape& grid_shape() {
 template <int NV>
 __global__ void __launch_bounds__(256)
 k_apply(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids, const float4* __restrict__ delta,
-        float4* __restrict__ table, uint32_t d4, uint32_t stride4, int input_rows_only) {
+        float4* __restrict__ table, uint32_t d4, uint32_t stride4, int input_rows_only, Limits lim) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const uint32_t limit = input_rows_only ? hdr->n_in_rows : hdr->n_rows;
+    if (!in_bounds(lim, limit, (uint64_t)lim.slot_rows + 1)) return;
     for (uint32_t m = warp; m < limit; m += nwarps) {
         const uint32_t id = __ldg(ids + m);
+        if (!in_bounds(lim, id, lim.table_rows)) continue;
         const float4* __restrict__ src = delta + (size_t)m * stride4;
         float4* __restrict__ dst = table + (size_t)id * stride4;
         float4 a[NV], b[NV];
@@ -52,7 +54,7 @@ cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uin
     Timed timed(L, input_rows_only ? K_APPLY_INPUT_ROWS : K_APPLY_MESSAGE);
 #define TENSAIR_APPLY(NV)                                                                 \
     k_apply<NV><<<L.sms * grid_shape().apply_blocks_per_sm, 256, 0, L.stream>>>(hdr, ids, d4p, t4, s.d4, stride4, \
-                                                                               input_rows_only)
+                                                                               input_rows_only, L.lim)
     if (s.d4 <= 32) TENSAIR_APPLY(1);
     else if (s.d4 <= 64) TENSAIR_APPLY(2);
     else if (s.d4 <= 96) TENSAIR_APPLY(3);
@@ -123,7 +125,7 @@ constexpr int kStepThreads = 128;
 template <int NV>
 __global__ void __launch_bounds__(kStepThreads)
 k_apply_step(StepMessages f, uint32_t n_receivers, float4* __restrict__ tables, size_t replica4, uint32_t d4,
-             uint32_t stride4, uint32_t n_buckets) {
+             uint32_t stride4, uint32_t n_buckets, Limits lim) {
     // two copies, used by alternate buckets: a warp may note the next bucket while another still works on this one
     __shared__ uint32_t first_row[2][kMaxStepMessages];
     __shared__ uint32_t held[2][kMaxStepMessages];
@@ -154,10 +156,21 @@ k_apply_step(StepMessages f, uint32_t n_receivers, float4* __restrict__ tables, 
             uint32_t todo = __ballot_sync(0xFFFFFFFFu, ((held_mine >> j) & 1u) && ((set_mine >> rcv) & 1u));
             if (!todo) continue;
             const uint32_t id = (b << kBucketShift) + j;
+            if (!in_bounds(lim, id, lim.table_rows)) continue;
             float4* dst = tables + (size_t)rcv * replica4 + (size_t)id * stride4;
             float4 r[NV], a[NV];
             uint32_t k = (uint32_t)__ffs((int)todo) - 1u;
             todo &= todo - 1;
+#ifdef TENSAIR_BOUNDS
+            {   // every message that holds the id must hold it inside its slot
+                bool inside = true;
+                for (uint32_t rest = todo | (1u << k); rest; rest &= rest - 1) {
+                    const uint32_t kk = (uint32_t)__ffs((int)rest) - 1u;
+                    inside = inside && in_bounds(lim, first_row[turn][kk] + __popc(held[turn][kk] & ((1u << j) - 1u)), lim.slot_rows);
+                }
+                if (!inside) continue;
+            }
+#endif
             const float4* __restrict__ src = reinterpret_cast<const float4*>(f.delta[k]) +
                 (size_t)(first_row[turn][k] + __popc(held[turn][k] & ((1u << j) - 1u))) * stride4;
 #pragma unroll
@@ -199,7 +212,7 @@ cudaError_t launch_apply_step(const Launcher& L, const StepMessages& f, uint32_t
     uint32_t blocks = (uint32_t)(L.sms * grid_shape().fused_blocks_per_sm);
     if (blocks > nb) blocks = nb;
     Timed timed(L, kind);
-#define TENSAIR_STEP(NV) k_apply_step<NV><<<blocks, kStepThreads, 0, L.stream>>>(f, n_receivers, t4, replica_floats / 4, s.d4, stride4, nb)
+#define TENSAIR_STEP(NV) k_apply_step<NV><<<blocks, kStepThreads, 0, L.stream>>>(f, n_receivers, t4, replica_floats / 4, s.d4, stride4, nb, L.lim)
     if (s.d4 <= 32) TENSAIR_STEP(1);
     else if (s.d4 <= 64) TENSAIR_STEP(2);
     else if (s.d4 <= 96) TENSAIR_STEP(3);

@@ -78,6 +78,30 @@ constexpr uint32_t kErrTimeout = 2u;    // a bounded wait for a warp's own bulk 
 constexpr uint32_t kErrBounds = 4u;     // checked build: an index left its array; the access was skipped
 constexpr uint32_t kErrOverflow = 8u;   // a merged message had more rows than its slot holds; the rest was dropped
 
+// Sizes of the arrays that kernels index with values computed from data.  In a checked build (-DTENSAIR_BOUNDS)
+// every such index is compared with its bound first; one out of bounds raises kErrBounds in the error word and the
+// access is skipped - nothing traps.  In a normal build the checks compile to nothing.
+struct Limits {
+    uint32_t* err;
+    uint32_t table_rows;   // 2V rows of one replica's unified table
+    uint32_t slot_rows;    // rows a message slot holds
+    uint32_t batch_rows;   // rows the message of one batch can have (bounds the per-batch segment list)
+    uint32_t items;        // sort items of a batch
+    uint32_t contrib;      // contributions of a batch (row ids, gradient scalars)
+    uint32_t positions;    // partial centre gradients of a batch: two per position
+    uint32_t long_rows;    // entries of the long-row list
+    uint32_t chunks;       // entries of the chunk list and of the chunk partials
+};
+#ifdef TENSAIR_BOUNDS
+__device__ inline bool in_bounds(const Limits& lim, uint64_t index, uint64_t bound) {
+    if (index < bound) return true;
+    atomicOr(lim.err, kErrBounds);
+    return false;
+}
+#else
+__device__ __forceinline__ bool in_bounds(const Limits&, uint64_t, uint64_t) { return true; }
+#endif
+
 struct Shape {
     uint32_t V, d, d4, stride, w, k, K1;
 };

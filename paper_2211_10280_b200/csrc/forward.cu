@@ -98,7 +98,7 @@ __global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d, uint32_t stride, uint32_t w,
           uint32_t k, uint32_t chunk_rows, uint32_t warp_stage, const float* __restrict__ table, const uint32_t* __restrict__ rows,
           Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err,
-          const uint32_t* __restrict__ owned, const uint32_t* __restrict__ n_owned) {
+          const uint32_t* __restrict__ owned, const uint32_t* __restrict__ n_owned, Limits lim) {
     if (*err) return;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -159,7 +159,7 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d, u
                 const uint32_t nr = K1 - j0 < chunk_rows ? K1 - j0 : chunk_rows;
                 uint32_t rid = __shfl_sync(0xFFFFFFFFu, ids_pair, (j0 + lane) & 31u);
                 if (!ids_in_lanes) rid = lane < nr ? __ldg(rows + cbase + j0 + lane) : 0u;
-                const bool mine = lane < nr && (j0 + lane == 0 || rid != ctx);
+                const bool mine = lane < nr && (j0 + lane == 0 || rid != ctx) && in_bounds(lim, rid, V);
                 const uint32_t live = __ballot_sync(0xFFFFFFFFu, mine);
                 // stage the live rows: the buffer was last read by this warp, so order those reads first
                 fence_generic_to_async();
@@ -236,7 +236,7 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d, u
                     const double y = positive ? x : -x;   // the term is -log(sigmoid(y))
                     if (writer) loss += (y < 0.0 ? -y : 0.0) + sl.softplus;
                 }
-                if (writer && jr < nr) rec[cbase + j0 + jr] = Rec{g, centre, 0u};
+                if (writer && jr < nr && in_bounds(lim, (uint64_t)cbase + j0 + jr, lim.contrib)) rec[cbase + j0 + jr] = Rec{g, centre, 0u};
                 // 4. centre gradient: acc += g_j * u_j
                 if (full) {
                     double gw[NR];
@@ -273,7 +273,7 @@ k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d, u
                 }
             }
         }
-        if (failed) break;
+        if (failed || !in_bounds(lim, 2ull * q + side, lim.positions)) break;
         double2* out = reinterpret_cast<double2*>(gin_pos + (size_t)(2 * q + side) * stride);
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -354,7 +354,7 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
         k_forward<NV, CR, NR, VW><<<grid, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d, s.stride, s.w, s.k,   \
                                                                             chunk_rows, warp_stage, table, rows,    \
                                                                             rec, gin_pos, loss_pos, err, owned,     \
-                                                                            n_owned);                               \
+                                                                            n_owned, L.lim);                        \
     } while (0)
     // k = 5 (six rows per pair) is common enough to have whole chunks of its own
 #define TENSAIR_FWD_ROWS(NV, VW)                                                     \

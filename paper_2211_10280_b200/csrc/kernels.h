@@ -41,6 +41,7 @@ struct Launcher {
     int sms;              // multiprocessors of the device
     Profiler* prof;       // nullable
     int device = 0;       // ordinal of the device the stream belongs to
+    Limits lim = {};      // array bounds handed to the kernels (used by the checked build only)
 };
 constexpr int kMaxDevices = 64;   // per-device launch state (function attributes, symbol addresses) is kept up to here
 
@@ -79,7 +80,8 @@ cudaError_t launch_validate(const Launcher& L, const int32_t* tok, uint32_t n, u
                             uint32_t* owned, uint32_t* n_owned, uint32_t W, uint32_t replica, uint64_t seed);
 cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, uint32_t replica,
                            uint32_t batch_lo, uint64_t seed, const uint2* alias_tab, uint32_t* rows,
-                           item_t* items, unsigned long long* counts, const uint32_t* err, const uint8_t* owner);
+                           item_t* items, unsigned long long* counts, uint32_t* err, const uint8_t* owner, bool check,
+                           bool count);
 cudaError_t launch_init_input_table(const Launcher& L, float* table, const Shape& s, uint64_t seed);
 void build_alias_host(const uint64_t* counts, uint32_t V, uint32_t* thresh, uint32_t* alias);
 int alias_mass_bits(uint32_t V);
@@ -113,9 +115,13 @@ cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t 
 
 // message.cu
 uint32_t heads_tiles(uint32_t n_items);
+// tok / counts / owner: when counts is given, the batch's n tokens are added to the running unigram counts here
+// (the first kernel that runs once the whole batch is known to be valid); nullptr = they were counted already.
+// long_counters: 4 words (long rows, chunks, and the ticket that picks the block that scans the tile counts).
 cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
                          MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
-                         const Rec* rec, Rec* terms, const uint32_t* err, LongRow* long_rows, ChunkItem* chunk_items);
+                         const Rec* rec, Rec* terms, const uint32_t* err, LongRow* long_rows, ChunkItem* chunk_items,
+                         const int32_t* tok, uint32_t n, unsigned long long* counts, const uint8_t* owner);
 cudaError_t launch_reduce_rows(const Launcher& L, const Rec* terms, const MsgHeader* hdr, const uint32_t* ids,
                                const uint32_t* seg_start, const double* gin_pos, float* table, float* delta,
                                const Shape& s, double scale);

@@ -36,46 +36,23 @@ __device__ inline uint32_t head_flags(const item_t* __restrict__ sorted, uint32_
     return flags;
 }
 
-__global__ void __launch_bounds__(kHeadThreads)
-k_heads_count(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t* __restrict__ tile_counts,
-              const uint32_t* __restrict__ err) {
-    if (*err) return;
-    __shared__ uint32_t warp_sum[kHeadThreads / 32];
-    uint32_t keys[kHeadItems];
-    const uint32_t first = blockIdx.x * kHeadTile + threadIdx.x * kHeadItems;
-    uint32_t c = __popc(head_flags(sorted, n_items, first, keys));
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
-    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = c;
-    __syncthreads();
-    if (threadIdx.x == 0) {
-        uint32_t t = 0;
-        for (int i = 0; i < kHeadThreads / 32; ++i) t += warp_sum[i];
-        tile_counts[blockIdx.x] = t;
-    }
-}
-
-// One block: exclusive scan of the tile counts, message header, counters of the long-row lists.
-__global__ void __launch_bounds__(1024)
-k_heads_scan(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, uint32_t* __restrict__ tile_counts,
-             uint32_t tiles, MsgHeader* __restrict__ hdr, uint32_t* __restrict__ seg_start,
-             uint32_t* __restrict__ long_counters, const uint32_t* __restrict__ err) {
-    __shared__ uint32_t warp_tot[32];
+// Exclusive scan of the tile counts (in place), message header, reset of the long-row counters: the work of one
+// block of kHeadThreads threads.
+__device__ inline void scan_tile_counts(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V,
+                                        uint32_t* tile_counts, uint32_t tiles, MsgHeader* __restrict__ hdr,
+                                        uint32_t* __restrict__ seg_start, uint32_t* __restrict__ long_counters) {
+    __shared__ uint32_t warp_tot[kHeadThreads / 32];
     __shared__ uint32_t carry_s;
     if (threadIdx.x == 0) {
         long_counters[0] = 0;
         long_counters[1] = 0;
         carry_s = 0;
     }
-    if (*err) {
-        if (threadIdx.x == 0) *hdr = MsgHeader{0, 0, 0, 0};
-        return;
-    }
     __syncthreads();
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
-    for (uint32_t base = 0; base < tiles; base += 1024) {
+    for (uint32_t base = 0; base < tiles; base += kHeadThreads) {
         const uint32_t idx = base + threadIdx.x;
-        const uint32_t v = idx < tiles ? tile_counts[idx] : 0;
+        const uint32_t v = idx < tiles ? __ldcg(tile_counts + idx) : 0;   // written by other blocks of this launch
         uint32_t incl = v;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -84,21 +61,12 @@ k_heads_scan(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, ui
         }
         if (lane == 31) warp_tot[wid] = incl;
         __syncthreads();
-        if (wid == 0) {
-            const uint32_t t = warp_tot[lane];
-            uint32_t ti = t;
-#pragma unroll
-            for (int o = 1; o < 32; o <<= 1) {
-                const uint32_t u = __shfl_up_sync(0xFFFFFFFFu, ti, o);
-                if (lane >= (uint32_t)o) ti += u;
-            }
-            warp_tot[lane] = ti - t;
-        }
-        __syncthreads();
+        uint32_t before = 0;
+        for (uint32_t x = 0; x < wid; ++x) before += warp_tot[x];
         const uint32_t carry = carry_s;
-        if (idx < tiles) tile_counts[idx] = carry + warp_tot[wid] + incl - v;
+        if (idx < tiles) tile_counts[idx] = carry + before + incl - v;
         __syncthreads();
-        if (threadIdx.x == 1023) carry_s = carry + warp_tot[wid] + incl;
+        if (threadIdx.x == kHeadThreads - 1) carry_s = carry + before + incl;
         __syncthreads();
     }
     if (threadIdx.x == 0) {
@@ -112,10 +80,53 @@ k_heads_scan(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, ui
     }
 }
 
+// Heads per tile; the block that finishes last (a ticket counts the blocks) scans the tile counts, so that no
+// separate one-block launch stands between this kernel and the one that writes the heads.  Also the first kernel
+// that runs once a batch is known to be valid as a whole: it adds the batch's tokens to the running unigram counts.
+__global__ void __launch_bounds__(kHeadThreads)
+k_heads_count(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts, uint32_t tiles,
+              MsgHeader* __restrict__ hdr, uint32_t* __restrict__ seg_start, uint32_t* __restrict__ long_counters,
+              const uint32_t* __restrict__ err, const int32_t* __restrict__ tok, uint32_t n,
+              unsigned long long* __restrict__ counts, const uint8_t* __restrict__ owner) {
+    if (*err) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) {
+            *hdr = MsgHeader{0, 0, 0, 0};
+            long_counters[0] = 0;
+            long_counters[1] = 0;
+        }
+        return;
+    }
+    __shared__ uint32_t warp_sum[kHeadThreads / 32];
+    __shared__ uint32_t last_s;
+    if (counts) {
+        const uint32_t q = blockIdx.x * kHeadThreads + threadIdx.x;      // there are at least as many items as tokens
+        if (q < n && (!owner || owner[q])) atomicAdd(counts + (uint32_t)tok[q], 1ULL);
+    }
+    uint32_t keys[kHeadItems];
+    const uint32_t first = blockIdx.x * kHeadTile + threadIdx.x * kHeadItems;
+    uint32_t c = __popc(head_flags(sorted, n_items, first, keys));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) c += __shfl_xor_sync(0xFFFFFFFFu, c, o);
+    if ((threadIdx.x & 31) == 0) warp_sum[threadIdx.x >> 5] = c;
+    __syncthreads();
+    if (threadIdx.x == 0) {
+        uint32_t t = 0;
+        for (int i = 0; i < kHeadThreads / 32; ++i) t += warp_sum[i];
+        tile_counts[blockIdx.x] = t;
+        __threadfence();                                       // the count is visible before the ticket is taken
+        last_s = atomicAdd(long_counters + 2, 1u) == tiles - 1 ? 1u : 0u;
+    }
+    __syncthreads();
+    if (!last_s) return;
+    __threadfence();
+    if (threadIdx.x == 0) long_counters[2] = 0;                // ready for the next batch
+    scan_tile_counts(sorted, n_items, V, tile_counts, tiles, hdr, seg_start, long_counters);
+}
+
 __global__ void __launch_bounds__(kHeadThreads)
 k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, const uint32_t* __restrict__ tile_base,
               MsgHeader* __restrict__ hdr, uint32_t* __restrict__ ids, uint32_t* __restrict__ seg_start,
-              const Rec* __restrict__ rec, Rec* __restrict__ terms, const uint32_t* __restrict__ err) {
+              const Rec* __restrict__ rec, Rec* __restrict__ terms, const uint32_t* __restrict__ err, Limits lim) {
     if (*err) return;
     // terms[i] = scalar and centre token of the i-th sorted contribution (for an input-row item: the
     // centre position), so that the row sums read their terms contiguously
@@ -123,7 +134,7 @@ k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, c
         const item_t it = sorted[i];
         const uint32_t key = item_key(it);
         if (key < V) terms[i] = Rec{1.0, item_payload(it), 0u};
-        else if (key < 2 * V) terms[i] = rec[item_payload(it)];
+        else if (key < 2 * V && in_bounds(lim, item_payload(it), lim.contrib)) terms[i] = rec[item_payload(it)];
     }
     __shared__ uint32_t warp_tot[kHeadThreads / 32];
     uint32_t keys[kHeadItems];
@@ -144,7 +155,7 @@ k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, c
     uint32_t prev = first > 0 && first <= n_items ? item_key(sorted[first - 1]) : 0u;
 #pragma unroll
     for (int i = 0; i < kHeadItems; ++i) {
-        if (flags & (1u << i)) {
+        if ((flags & (1u << i)) && in_bounds(lim, m, (uint64_t)lim.batch_rows + 1)) {
             const uint32_t key = keys[i];
             seg_start[m] = first + i;
             if (key < 2 * V) ids[m] = key;
@@ -161,7 +172,7 @@ k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, c
 __global__ void __launch_bounds__(256)
 k_list_long_rows(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ seg_start,
                  uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows,
-                 ChunkItem* __restrict__ chunk_items, const uint32_t* __restrict__ err) {
+                 ChunkItem* __restrict__ chunk_items, const uint32_t* __restrict__ err, Limits lim) {
     if (*err) return;
     const uint32_t n_rows = hdr->n_rows, lane = threadIdx.x & 31;
     const uint32_t first = (blockIdx.x * blockDim.x + threadIdx.x) - lane;   // row of lane 0
@@ -174,7 +185,10 @@ k_list_long_rows(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__
                 nch = (len + kChunk - 1) / kChunk;
                 const uint32_t slot = atomicAdd(long_counters, 1u);
                 base = atomicAdd(long_counters + 1, nch);
-                long_rows[slot] = LongRow{m, base, nch};
+                if (in_bounds(lim, slot, lim.long_rows) && in_bounds(lim, (uint64_t)base + nch - 1, lim.chunks))
+                    long_rows[slot] = LongRow{m, base, nch};
+                else
+                    nch = 0;
             }
         }
         uint32_t todo = __ballot_sync(0xFFFFFFFFu, nch != 0);
@@ -190,23 +204,22 @@ k_list_long_rows(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__
 
 cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_items, uint32_t V, uint32_t* tile_counts,
                          MsgHeader* hdr, uint32_t* ids, uint32_t* seg_start, uint32_t* long_counters,
-                         const Rec* rec, Rec* terms, const uint32_t* err, LongRow* long_rows, ChunkItem* chunk_items) {
+                         const Rec* rec, Rec* terms, const uint32_t* err, LongRow* long_rows, ChunkItem* chunk_items,
+                         const int32_t* tok, uint32_t n, unsigned long long* counts, const uint8_t* owner) {
     const uint32_t tiles = heads_tiles(n_items);
-    if (tiles) {
-        Timed timed(L, K_HEADS_COUNT);
-        k_heads_count<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, tile_counts, err);
-    }
+    if (!tiles) return cudaSuccess;
     {
-        Timed timed(L, K_HEADS_SCAN);
-        k_heads_scan<<<1, 1024, 0, L.stream>>>(sorted, n_items, V, tile_counts, tiles, hdr, seg_start, long_counters, err);
+        Timed timed(L, K_HEADS_COUNT);
+        k_heads_count<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, tiles, hdr, seg_start,
+                                                            long_counters, err, tok, n, counts, owner);
     }
     if (tiles) {
         Timed timed(L, K_HEADS_WRITE);
-        k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, rec, terms, err);
+        k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, rec, terms, err, L.lim);
     }
     if (tiles) {
         Timed timed(L, K_HEADS_LONG);
-        k_list_long_rows<<<L.sms * 4, 256, 0, L.stream>>>(hdr, seg_start, long_counters, long_rows, chunk_items, err);
+        k_list_long_rows<<<L.sms * 4, 256, 0, L.stream>>>(hdr, seg_start, long_counters, long_rows, chunk_items, err, L.lim);
     }
     return cudaGetLastError();
 }
@@ -235,7 +248,7 @@ struct RowSum {
 template <int NV, int kTermsInFlight>
 __device__ inline void accumulate_segment(const Rec* __restrict__ terms, uint32_t beg, uint32_t end, bool input_row,
                                           const double* __restrict__ gin_pos, const float4* __restrict__ table,
-                                          uint32_t d4, uint32_t stride4, uint32_t lane, RowSum<NV>& sum,
+                                          uint32_t d4, uint32_t stride4, uint32_t lane, RowSum<NV>& sum, const Limits& lim,
                                           bool have_first = false, Rec first = Rec{0.0, 0u, 0u}) {
     for (uint32_t base = beg; base < end; base += 32) {
         const uint32_t cnt = end - base < 32 ? end - base : 32;
@@ -243,16 +256,48 @@ __device__ inline void accumulate_segment(const Rec* __restrict__ terms, uint32_
         if (have_first && base == beg) mine = first;   // the caller fetched the first 32 terms ahead of time
         else if (lane < cnt) mine = terms[base + lane];
         if (input_row) {
-            // sources are the fp64 partial centre gradients of the positions holding this token
-            for (uint32_t t = 0; t < cnt; ++t) {
-                const uint32_t q = __shfl_sync(0xFFFFFFFFu, mine.centre, t);
-                const double2* src = reinterpret_cast<const double2*>(gin_pos + (size_t)q * stride4 * 4);
+            // Sources are the fp64 partial centre gradients of the positions holding this token.
+            if constexpr (kTermsInFlight == 1) {
+                for (uint32_t t = 0; t < cnt; ++t) {
+                    const uint32_t q = __shfl_sync(0xFFFFFFFFu, mine.centre, t);
+                    if (!in_bounds(lim, q, lim.positions)) continue;
+                    const double2* src = reinterpret_cast<const double2*>(gin_pos + (size_t)q * stride4 * 4);
 #pragma unroll
-                for (int j = 0; j < NV; ++j) {
-                    const uint32_t e = lane + 32 * j;
-                    if (e < d4) {
-                        const double2 lo = src[2 * e], hi = src[2 * e + 1];
-                        sum.a[j][0] += lo.x; sum.a[j][1] += lo.y; sum.a[j][2] += hi.x; sum.a[j][3] += hi.y;
+                    for (int j = 0; j < NV; ++j) {
+                        const uint32_t e = lane + 32 * j;
+                        if (e < d4) {
+                            const double2 lo = src[2 * e], hi = src[2 * e + 1];
+                            sum.a[j][0] += lo.x; sum.a[j][1] += lo.y; sum.a[j][2] += hi.x; sum.a[j][3] += hi.y;
+                        }
+                    }
+                }
+            } else {
+                // The chunk kernel, whose segments are long, fetches the rows of several terms before any is added
+                // (in term order), so that several loads are in flight, not one; how many, the row width decides.
+                constexpr int kAhead = NV <= 2 ? 4 : (NV <= 4 ? 2 : 1);
+                for (uint32_t t0 = 0; t0 < cnt; t0 += kAhead) {
+                    double2 part[kAhead][NV][2];
+#pragma unroll
+                    for (int t = 0; t < kAhead; ++t) {
+                        const uint32_t q = __shfl_sync(0xFFFFFFFFu, mine.centre, (t0 + t) & 31);
+                        const double2* src = reinterpret_cast<const double2*>(gin_pos + (size_t)q * stride4 * 4);
+#pragma unroll
+                        for (int j = 0; j < NV; ++j) {
+                            const uint32_t e = lane + 32 * j;
+                            const bool on = t0 + t < cnt && e < d4 && in_bounds(lim, q, lim.positions);
+                            part[t][j][0] = on ? src[2 * e] : make_double2(0.0, 0.0);
+                            part[t][j][1] = on ? src[2 * e + 1] : make_double2(0.0, 0.0);
+                        }
+                    }
+#pragma unroll
+                    for (int t = 0; t < kAhead; ++t) {
+                        if (t0 + t < cnt) {
+#pragma unroll
+                            for (int j = 0; j < NV; ++j) {
+                                sum.a[j][0] += part[t][j][0].x; sum.a[j][1] += part[t][j][0].y;
+                                sum.a[j][2] += part[t][j][1].x; sum.a[j][3] += part[t][j][1].y;
+                            }
+                        }
                     }
                 }
             }
@@ -266,7 +311,7 @@ __device__ inline void accumulate_segment(const Rec* __restrict__ terms, uint32_
                 const uint32_t from = (t0 + t) & 31;
                 const double g = __shfl_sync(0xFFFFFFFFu, mine.g, from);
                 const uint32_t centre = __shfl_sync(0xFFFFFFFFu, mine.centre, from);
-                const bool on = t0 + t < cnt;
+                const bool on = t0 + t < cnt && in_bounds(lim, centre, lim.table_rows / 2);
                 coef[t] = on ? g * kWidenUp : 0.0;   // exact (|g| <= 1); the factor the widened source lacks
                 src[t] = table + (size_t)(on ? centre : 0u) * stride4;
             }
@@ -362,13 +407,14 @@ __global__ void __launch_bounds__(kReduceThreads)
 k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids,
               const uint32_t* __restrict__ seg_start, const double* __restrict__ gin_pos,
               float4* __restrict__ table, float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4,
-              double scale) {
+              double scale, Limits lim) {
     extern __shared__ __align__(128) float4 out_rows[];   // [warps in block][kOutBuffers][stride4]
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     float4* my_out = out_rows + (size_t)(threadIdx.x >> 5) * kOutBuffers * stride4;
     const uint32_t n_rows = hdr->n_rows;
+    if (!in_bounds(lim, n_rows, (uint64_t)lim.batch_rows + 1)) return;
     const uint32_t row_bytes = d4 * 16;
     const double nscale = -scale;
     struct Meta { uint32_t beg, end, id; };
@@ -392,8 +438,8 @@ k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, 
         if (cur.end - cur.beg <= kChunk) {   // longer rows are on the long-row list and summed by the chunk kernels
             RowSum<NV> sum;
             sum.clear();
-            accumulate_segment<NV, kTermsInFlightRows>(terms, cur.beg, cur.end, cur.id < V, gin_pos, table, d4, stride4, lane, sum, true,
-                                   cur_terms);
+            accumulate_segment<NV, kTermsInFlightRows>(terms, cur.beg, cur.end, cur.id < V, gin_pos, table, d4, stride4, lane, sum, lim,
+                                   true, cur_terms);
             // the buffer about to be refilled must have been read by the copies issued from it
             if (lane == 0) bulk_wait_read<kOutBuffers - 1>();
             __syncwarp();
@@ -407,7 +453,7 @@ k_reduce_rows(const Rec* __restrict__ terms, const MsgHeader* __restrict__ hdr, 
             }
             fence_smem_writes_for_async();
             __syncwarp();
-            if (lane == 0) {
+            if (lane == 0 && in_bounds(lim, m, lim.slot_rows) && in_bounds(lim, cur.id, lim.table_rows)) {
                 bulk_store_s2g(delta + (size_t)m * stride4, out, row_bytes);
                 if (cur.id >= V) bulk_add_f32_s2g(table + (size_t)cur.id * stride4, out, row_bytes);
                 bulk_commit();
@@ -427,19 +473,21 @@ __global__ void __launch_bounds__(kReduceThreads)
 k_reduce_chunks(const Rec* __restrict__ terms, const uint32_t* __restrict__ ids, const uint32_t* __restrict__ seg_start,
                 const double* __restrict__ gin_pos, const float4* __restrict__ table,
                 uint32_t V, uint32_t d4, uint32_t stride4, const uint32_t* __restrict__ long_counters,
-                const ChunkItem* __restrict__ chunk_items, double* __restrict__ partials) {
+                const ChunkItem* __restrict__ chunk_items, double* __restrict__ partials, Limits lim) {
     const uint32_t lane = threadIdx.x & 31;
     const uint32_t warp = (blockIdx.x * blockDim.x + threadIdx.x) >> 5;
     const uint32_t nwarps = (gridDim.x * blockDim.x) >> 5;
     const uint32_t n_chunks = long_counters[1];
+    if (!in_bounds(lim, n_chunks, (uint64_t)lim.chunks + 1)) return;
     for (uint32_t x = warp; x < n_chunks; x += nwarps) {
         const ChunkItem ci = chunk_items[x];
+        if (!in_bounds(lim, ci.m, lim.batch_rows)) continue;
         const uint32_t beg = seg_start[ci.m] + ci.chunk * kChunk;
         const uint32_t seg_end = seg_start[ci.m + 1];
         const uint32_t end = beg + kChunk < seg_end ? beg + kChunk : seg_end;
         RowSum<NV> sum;
         sum.clear();
-        accumulate_segment<NV, kTermsInFlightChunks>(terms, beg, end, ids[ci.m] < V, gin_pos, table, d4, stride4, lane, sum);
+        accumulate_segment<NV, kTermsInFlightChunks>(terms, beg, end, ids[ci.m] < V, gin_pos, table, d4, stride4, lane, sum, lim);
         double* out = partials + (size_t)x * stride4 * 4;
 #pragma unroll
         for (int i = 0; i < NV; ++i) {
@@ -460,13 +508,17 @@ template <int NV>
 __global__ void __launch_bounds__(kLongWarps * 32)
 k_reduce_long(const uint32_t* __restrict__ ids, const double* __restrict__ partials, float4* __restrict__ table,
               float4* __restrict__ delta, uint32_t V, uint32_t d4, uint32_t stride4, double scale,
-              const uint32_t* __restrict__ long_counters, const LongRow* __restrict__ long_rows, uint32_t warps) {
+              const uint32_t* __restrict__ long_counters, const LongRow* __restrict__ long_rows, uint32_t warps, Limits lim) {
     extern __shared__ __align__(16) double runs[];   // [warps][4 * d4]
     const uint32_t lane = threadIdx.x & 31, wid = threadIdx.x >> 5;
     const uint32_t n_long = long_counters[0];
+    if (!in_bounds(lim, n_long, (uint64_t)lim.long_rows + 1)) return;
     for (uint32_t x = blockIdx.x; x < n_long; x += gridDim.x) {
         const LongRow row = long_rows[x];
+        // block-uniform: every thread sees the same row record
+        if (!in_bounds(lim, row.m, lim.batch_rows) || !in_bounds(lim, (uint64_t)row.base + row.nchunks, (uint64_t)lim.chunks + 1)) continue;
         const uint32_t id = ids[row.m];
+        if (!in_bounds(lim, id, lim.table_rows) || !in_bounds(lim, row.m, lim.slot_rows)) continue;
         const uint32_t per = (row.nchunks + warps - 1) / warps;
         const uint32_t c_beg = wid * per < row.nchunks ? wid * per : row.nchunks;
         const uint32_t c_end = c_beg + per < row.nchunks ? c_beg + per : row.nchunks;
@@ -532,7 +584,7 @@ static cudaError_t reduce_short(const Launcher& L, const Rec* terms, const MsgHe
     Timed timed(L, K_REDUCE_ROWS);
     k_reduce_rows<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, out_smem, L.stream>>>(
         terms, hdr, ids, seg_start, gin_pos, reinterpret_cast<float4*>(table), reinterpret_cast<float4*>(delta), s.V, s.d4,
-        stride4, scale);
+        stride4, scale, L.lim);
     return cudaGetLastError();
 }
 
@@ -547,7 +599,7 @@ static cudaError_t reduce_listed(const Launcher& L, const Rec* terms, const uint
     {
         Timed timed(L, K_REDUCE_CHUNKS);
         k_reduce_chunks<NV><<<L.sms * grid_shape().reduce_blocks_per_sm, kReduceThreads, 0, L.stream>>>(
-            terms, ids, seg_start, gin_pos, t4, s.V, s.d4, stride4, long_counters, chunk_items, partials);
+            terms, ids, seg_start, gin_pos, t4, s.V, s.d4, stride4, long_counters, chunk_items, partials, L.lim);
     }
     {
         Timed timed(L, K_REDUCE_LONG);
@@ -555,7 +607,7 @@ static cudaError_t reduce_listed(const Launcher& L, const Rec* terms, const uint
         if (long_warps > (uint32_t)kLongWarps) long_warps = kLongWarps;
         if (long_warps < 1) long_warps = 1;
         k_reduce_long<NV><<<L.sms * 2, long_warps * 32, (size_t)long_warps * s.d * 8, L.stream>>>(
-            ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters, long_rows, long_warps);
+            ids, partials, t4, d4p, s.V, s.d4, stride4, scale, long_counters, long_rows, long_warps, L.lim);
     }
     return cudaGetLastError();
 }

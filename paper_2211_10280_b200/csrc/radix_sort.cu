@@ -1,7 +1,8 @@
 // Stable least-significant-digit radix sort of 64-bit items by (a bit range of) their 32-bit keys.
 //
 // Keys are row ids, dense in [0, 2V], so few digit passes are needed.  Every pass is three kernels:
-// per-tile digit histogram, per-digit scan over the tiles (one warp per digit), stable scatter.  Stability
+// per-tile digit histogram, per-digit scan over the tiles (one warp per digit), stable scatter; with few tiles
+// the scan is left out and every scatter block sums the tile counts it needs itself.  Stability
 // (equal keys keep their input order) is what makes the later per-row sums run in a fixed order.
 // The whole working set (two item buffers) stays in L2 at the sizes of interest.
 #include "kernels.h"
@@ -62,9 +63,13 @@ k_scan_digits(uint32_t* __restrict__ hist, uint32_t tiles, uint32_t* __restrict_
 // rounds are ranked by their order, so the rank of an item among equal digits follows input order.
 // At most 64 registers per thread: a block of 256 threads then needs 16 K registers of a multiprocessor, which the
 // forward kernel, beside which the sort runs, leaves free when it sizes its grid.
+// kRawHist: `hist` holds the per-tile counts as the histogram kernel left them (no scan kernel ran): every block adds
+// up, per digit, the tiles before it and all tiles itself - cheaper than a launch when there are few tiles.
+constexpr uint32_t kMaxRawTiles = 128;
+template <bool kRawHist>
 __global__ void __launch_bounds__(kSortThreads, 4)
 k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_t n, uint32_t shift,
-                const uint32_t* __restrict__ hist, uint32_t tiles, const uint32_t* __restrict__ totals) {
+                const uint32_t* __restrict__ hist, uint32_t tiles, const uint32_t* __restrict__ totals, Limits lim) {
     __shared__ uint32_t cnt[kSortWarps][kBins];
     __shared__ uint32_t digit_base[kBins];
     __shared__ uint32_t warp_tot[kSortWarps];
@@ -97,9 +102,22 @@ k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_
         __syncwarp();
     }
     __syncthreads();
+    // this tile's offset inside its digit's run, and the digit's total
+    uint32_t tile_offset, t;
+    if (kRawHist) {
+        tile_offset = 0;
+        t = 0;
+        for (uint32_t x = 0; x < tiles; ++x) {
+            const uint32_t c = hist[threadIdx.x * tiles + x];
+            if (x < blockIdx.x) tile_offset += c;
+            t += c;
+        }
+    } else {
+        tile_offset = hist[threadIdx.x * tiles + blockIdx.x];
+        t = totals[threadIdx.x];
+    }
     // exclusive scan of the digit totals: where each digit's run starts in the output
     {
-        const uint32_t t = totals[threadIdx.x];
         uint32_t incl = t;
 #pragma unroll
         for (int o = 1; o < 32; o <<= 1) {
@@ -115,7 +133,7 @@ k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_
     // per digit: start of the digit, this tile's offset in it, then exclusive prefix over the warps of the block
     {
         const uint32_t digit = threadIdx.x;
-        uint32_t run = digit_base[digit] + hist[digit * tiles + blockIdx.x];
+        uint32_t run = digit_base[digit] + tile_offset;
 #pragma unroll
         for (int w = 0; w < kSortWarps; ++w) {
             const uint32_t c = cnt[w][digit];
@@ -129,7 +147,8 @@ k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_
         const uint32_t idx = wbase + r * 32 + lane;
         if (idx < n) {
             const uint32_t digit = (item_key(item[r]) >> shift) & (kBins - 1);
-            out[cnt[wid][digit] + rank[r]] = item[r];
+            const uint32_t pos = cnt[wid][digit] + rank[r];
+            if (in_bounds(lim, pos, n)) out[pos] = item[r];
         }
     }
 }
@@ -146,13 +165,16 @@ cudaError_t launch_sort(const Launcher& L, item_t* a, item_t* b, uint32_t n, uin
             Timed timed(L, K_SORT_HIST);
             k_radix_hist<<<tiles, kSortThreads, 0, L.stream>>>(src, n, shift, hist, tiles);
         }
-        {
+        if (tiles > kMaxRawTiles) {
             Timed timed(L, K_SORT_SCAN);
             k_scan_digits<<<kBins / kScanWarps, kScanWarps * 32, 0, L.stream>>>(hist, tiles, hist + (size_t)tiles * kBins);
         }
         {
             Timed timed(L, K_SORT_SCATTER);
-            k_radix_scatter<<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles, hist + (size_t)tiles * kBins);
+            if (tiles > kMaxRawTiles)
+                k_radix_scatter<false><<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles, hist + (size_t)tiles * kBins, L.lim);
+            else
+                k_radix_scatter<true><<<tiles, kSortThreads, 0, L.stream>>>(src, dst, n, shift, hist, tiles, hist + (size_t)tiles * kBins, L.lim);
         }
         item_t* t = src; src = dst; dst = t;
     }

@@ -120,8 +120,10 @@ __device__ inline uint32_t alias_pick(const uint2* __restrict__ tab, uint32_t V,
 
 // One thread per (centre position q, window slot s, draw pair jp).  Window slot s in [0, 2w) stands
 // for context position q + (s < w ? s - w : s - w + 1); slots outside the batch do nothing.
-// Thread jp = 0 also emits the positive contribution; thread (s = 0, jp = 0) counts the token and emits the
-// position's two input-row items: the forward kernel leaves one partial centre gradient for the pairs
+// Thread jp = 0 also emits the positive contribution; thread (s = 0, jp = 0) checks the position's token id (when
+// `check` is set: the unrouted path has no separate validation kernel), counts the token (when `count` is set: only
+// batches too short to have pairs are counted here, the others once the whole batch is known to be valid, by the
+// first kernel of the message build) and emits the position's two input-row items: the forward kernel leaves one partial centre gradient for the pairs
 // to the left of the position and one for those to its right (items 2q and 2q + 1; the contributions
 // follow from item 2n on).  In a routed batch (owner != nullptr) the positions of other
 // replicas' centre words emit only items that sort past every row and are never read.
@@ -129,7 +131,7 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
                           uint32_t replica, uint32_t batch_lo, uint32_t key0, uint32_t key1,
                           const uint2* __restrict__ alias_tab, uint32_t* __restrict__ rows,
                           item_t* __restrict__ items, unsigned long long* __restrict__ counts,
-                          const uint32_t* __restrict__ err, const uint8_t* __restrict__ owner) {
+                          uint32_t* __restrict__ err, const uint8_t* __restrict__ owner, int check, int count, Limits lim) {
     if (*err) return;
     const uint32_t JP = (k + 1) / 2;
     const uint64_t t = (uint64_t)blockIdx.x * blockDim.x + threadIdx.x;
@@ -142,8 +144,11 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
     const uint32_t centre = (uint32_t)tok[q];
     const bool own = !owner || owner[q];
     if (s == 0 && jp == 0) {
-        if (own) atomicAdd(counts + centre, 1ULL);
-        if (n >= 2) {
+        // A bad id only raises the flag here: nothing below indexes memory by a token id (row ids are stored, keys are
+        // sorted by their low bits), and every later kernel of the batch sees the flag and leaves.
+        if (check && centre >= V) atomicOr(err, kErrBadToken);
+        if (count && own && centre < V) atomicAdd(counts + centre, 1ULL);
+        if (n >= 2 && in_bounds(lim, 2ull * q + 1, lim.items)) {
             items[2 * q] = make_item(own ? centre : 2 * V, 2 * q);
             items[2 * q + 1] = make_item(own ? centre : 2 * V, 2 * q + 1);
         }
@@ -155,6 +160,7 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
     const uint32_t K1 = k + 1;
     const uint32_t ctx = (uint32_t)tok[c];
     const uint32_t cbase = p * K1;
+    if (!in_bounds(lim, (uint64_t)cbase + K1 - 1, lim.contrib) || !in_bounds(lim, 2ull * n + cbase + K1 - 1, lim.items)) return;
     if (!own) {
         if (jp == 0) items[2 * n + cbase] = make_item(2 * V, cbase);
         const uint32_t j0 = 2 * jp;
@@ -180,13 +186,15 @@ __global__ void k_prepare(const int32_t* __restrict__ tok, uint32_t n, uint32_t 
 
 cudaError_t launch_prepare(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, uint32_t replica,
                            uint32_t batch_lo, uint64_t seed, const uint2* alias_tab, uint32_t* rows,
-                           item_t* items, unsigned long long* counts, const uint32_t* err, const uint8_t* owner) {
+                           item_t* items, unsigned long long* counts, uint32_t* err, const uint8_t* owner, bool check,
+                           bool count) {
     if (n == 0) return cudaSuccess;
     const uint64_t total = (uint64_t)n * 2 * s.w * ((s.k + 1) / 2);
     const uint32_t blocks = (uint32_t)((total + 255) / 256);
     Timed timed(L, K_PREPARE);
     k_prepare<<<blocks, 256, 0, L.stream>>>(tok, n, s.V, s.w, s.k, replica, batch_lo, (uint32_t)seed,
-                                            (uint32_t)(seed >> 32), alias_tab, rows, items, counts, err, owner);
+                                            (uint32_t)(seed >> 32), alias_tab, rows, items, counts, err, owner, check ? 1 : 0,
+                                            count ? 1 : 0, L.lim);
     return cudaGetLastError();
 }
 

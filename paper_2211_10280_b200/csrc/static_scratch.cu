@@ -38,7 +38,7 @@ struct StaticCarve {
 void carve_static(const tensair_config& c, const Carve& cv, StaticCarve& k) {
     uint64_t off = 0;
     auto take = [&off](uint64_t bytes) { const uint64_t at = off; off = round_up(off + bytes, 256); return at; };
-    k.long_counters = take(8);
+    k.long_counters = take(16);
     k.items_a = take((uint64_t)cv.max_items * 8);
     k.items_b = take((uint64_t)cv.max_items * 8);
     k.terms = take((uint64_t)cv.max_items * sizeof(Rec));
@@ -110,11 +110,11 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
     uint32_t* long_counters = reinterpret_cast<uint32_t*>(in_ws(sc.long_counters));
 
     // the array keeps what the previous call left: the list counters must start at zero
-    TENSAIR_CUDA(ctx, cudaMemsetAsync(long_counters, 0, 8, ctx->stream));
+    TENSAIR_CUDA(ctx, cudaMemsetAsync(long_counters, 0, 16, ctx->stream));
     TENSAIR_CUDA(ctx, launch_validate(ctx->L, tokens_dev, n_tokens, c.V, err, nullptr, nullptr, nullptr, ctx->world_W, me, c.seed));
     TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tokens_dev, n_tokens, ctx->shape, me, (uint32_t)batch_index, c.seed,
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows), items_a,
-                                     ctx->at<unsigned long long>(cv.counts), err, nullptr));
+                                     ctx->at<unsigned long long>(cv.counts), err, nullptr, false, true));
     if (n_items) {
         TENSAIR_CUDA(ctx, launch_forward(ctx->L, tokens_dev, n_tokens, ctx->shape, table, ctx->at<uint32_t>(cv.rows),
                                          ctx->at<Rec>(cv.rec), gin_pos, loss_pos, err, nullptr, nullptr));
@@ -125,7 +125,7 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
                                        ctx->slot_ids(slot), reinterpret_cast<uint32_t*>(in_ws(sc.seg_start)),
                                        long_counters, ctx->at<Rec>(cv.rec), terms, err,
                                        reinterpret_cast<LongRow*>(in_ws(sc.long_rows)),
-                                       reinterpret_cast<ChunkItem*>(in_ws(sc.chunk_items))));
+                                       reinterpret_cast<ChunkItem*>(in_ws(sc.chunk_items)), nullptr, 0, nullptr, nullptr));
         TENSAIR_CUDA(ctx, launch_reduce_rows(ctx->L, terms, hdr, ctx->slot_ids(slot),
                                              reinterpret_cast<uint32_t*>(in_ws(sc.seg_start)), gin_pos, table,
                                              ctx->slot_delta(slot), ctx->shape, scale));

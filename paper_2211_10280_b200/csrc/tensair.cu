@@ -48,7 +48,7 @@ void carve(const tensair_config& c, Carve& k) {
     auto take = [&off](uint64_t bytes) { const uint64_t at = off; off = round_up(off + bytes, 256); return at; };
     k.err = take(4);
     k.loss = take(8);
-    k.long_counters = take(8);
+    k.long_counters = take(16);
     k.counts = take((uint64_t)c.V * 8);
     k.alias_tab = take((uint64_t)c.V * 8);
     k.tok = take((uint64_t)c.batch * 4);
@@ -164,10 +164,15 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
     uint8_t* owner = routed ? ctx->at<uint8_t>(cv.owner) : nullptr;
     uint32_t* owned = routed ? ctx->at<uint32_t>(cv.owned) : nullptr;
     uint32_t* n_owned = routed ? ctx->at<uint32_t>(cv.n_owned) : nullptr;
-    TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err, owner, owned, n_owned, ctx->world_W, me, c.seed));
+    // A routed batch needs the owner of every centre word before anything else, and that kernel checks the token ids
+    // as well; otherwise the prepare kernel checks them itself.  A batch with pairs has its tokens counted by the
+    // first kernel of the message build (by then the whole batch is known to be valid), a shorter one here.
+    if (routed || !n_items)
+        TENSAIR_CUDA(ctx, launch_validate(ctx->L, tok_dev, n, c.V, err, owner, owned, n_owned, ctx->world_W, me, c.seed));
     TENSAIR_CUDA(ctx, launch_prepare(ctx->L, tok_dev, n, ctx->shape, routed ? 0u : me, (uint32_t)batch_index, c.seed,
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows),
-                                     ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err, owner));
+                                     ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err, owner,
+                                     !routed && n_items, !n_items));
     if (n_items) {
         // The sort needs only the items written by the prepare kernel and the forward kernel does not
         // touch them: the two run side by side (the sort is latency-bound and leaves the machine idle).
@@ -190,7 +195,8 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                                        ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
                                        ctx->at<uint32_t>(cv.long_counters), ctx->at<Rec>(cv.rec),
                                        ctx->at<Rec>(cv.terms), err, ctx->at<LongRow>(cv.long_rows),
-                                       ctx->at<ChunkItem>(cv.chunk_items)));
+                                       ctx->at<ChunkItem>(cv.chunk_items), tok_dev, n,
+                                       ctx->at<unsigned long long>(cv.counts), owner));
         // The few rows with many contributions, the message's bucket index and the loss are small latency-bound
         // kernels; they touch nothing the short-row kernel writes, so they run beside it on the second stream.
         const bool beside = ctx->side && grid_shape().overlap_long_rows;
@@ -370,6 +376,8 @@ int tensair_init_sharded(const tensair_config* cfg, const tensair_buffers* bufs,
     };
     if (cudaGetDeviceProperties(&prop, cfg->device) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->L = Launcher{ctx->stream, &ctx->launches, prop.multiProcessorCount, &ctx->prof, cfg->device};
+    ctx->L.lim = Limits{reinterpret_cast<uint32_t*>(ctx->scratch + ctx->cv.err), 2 * cfg->V, ctx->cv.slot_rows, ctx->cv.max_rows,
+                        ctx->cv.max_items, ctx->cv.max_contrib, 2 * cfg->batch, ctx->cv.max_long, ctx->cv.max_chunks};
     if (cudaMallocHost((void**)&ctx->stage, sizeof(*ctx->stage)) != cudaSuccess) return bail(TENSAIR_ECUDA);
     ctx->sched = new Schedule(world_W, cfg->max_delay, cfg->seed);
     ctx->buffered.assign(cfg->W, 0);
@@ -822,6 +830,14 @@ const char* tensair_strerror(int code) {
 const char* tensair_last_error(const tensair_ctx* ctx) { return ctx ? ctx->last_error.c_str() : ""; }
 
 int tensair_error_of_flags(uint32_t flags) { return error_of_flags(flags, nullptr); }
+
+int tensair_checked_build(void) {
+#ifdef TENSAIR_BOUNDS
+    return 1;
+#else
+    return 0;
+#endif
+}
 
 int tensair_raise_error_flags(tensair_ctx* ctx, uint32_t flags) {
     if (!ctx) return TENSAIR_EINVAL;

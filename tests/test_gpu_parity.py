@@ -864,3 +864,30 @@ def test_long_parity_runner_on_a_short_drifting_run(torch):
     res = long_parity.run(wl, steps=25, check_every=10)
     assert res["sampler_rebuilds"] == 2 and [c["step"] for c in res["checks"]] == [10, 20, 25]
     assert res["max_rel_err"] <= TOL_200 and res["after_drain"] <= TOL_200
+
+
+def test_checked_build_reports_a_row_id_outside_the_table_and_skips_it(torch):
+    """Only with the checked build loaded (TENSAIR_CHECKED=1): a received message that names a row past the end of
+    the receiver's table (a corrupted transfer) is reported as TENSAIR_EBOUNDS and the row is left out; the rows in
+    range are applied.  (The address the bad id stands for lies inside the tables buffer - in the other local
+    replica's table - so even the normal build, where this test is skipped, would not touch foreign memory.)"""
+    from paper_2211_10280_b200 import binding as B
+
+    if not B.lib().tensair_checked_build():
+        pytest.skip("needs the checked build: TENSAIR_CHECKED=1 with libtensair_checked.so built")
+    V, d = 400, 8
+    g = B.Context(V=V, d=d, window=2, k=3, batch=32, W=2, world_replicas=3, first_replica=0, max_delay=0)
+    before = [[g.tensair_read_embeddings(r, w) for w in (0, 1)] for r in range(2)]
+    ids, delta = g.tensair_message_buffers(2, 0)
+    stride = delta.numel() // ids.numel()
+    ids[:2].copy_(torch.tensor([7, 2 * V + 5], dtype=torch.int32))
+    delta[:2 * stride].fill_(0.25)
+    g.tensair_commit_message(2, 0, 2, 1)
+    assert g.tensair_apply_messages(0, 0) == 1
+    assert g.tensair_sync() == B.EBOUNDS and "outside its array" in g.tensair_last_error()
+    after = [[g.tensair_read_embeddings(r, w) for w in (0, 1)] for r in range(2)]
+    want = before[0][0].copy()
+    want[7] += np.float32(0.25)
+    assert np.array_equal(after[0][0], want) and np.array_equal(after[0][1], before[0][1])
+    assert np.array_equal(after[1][0], before[1][0]) and np.array_equal(after[1][1], before[1][1])
+    assert g.tensair_sync() == B.OK
