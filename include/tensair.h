@@ -219,6 +219,20 @@ TENSAIR_API int tensair_commit_message_on(tensair_ctx* ctx, uint32_t sender, uin
  */
 TENSAIR_API int tensair_shadow_apply(tensair_ctx* ctx, uint32_t receiver, uint64_t step, int drain, uint32_t* n_applied);
 
+/*
+ * Resuming a run in flight (Section 3.3: models are saved and loaded; here the run around them as well).  What a run
+ * consists of: the tables and the message pool (the caller's device buffers: copy them as they are, after
+ * tensair_sync), and what the library keeps - the running unigram counts, the sampler table in use, the messages
+ * buffered under max_grad_buffer > 1 (their count; the rows are in the pool) and the delivery schedule with its
+ * pending deliveries, applied-gradient sets and logs.  tensair_save_state writes the library's part to host memory
+ * (dst NULL: only *bytes, the size needed; TENSAIR_ENOMEM if capacity is short); tensair_load_state puts it into a
+ * context made by tensair_init / tensair_init_sharded with the SAME configuration (TENSAIR_EINVAL otherwise), after
+ * which the caller restores its copies of tables and pool.  The resumed run then computes, bit for bit, what the
+ * uninterrupted run computes.  Both synchronise.
+ */
+TENSAIR_API int tensair_save_state(tensair_ctx* ctx, void* host_dst, uint64_t capacity, uint64_t* bytes);
+TENSAIR_API int tensair_load_state(tensair_ctx* ctx, const void* host_src, uint64_t bytes);
+
 /* Frees host state only; synchronises the stream first. */
 TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
 
@@ -467,6 +481,10 @@ TENSAIR_API int tensair_schedule_on_train(tensair_schedule* s, uint32_t replica,
 TENSAIR_API int tensair_schedule_take_due(tensair_schedule* s, uint32_t receiver, uint64_t step, int drain,
                               uint64_t max_records, tensair_delivery* out, uint64_t* n);
 TENSAIR_API int tensair_schedule_pending(const tensair_schedule* s, uint32_t receiver, uint64_t* n);
+/* The schedule's whole book-keeping as bytes (dst NULL: only *bytes, the size needed) and back; load accepts only what
+ * a schedule of the same W, max_delay and seed saved (TENSAIR_EINVAL otherwise, nothing changed). */
+TENSAIR_API int tensair_schedule_save(const tensair_schedule* s, void* dst, uint64_t capacity, uint64_t* bytes);
+TENSAIR_API int tensair_schedule_load(tensair_schedule* s, const void* src, uint64_t bytes);
 
 #ifdef __cplusplus
 }

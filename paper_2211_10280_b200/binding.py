@@ -119,6 +119,10 @@ SYMBOLS = {
     "tensair_schedule_on_train": (_int, [_vp, _u32, _u64]),
     "tensair_schedule_take_due": (_int, [_vp, _u32, _u64, _int, _u64, _vp, _P(_u64)]),
     "tensair_schedule_pending": (_int, [_vp, _u32, _P(_u64)]),
+    "tensair_schedule_save": (_int, [_vp, _vp, _u64, _P(_u64)]),
+    "tensair_schedule_load": (_int, [_vp, C.c_char_p, _u64]),
+    "tensair_save_state": (_int, [_vp, _vp, _u64, _P(_u64)]),
+    "tensair_load_state": (_int, [_vp, C.c_char_p, _u64]),
 }
 
 _lib = None
@@ -229,6 +233,16 @@ class Schedule:
         n = C.c_uint64(0)
         _check(lib().tensair_schedule_pending(self._h, receiver, C.byref(n)), "tensair_schedule_pending")
         return int(n.value)
+
+    def save(self) -> bytes:
+        n = C.c_uint64(0)
+        _check(lib().tensair_schedule_save(self._h, None, 0, C.byref(n)), "tensair_schedule_save")
+        buf = C.create_string_buffer(n.value)
+        _check(lib().tensair_schedule_save(self._h, buf, n.value, C.byref(n)), "tensair_schedule_save")
+        return buf.raw[:n.value]
+
+    def load(self, blob: bytes) -> int:
+        return int(lib().tensair_schedule_load(self._h, blob, len(blob)))
 
     def __del__(self):
         try:
@@ -384,6 +398,17 @@ class Context:
         n = C.c_uint32(0)
         _check(lib().tensair_shadow_apply(self._h, receiver, step, int(drain), C.byref(n)), "tensair_shadow_apply", self._h)
         return int(n.value)
+
+    def tensair_save_state(self) -> bytes:
+        """The library's part of a run in flight (sampler state, buffered-message counts, delivery schedule)."""
+        n = C.c_uint64(0)
+        _check(lib().tensair_save_state(self._h, None, 0, C.byref(n)), "tensair_save_state", self._h)
+        buf = C.create_string_buffer(n.value)
+        _check(lib().tensair_save_state(self._h, buf, n.value, C.byref(n)), "tensair_save_state", self._h)
+        return buf.raw[:n.value]
+
+    def tensair_load_state(self, blob: bytes):
+        _check(lib().tensair_load_state(self._h, blob, len(blob)), "tensair_load_state", self._h)
 
     def tensair_update_sampler(self):
         _check(lib().tensair_update_sampler(self._h), "tensair_update_sampler", self._h)

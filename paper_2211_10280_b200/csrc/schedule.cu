@@ -97,6 +97,93 @@ std::vector<Due> Schedule::take_due(uint32_t receiver, uint64_t step, bool drain
     return out;
 }
 
+namespace {
+
+struct Writer {
+    std::vector<uint8_t>& out;
+    void u64(uint64_t v) { for (int i = 0; i < 8; ++i) out.push_back((uint8_t)(v >> (8 * i))); }
+    void words(const std::vector<uint64_t>& w) { u64(w.size()); for (uint64_t x : w) u64(x); }
+};
+struct Reader {
+    const uint8_t* p;
+    size_t left;
+    bool ok = true;
+    uint64_t u64() {
+        if (left < 8) { ok = false; return 0; }
+        uint64_t v = 0;
+        for (int i = 0; i < 8; ++i) v |= (uint64_t)p[i] << (8 * i);
+        p += 8; left -= 8;
+        return v;
+    }
+    // a length read from the blob is believed only as far as the bytes that are left can back it
+    uint64_t count(uint64_t bytes_each) {
+        const uint64_t n = u64();
+        if (bytes_each && n > left / bytes_each) { ok = false; return 0; }
+        return n;
+    }
+    void words(std::vector<uint64_t>& w) {
+        const uint64_t n = count(8);
+        w.assign(ok ? n : 0, 0);
+        for (uint64_t& x : w) x = u64();
+    }
+};
+constexpr uint64_t kScheduleMagic = 0x3144454853524941ull;   // "AIRSHED1"
+
+}  // namespace
+
+void Schedule::save(std::vector<uint8_t>& out) const {
+    Writer w{out};
+    w.u64(kScheduleMagic); w.u64(W_); w.u64(D_); w.u64(seed_); w.u64(next_seq_); w.u64(floor_word_);
+    for (const Bits& g : G_) { w.u64(g.first_word); w.words(g.words); }
+    for (const Slot& s : slots_) {
+        w.u64(s.used ? 1 : 0); w.u64(s.step); w.u64(s.outstanding); w.u64(s.seq);
+        w.u64(s.snapshot.first_word); w.words(s.snapshot.words);
+    }
+    for (const std::vector<Pending>& in : inbox_) {
+        w.u64(in.size());
+        for (const Pending& p : in) { w.u64(p.due); w.u64(p.origin); w.u64(p.sender); w.u64(p.slot); }
+    }
+    for (const std::vector<tensair_delivery>& lg : log_) {
+        w.u64(lg.size());
+        for (const tensair_delivery& d : lg) { w.u64(d.origin_step); w.u64(d.sender); w.u64(d.due_step); w.u64(d.applied_at); w.u64(d.staleness); }
+    }
+}
+
+bool Schedule::load(const uint8_t* data, size_t bytes) {
+    Reader r{data, bytes};
+    if (r.u64() != kScheduleMagic || r.u64() != W_ || r.u64() != D_ || r.u64() != seed_ || !r.ok) return false;
+    Schedule t(W_, D_, seed_);
+    t.next_seq_ = r.u64();
+    t.floor_word_ = r.u64();
+    for (Bits& g : t.G_) { g.first_word = r.u64(); r.words(g.words); }
+    for (Slot& s : t.slots_) {
+        s.used = r.u64() != 0; s.step = r.u64(); s.outstanding = (uint32_t)r.u64(); s.seq = r.u64();
+        s.snapshot.first_word = r.u64(); r.words(s.snapshot.words);
+        if (s.outstanding >= W_) r.ok = false;
+    }
+    for (std::vector<Pending>& in : t.inbox_) {
+        const uint64_t n = r.count(32);
+        for (uint64_t i = 0; i < n && r.ok; ++i) {
+            Pending p{r.u64(), r.u64(), 0, 0};
+            p.sender = (uint32_t)r.u64();
+            p.slot = (uint32_t)r.u64();
+            if (p.sender >= W_ || p.slot >= t.slots_.size()) r.ok = false;
+            in.push_back(p);
+        }
+    }
+    for (std::vector<tensair_delivery>& lg : t.log_) {
+        const uint64_t n = r.count(40);
+        for (uint64_t i = 0; i < n && r.ok; ++i) {
+            tensair_delivery d;
+            d.origin_step = r.u64(); d.sender = r.u64(); d.due_step = r.u64(); d.applied_at = r.u64(); d.staleness = r.u64();
+            lg.push_back(d);
+        }
+    }
+    if (!r.ok || r.left != 0) return false;
+    *this = std::move(t);
+    return true;
+}
+
 }  // namespace tensair
 
 using tensair::Schedule;
@@ -146,6 +233,22 @@ int tensair_schedule_take_due(tensair_schedule* s, uint32_t receiver, uint64_t s
         out[i] = tensair_delivery{due[i].origin, due[i].sender, due[i].due, drain ? due[i].due : step, due[i].staleness};
     if (n) *n = due.size();
     return TENSAIR_OK;
+}
+
+int tensair_schedule_save(const tensair_schedule* s, void* dst, uint64_t capacity, uint64_t* bytes) {
+    if (!s || !bytes) return TENSAIR_EINVAL;
+    std::vector<uint8_t> blob;
+    s->impl.save(blob);
+    *bytes = blob.size();
+    if (!dst) return TENSAIR_OK;                    // size query
+    if (capacity < blob.size()) return TENSAIR_ENOMEM;
+    std::copy(blob.begin(), blob.end(), static_cast<uint8_t*>(dst));
+    return TENSAIR_OK;
+}
+
+int tensair_schedule_load(tensair_schedule* s, const void* src, uint64_t bytes) {
+    if (!s || !src) return TENSAIR_EINVAL;
+    return s->impl.load(static_cast<const uint8_t*>(src), bytes) ? TENSAIR_OK : TENSAIR_EINVAL;
 }
 
 int tensair_schedule_pending(const tensair_schedule* s, uint32_t receiver, uint64_t* n) {

@@ -35,6 +35,10 @@ public:
     bool slot_busy(uint32_t slot) const { return slots_[slot].used && slots_[slot].outstanding; }
     bool slot_holds(uint32_t slot, uint64_t step) const { return slots_[slot].used && slots_[slot].step == step; }
     uint32_t W() const { return W_; }
+    // The whole book-keeping (pending deliveries, slots, applied-gradient sets, delivery logs) as bytes, and back.
+    // load() accepts only what a schedule of the same W, max_delay and seed saved; on failure nothing is changed.
+    void save(std::vector<uint8_t>& out) const;
+    bool load(const uint8_t* data, size_t bytes);
 
 private:
     struct Bits {                      // bit set over gradient sequence numbers >= 64 * first_word

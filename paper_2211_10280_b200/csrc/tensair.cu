@@ -602,6 +602,83 @@ int tensair_shadow_apply(tensair_ctx* ctx, uint32_t receiver, uint64_t step, int
     return TENSAIR_OK;
 }
 
+namespace {
+
+constexpr uint64_t kStateMagic = 0x3154535249415354ull;   // "TSAIRST1"
+
+// The configuration a saved state belongs to, field by field.
+std::vector<uint64_t> state_header(const tensair_ctx* ctx) {
+    const tensair_config& c = ctx->cfg;
+    uint32_t lr_bits;
+    std::memcpy(&lr_bits, &c.lr, 4);
+    return {kStateMagic, c.V, c.d, c.window, c.k, c.batch, c.W, lr_bits, c.max_grad_buffer, c.max_delay, ctx->cv.stride,
+            c.seed, c.reduction, ctx->world_W, ctx->first};
+}
+
+}  // namespace
+
+int tensair_save_state(tensair_ctx* ctx, void* host_dst, uint64_t capacity, uint64_t* bytes) {
+    if (!ctx || !bytes) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const int st = collect(ctx);
+    if (st != TENSAIR_OK) return st;
+    const std::vector<uint64_t> head = state_header(ctx);
+    std::vector<uint8_t> sched;
+    ctx->sched->save(sched);
+    const uint64_t V = ctx->cfg.V;
+    const uint64_t need = head.size() * 8 + 8 + ctx->buffered.size() * 8 + V * 16 + 8 + sched.size();
+    *bytes = need;
+    if (!host_dst) return TENSAIR_OK;
+    if (capacity < need) return TENSAIR_ENOMEM;
+    uint8_t* out = static_cast<uint8_t*>(host_dst);
+    auto put = [&out](uint64_t v) { std::memcpy(out, &v, 8); out += 8; };
+    for (uint64_t v : head) put(v);
+    put(ctx->buffered.size());
+    for (uint32_t b : ctx->buffered) put(b);
+    TENSAIR_CUDA(ctx, cudaMemcpy(out, ctx->at<uint64_t>(ctx->cv.counts), V * 8, cudaMemcpyDeviceToHost));
+    out += V * 8;
+    TENSAIR_CUDA(ctx, cudaMemcpy(out, ctx->at<uint2>(ctx->cv.alias_tab), V * 8, cudaMemcpyDeviceToHost));
+    out += V * 8;
+    put(sched.size());
+    std::memcpy(out, sched.data(), sched.size());
+    return TENSAIR_OK;
+}
+
+int tensair_load_state(tensair_ctx* ctx, const void* host_src, uint64_t bytes) {
+    if (!ctx || !host_src) return TENSAIR_EINVAL;
+    DeviceGuard guard(ctx->cfg.device);
+    if (!guard.ok) return TENSAIR_ECUDA;
+    const std::vector<uint64_t> head = state_header(ctx);
+    const uint64_t V = ctx->cfg.V;
+    const uint64_t fixed = head.size() * 8 + 8 + ctx->buffered.size() * 8 + V * 16 + 8;
+    if (bytes < fixed) return TENSAIR_EINVAL;
+    const uint8_t* in = static_cast<const uint8_t*>(host_src);
+    auto get = [&in]() { uint64_t v; std::memcpy(&v, in, 8); in += 8; return v; };
+    for (uint64_t v : head)
+        if (get() != v) { ctx->last_error = "the saved state belongs to another configuration"; return TENSAIR_EINVAL; }
+    if (get() != ctx->buffered.size()) return TENSAIR_EINVAL;
+    std::vector<uint32_t> buffered(ctx->buffered.size());
+    for (uint32_t& b : buffered) {
+        const uint64_t v = get();
+        if (v >= ctx->cfg.max_grad_buffer) return TENSAIR_EINVAL;
+        b = (uint32_t)v;
+    }
+    const uint8_t* counts = in;
+    const uint8_t* alias = in + V * 8;
+    in += V * 16;
+    const uint64_t sched_bytes = get();
+    if (sched_bytes != bytes - fixed) return TENSAIR_EINVAL;
+    // the schedule checks its own blob and changes nothing unless all of it is sound
+    if (!ctx->sched->load(in, sched_bytes)) { ctx->last_error = "the saved delivery schedule is damaged"; return TENSAIR_EINVAL; }
+    TENSAIR_CUDA(ctx, cudaStreamSynchronize(ctx->stream));
+    TENSAIR_CUDA(ctx, cudaMemcpy(ctx->at<uint64_t>(ctx->cv.counts), counts, V * 8, cudaMemcpyHostToDevice));
+    TENSAIR_CUDA(ctx, cudaMemcpy(ctx->at<uint2>(ctx->cv.alias_tab), alias, V * 8, cudaMemcpyHostToDevice));
+    ctx->buffered = buffered;
+    ctx->have_last = false;
+    return TENSAIR_OK;
+}
+
 int tensair_update_sampler(tensair_ctx* ctx) {
     if (!ctx) return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);

@@ -891,3 +891,58 @@ def test_checked_build_reports_a_row_id_outside_the_table_and_skips_it(torch):
     assert np.array_equal(after[0][0], want) and np.array_equal(after[0][1], before[0][1])
     assert np.array_equal(after[1][0], before[1][0]) and np.array_equal(after[1][1], before[1][1])
     assert g.tensair_sync() == B.OK
+
+
+@pytest.mark.parametrize("m", [1, 2])
+def test_a_run_saved_in_flight_resumes_bit_for_bit(torch, m):
+    """Tables and pool copied by the caller, the library's part by tensair_save_state, in the middle of a step (batches
+    trained, their messages not yet applied, older messages still pending); a fresh context given all three goes on to
+    compute exactly what the uninterrupted run computes - tables, messages, delivery order and staleness."""
+    from paper_2211_10280_b200 import binding as B
+
+    wl = synth.scaled(synth.LARGE_DRIFT, V=6000, d=24, batch=256, W=3, k=5, drift_every=4, stream_seeds=(6, 7, 8),
+                      max_delay=2)
+    steps, cut = 11, 4                              # with m = 2 every replica holds one buffered message at the cut
+    streams = synth.all_streams(wl, steps)
+    kw = dict(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=wl.W, lr=wl.lr, max_delay=wl.max_delay,
+              seed=wl.seed, reduction=wl.reduction, max_grad_buffer=m)
+    a = B.Context(**kw)
+
+    def train(ctx, t):
+        if t and t % wl.drift_every == 0:
+            ctx.tensair_update_sampler()
+        for i in range(wl.W):
+            ctx.tensair_train_batch(i, dev(torch, streams[i][t]), t)
+
+    for t in range(cut):
+        train(a, t)
+        a.tensair_apply_step(t)
+    train(a, cut)                                   # the cut: step `cut` trained, nothing of it applied
+    assert a.tensair_sync() == B.OK
+    blob = a.tensair_save_state()
+    tables = [[a.tensair_read_embeddings(r, w) for w in (0, 1)] for r in range(wl.W)]
+    pool = a.pool.clone()
+    b = B.Context(**kw)
+    b.tensair_load_state(blob)
+    for r in range(wl.W):
+        for w in (0, 1):
+            b.tensair_write_embeddings(r, w, 0, tables[r][w])
+    b.pool.copy_(pool)
+    assert all(np.array_equal(x, y) for x, y in zip(a.tensair_read_sampler(), b.tensair_read_sampler()))
+    for ctx in (a, b):
+        ctx.tensair_apply_step(cut)
+        for t in range(cut + 1, steps):
+            train(ctx, t)
+            ctx.tensair_apply_step(t)
+        ctx.tensair_drain()
+        assert ctx.tensair_sync() == B.OK
+    for r in range(wl.W):
+        la, lb = a.tensair_read_delivery_log(r), b.tensair_read_delivery_log(r)
+        assert np.array_equal(la, lb) and la.shape[0] > 0
+        for w in (0, 1):
+            assert np.array_equal(a.tensair_read_embeddings(r, w).view(np.uint32), b.tensair_read_embeddings(r, w).view(np.uint32))
+    # a state saved under another configuration is refused
+    other = B.Context(**dict(kw, max_delay=1))
+    with pytest.raises(B.TensairError) as e:
+        other.tensair_load_state(blob)
+    assert e.value.code == B.EINVAL

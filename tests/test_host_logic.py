@@ -270,3 +270,35 @@ def test_sharded_job_with_buffered_gradients_is_refused():
     h = C.c_void_p()
     assert B.lib().tensair_init_sharded(C.byref(cfg), C.byref(bufs), None, None, None, 0, 2, C.byref(h)) == B.EINVAL
     assert not h.value
+
+
+def test_schedule_saved_and_loaded_continues_as_if_never_interrupted():
+    W, D, seed = 4, 2, 5
+    a = B.Schedule(W, D, seed)
+    for t in range(70):                       # past the point where fully applied gradients are trimmed from the sets
+        for g in range(W):
+            assert a.on_train(g, t) == B.OK
+        for g in range(W):
+            a.take_due(g, t)
+    for g in range(W):
+        assert a.on_train(g, 70) == B.OK      # saved with the messages of step 70 computed and none of them applied
+    blob = a.save()
+    b = B.Schedule(W, D, seed)
+    assert b.load(blob) == B.OK
+    assert [b.pending(g) for g in range(W)] == [a.pending(g) for g in range(W)] and sum(a.pending(g) for g in range(W)) > 0
+    for t in range(70, 90):
+        if t > 70:
+            for g in range(W):
+                assert a.on_train(g, t) == b.on_train(g, t) == B.OK
+        for g in range(W):
+            assert np.array_equal(a.take_due(g, t), b.take_due(g, t))      # order, due steps and staleness
+    for g in range(W):
+        assert np.array_equal(a.take_due(g, 0, True), b.take_due(g, 0, True))
+    # a schedule of another shape, or damaged bytes, are refused and change nothing
+    assert B.Schedule(W, D + 1, seed).load(blob) == B.EINVAL
+    assert B.Schedule(W, D, seed + 1).load(blob) == B.EINVAL
+    c = B.Schedule(W, D, seed)
+    assert c.load(blob[:-8]) == B.EINVAL and c.load(blob + b"\0" * 8) == B.EINVAL
+    assert c.on_train(0, 0) == B.OK           # the refused loads left it untouched
+    for at in range(48, len(blob) - 8, 8):      # any one field overwritten: refused or accepted, never a crash
+        assert B.Schedule(W, D, seed).load(blob[:at] + b"\xff" * 8 + blob[at + 8:]) in (B.EINVAL, B.OK)
