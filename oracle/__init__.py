@@ -238,6 +238,15 @@ class Oracle:
         lib().orc_read_message(self._h, replica, batch_index, _ptr(ids), _ptr(delta))
         return ids, delta
 
+    def read_message_ids(self, replica, batch_index):
+        """The row ids of a held message without its delta rows, or None."""
+        n = int(lib().orc_read_message(self._h, replica, batch_index, None, None))
+        if n < 0:
+            return None
+        ids = np.empty(n, dtype=np.uint32)
+        lib().orc_read_message(self._h, replica, batch_index, _ptr(ids), None)
+        return ids
+
     def delay(self, step, sender, receiver):
         return int(lib().orc_delay(self._h, step, sender, receiver))
 

@@ -140,6 +140,11 @@ def lib():
             fn = getattr(L, name)
             fn.restype, fn.argtypes = res, args
         _lib = L
+        # launch-shape knobs from the environment: TENSAIR_TUNE="knob=value,knob=value" (see tensair_tune)
+        for item in filter(None, os.environ.get("TENSAIR_TUNE", "").split(",")):
+            name, value = item.split("=")
+            if L.tensair_tune(name.strip().encode(), int(value)) != OK:
+                raise RuntimeError(f"TENSAIR_TUNE: unknown knob or bad value in {item!r}")
     return _lib
 
 

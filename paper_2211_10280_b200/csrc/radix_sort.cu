@@ -65,7 +65,7 @@ k_scan_digits(uint32_t* __restrict__ hist, uint32_t tiles, uint32_t* __restrict_
 // forward kernel, beside which the sort runs, leaves free when it sizes its grid.
 // kRawHist: `hist` holds the per-tile counts as the histogram kernel left them (no scan kernel ran): every block adds
 // up, per digit, the tiles before it and all tiles itself - cheaper than a launch when there are few tiles.
-constexpr uint32_t kMaxRawTiles = 128;
+constexpr uint32_t kMaxRawTiles = 32;   // measured: at 81 tiles the scan kernel is the cheaper way again
 template <bool kRawHist>
 __global__ void __launch_bounds__(kSortThreads, 4)
 k_radix_scatter(const item_t* __restrict__ in, item_t* __restrict__ out, uint32_t n, uint32_t shift,

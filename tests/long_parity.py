@@ -57,7 +57,7 @@ def run(wl: synth.Workload, steps: int, check_every: int, tol: float = 1e-3, rep
             loss_g, info = g.tensair_train_batch(i, dstreams[i][t], t, want_loss=True, want_info=True)
             t_gpu += time.time() - t0
             assert info.n_rows == rows_o, f"step {t} replica {i}: {info.n_rows} message rows, oracle {rows_o}"
-            assert np.array_equal(o.read_message(i, t)[0], g.tensair_read_message_ids(i, t)), \
+            assert np.array_equal(o.read_message_ids(i, t), g.tensair_read_message_ids(i, t)), \
                 f"step {t} replica {i}: message row ids differ"
             if last:
                 assert np.array_equal(o.read_negatives(), g.tensair_read_negatives()), f"step {t}: negatives differ"
@@ -86,7 +86,7 @@ def run(wl: synth.Workload, steps: int, check_every: int, tol: float = 1e-3, rep
         for which in (0, 1):
             errs.append(rel_err(g.tensair_read_embeddings(j, which), o.read_embeddings(j, which)))
     assert max(errs) <= tol, ("after the drain", max(errs), tol)
-    out = {"workload": wl.name, "steps": steps, "replicas": wl.W, "tolerance": tol, "checks": checks,
+    out = {"workload": wl.name, "steps": steps, "replicas": wl.W, "replicas_compared": checked, "tolerance": tol, "checks": checks,
            "max_rel_err": max(c["max_rel_err"] for c in checks), "after_drain": max(errs),
            "sampler_rebuilds": rebuilds, "loss_of_replica_0": {"first": loss_first, "last_oracle": loss_last[0], "last_cuda": loss_last[1]},
            "oracle_seconds": round(t_oracle, 1), "cuda_seconds_with_readbacks": round(t_gpu, 1),
@@ -103,9 +103,12 @@ def main():
     ap.add_argument("--check-every", type=int, default=100)
     ap.add_argument("--tol", type=float, default=1e-3)
     ap.add_argument("--out", default="")
+    ap.add_argument("--check-replicas", default="", help="comma-separated replicas whose tables and logs are compared (default: all)")
     args = ap.parse_args()
     wl = synth.WORKLOADS[args.workload]
-    res = run(wl, args.steps, args.check_every, args.tol, log=lambda m: print(m, file=sys.stderr, flush=True))
+    checked = [int(x) for x in args.check_replicas.split(",")] if args.check_replicas else None
+    res = run(wl, args.steps, args.check_every, args.tol, replicas_checked=checked,
+              log=lambda m: print(m, file=sys.stderr, flush=True))
     line = json.dumps(res)
     print(line)
     if args.out:
