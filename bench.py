@@ -140,11 +140,11 @@ def config_of(wl: synth.Workload, world: int, parallelism: str) -> dict:
             "parallelism": parallelism}
 
 
-def repeats_for(ms_one_region: float) -> int:
-    """How many K-step regions to time so that at least MIN_TIMED_SECONDS are covered."""
-    if ms_one_region <= 0:
+def repeats_for(ms_one_region: float, min_seconds: float = MIN_TIMED_SECONDS) -> int:
+    """How many K-step regions to time so that at least min_seconds are covered."""
+    if ms_one_region <= 0 or min_seconds <= 0:
         return 1
-    return max(1, min(MAX_REPEATS, int(-(-MIN_TIMED_SECONDS * 1e3 // ms_one_region))))
+    return max(1, min(MAX_REPEATS, int(-(-min_seconds * 1e3 // ms_one_region))))
 
 
 def pick_workload(name: str, override: str = "") -> synth.Workload:
@@ -264,7 +264,7 @@ def run_sharded(args):
         ms0, wall0, wall1 = timed(first, host)
         first += K
         regions = [ms0]
-        reps = repeats_for(ms0)
+        reps = repeats_for(ms0, args.min_seconds)
         if world > 1:
             reps = int(max_over_ranks(float(reps), dist, "cuda"))
         for _ in range(reps - 1):
@@ -411,7 +411,7 @@ def run_ours(args):
         ms0, wall0, wall1 = timed(first, host)
         first += K
         regions = [ms0]
-        reps = repeats_for(ms0)
+        reps = repeats_for(ms0, args.min_seconds)
         if world > 1:                                        # every rank must time the same number of regions
             reps = int(max_over_ranks(float(reps), dist, "cuda"))
         for _ in range(reps - 1):
@@ -749,6 +749,8 @@ def main():
     ap.add_argument("--log-applies", default="", help="write one JSON line per apply call (bytes to move) to this file")
     ap.add_argument("--sweep", action="store_true", help="run the 32-point throughput sweep instead (one line per point)")
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--min-seconds", type=float, default=MIN_TIMED_SECONDS,
+                    help="repeat the K-step timed region until this much has been timed (0: time it once; for captures under a profiler)")
     ap.add_argument("--apply-per-replica", action="store_true",
                     help="apply the due messages with one tensair_apply_messages call per replica instead of tensair_apply_step")
     ap.add_argument("--sharded", action="store_true",

@@ -64,10 +64,33 @@ cudaError_t launch_apply_rows(const Launcher& L, const MsgHeader* hdr, const uin
     return cudaGetLastError();
 }
 
-// One thread per bucket boundary: lower bound of b << kBucketShift in the ascending id list.
+// One thread per bucket boundary: lower bound of b << kBucketShift in the ascending id list.  One block more than the
+// boundaries need adds up the batch's loss (the per-half-position losses in a fixed order, in fp64; in a routed
+// batch only the replica's own positions): both are small, independent of each other and wanted at the same point of
+// the batch, so they share a launch.
 __global__ void __launch_bounds__(256)
 k_bucket_index(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ ids, uint32_t* __restrict__ bucket_start,
-               uint32_t n_buckets) {
+               uint32_t n_buckets, const double* __restrict__ loss_pos, uint32_t n_loss, double* __restrict__ loss,
+               const uint32_t* __restrict__ err, const uint8_t* __restrict__ owner) {
+    if (loss && blockIdx.x == gridDim.x - 1) {
+        // the association of the one-block loss kernel (1024 strided partial sums, then a binary tree), so that every
+        // entry point reports the same bits
+        __shared__ double part[1024];
+        for (uint32_t t = threadIdx.x; t < 1024; t += 256) {
+            double s = 0.0;
+            if (!*err)
+                for (uint32_t i = t; i < n_loss; i += 1024)
+                    if (!owner || owner[i >> 1]) s += loss_pos[i];
+            part[t] = s;
+        }
+        __syncthreads();
+        for (uint32_t o = 512; o > 0; o >>= 1) {
+            for (uint32_t t = threadIdx.x; t < o; t += 256) part[t] += part[t + o];
+            __syncthreads();
+        }
+        if (threadIdx.x == 0) *loss = part[0];
+        return;
+    }
     const uint32_t b = blockIdx.x * blockDim.x + threadIdx.x;
     if (b > n_buckets) return;
     const uint32_t n_rows = hdr->n_rows;
@@ -81,10 +104,12 @@ k_bucket_index(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ i
 }
 
 cudaError_t launch_bucket_index(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
-                                uint32_t V) {
+                                uint32_t V, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err,
+                                const uint8_t* owner) {
     const uint32_t nb = bucket_count(V);
     Timed timed(L, K_BUCKET_INDEX);
-    k_bucket_index<<<(nb + 1 + 255) / 256, 256, 0, L.stream>>>(hdr, ids, bucket_start, nb);
+    k_bucket_index<<<(nb + 1 + 255) / 256 + (loss ? 1 : 0), 256, 0, L.stream>>>(hdr, ids, bucket_start, nb, loss_pos,
+                                                                               n < 2 ? 0 : 2 * n, loss, err, owner);
     return cudaGetLastError();
 }
 

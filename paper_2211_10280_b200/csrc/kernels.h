@@ -173,8 +173,11 @@ cudaError_t launch_top_drifted(const Launcher& L, const float* diff, uint32_t n,
 cudaError_t launch_cosine_difference(const Launcher& L, const float* rows, const float* snap, float* out, uint32_t nrows,
                                      const Shape& s);
 // bucket_start[b] = first row of the message with id >= b << kBucketShift, for b in [0, bucket_count(V)].
+// loss != nullptr: the same launch also adds up the batch's loss from the 2n per-half-position losses (see
+// launch_loss_sum, which does that on its own).
 cudaError_t launch_bucket_index(const Launcher& L, const MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
-                                uint32_t V);
+                                uint32_t V, const double* loss_pos = nullptr, uint32_t n = 0, double* loss = nullptr,
+                                const uint32_t* err = nullptr, const uint8_t* owner = nullptr);
 // The index of a message received from another process; also writes the slot's header from the given counts.
 cudaError_t launch_index_received(const Launcher& L, MsgHeader* hdr, const uint32_t* ids, uint32_t* bucket_start,
                                   uint32_t V, uint32_t n_rows, uint32_t n_in_rows);

@@ -126,7 +126,9 @@ k_heads_count(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, u
 __global__ void __launch_bounds__(kHeadThreads)
 k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, const uint32_t* __restrict__ tile_base,
               MsgHeader* __restrict__ hdr, uint32_t* __restrict__ ids, uint32_t* __restrict__ seg_start,
-              const Rec* __restrict__ rec, Rec* __restrict__ terms, const uint32_t* __restrict__ err, Limits lim) {
+              const Rec* __restrict__ rec, Rec* __restrict__ terms, const uint32_t* __restrict__ err,
+              uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows, ChunkItem* __restrict__ chunk_items,
+              Limits lim) {
     if (*err) return;
     // terms[i] = scalar and centre token of the i-th sorted contribution (for an input-row item: the
     // centre position), so that the row sums read their terms contiguously
@@ -157,48 +159,32 @@ k_heads_write(const item_t* __restrict__ sorted, uint32_t n_items, uint32_t V, c
     for (int i = 0; i < kHeadItems; ++i) {
         if ((flags & (1u << i)) && in_bounds(lim, m, (uint64_t)lim.batch_rows + 1)) {
             const uint32_t key = keys[i];
-            seg_start[m] = first + i;
+            const uint32_t start = first + i;
+            seg_start[m] = start;
             if (key < 2 * V) ids[m] = key;
-            else hdr->n_items = first + i;                       // first dropped negative
-            if (key >= V && (first + i == 0 || prev < V)) hdr->n_in_rows = m;   // first output row
+            else hdr->n_items = start;                           // first dropped negative
+            if (key >= V && (start == 0 || prev < V)) hdr->n_in_rows = m;   // first output row
+            // A row with more than kChunk contributions goes on the long-row list, cut into chunks (the order of the
+            // lists does not reach any sum).  Its end is the upper bound of its key among the sorted items; only the
+            // few long rows pay for that search.
+            const uint32_t probe = start + kChunk;
+            if (key < 2 * V && probe < n_items && item_key(sorted[probe]) == key) {
+                uint32_t lo = probe + 1, hi = n_items;
+                while (lo < hi) {
+                    const uint32_t mid = lo + ((hi - lo) >> 1);
+                    if (item_key(sorted[mid]) <= key) lo = mid + 1; else hi = mid;
+                }
+                const uint32_t nch = (lo - start + kChunk - 1) / kChunk;
+                const uint32_t slot = atomicAdd(long_counters, 1u);
+                const uint32_t base = atomicAdd(long_counters + 1, nch);
+                if (in_bounds(lim, slot, lim.long_rows) && in_bounds(lim, (uint64_t)base + nch - 1, lim.chunks)) {
+                    long_rows[slot] = LongRow{m, base, nch};
+                    for (uint32_t ch = 0; ch < nch; ++ch) chunk_items[base + ch] = ChunkItem{m, ch};
+                }
+            }
             ++m;
         }
         prev = keys[i];
-    }
-}
-
-// Lists the rows with more than kChunk contributions and cuts them into chunks (one thread per row finds
-// them, its warp writes the chunk items).  The order of the lists does not reach any sum.
-__global__ void __launch_bounds__(256)
-k_list_long_rows(const MsgHeader* __restrict__ hdr, const uint32_t* __restrict__ seg_start,
-                 uint32_t* __restrict__ long_counters, LongRow* __restrict__ long_rows,
-                 ChunkItem* __restrict__ chunk_items, const uint32_t* __restrict__ err, Limits lim) {
-    if (*err) return;
-    const uint32_t n_rows = hdr->n_rows, lane = threadIdx.x & 31;
-    const uint32_t first = (blockIdx.x * blockDim.x + threadIdx.x) - lane;   // row of lane 0
-    for (uint32_t m0 = first; m0 < n_rows; m0 += gridDim.x * blockDim.x) {
-        const uint32_t m = m0 + lane;
-        uint32_t nch = 0, base = 0;
-        if (m < n_rows) {
-            const uint32_t len = seg_start[m + 1] - seg_start[m];
-            if (len > kChunk) {
-                nch = (len + kChunk - 1) / kChunk;
-                const uint32_t slot = atomicAdd(long_counters, 1u);
-                base = atomicAdd(long_counters + 1, nch);
-                if (in_bounds(lim, slot, lim.long_rows) && in_bounds(lim, (uint64_t)base + nch - 1, lim.chunks))
-                    long_rows[slot] = LongRow{m, base, nch};
-                else
-                    nch = 0;
-            }
-        }
-        uint32_t todo = __ballot_sync(0xFFFFFFFFu, nch != 0);
-        while (todo) {
-            const int src = __ffs(todo) - 1;
-            todo &= todo - 1;
-            const uint32_t row = m0 + src;
-            const uint32_t n = __shfl_sync(0xFFFFFFFFu, nch, src), b = __shfl_sync(0xFFFFFFFFu, base, src);
-            for (uint32_t c = lane; c < n; c += 32) chunk_items[b + c] = ChunkItem{row, c};
-        }
     }
 }
 
@@ -215,11 +201,8 @@ cudaError_t launch_heads(const Launcher& L, const item_t* sorted, uint32_t n_ite
     }
     if (tiles) {
         Timed timed(L, K_HEADS_WRITE);
-        k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, rec, terms, err, L.lim);
-    }
-    if (tiles) {
-        Timed timed(L, K_HEADS_LONG);
-        k_list_long_rows<<<L.sms * 4, 256, 0, L.stream>>>(hdr, seg_start, long_counters, long_rows, chunk_items, err, L.lim);
+        k_heads_write<<<tiles, kHeadThreads, 0, L.stream>>>(sorted, n_items, V, tile_counts, hdr, ids, seg_start, rec, terms, err,
+                                                            long_counters, long_rows, chunk_items, L.lim);
     }
     return cudaGetLastError();
 }

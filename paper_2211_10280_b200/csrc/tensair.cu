@@ -209,8 +209,8 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                                                   ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot), ctx->shape, scale,
                                                   ctx->at<uint32_t>(cv.long_counters), ctx->at<LongRow>(cv.long_rows),
                                                   ctx->at<ChunkItem>(cv.chunk_items), ctx->at<double>(cv.partials)));
-        TENSAIR_CUDA(ctx, launch_bucket_index(L2, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V));
-        TENSAIR_CUDA(ctx, launch_loss_sum(L2, ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err, owner));
+        TENSAIR_CUDA(ctx, launch_bucket_index(L2, hdr, ctx->slot_ids(slot), ctx->slot_buckets(slot), c.V,
+                                              ctx->at<double>(cv.loss_pos), n, ctx->at<double>(cv.loss), err, owner));
         TENSAIR_CUDA(ctx, launch_reduce_rows(ctx->L, ctx->at<Rec>(cv.terms), hdr, ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
                                              ctx->at<double>(cv.gin_pos), table, ctx->slot_delta(slot), ctx->shape, scale));
         if (beside) {
