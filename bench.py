@@ -44,7 +44,7 @@ FALLBACK_HBM_GBS = 6650.0
 # of their messages, so traffic grows in proportion to the algorithmic bytes of a launch.  Only valid for the
 # source file the capture ran (checked by its SHA-256), null otherwise.
 NCU_TRAFFIC = {"apply_step": {"traffic_per_algorithmic_byte": 1.026, "source": "paper_2211_10280_b200/csrc/apply.cu",
-                              "sha256": "0fbd0c9d1aa90b2ff98518c7af8f160f2efc609bc9c97a02da3bcbe088d29569",
+                              "sha256": "70cf5670dd3f12c83ff5bd2911bfa1de26036855059592189bafebb3ef2398b9",
                               "profile": "profiles/k_apply_step_small_case_V250k_W4.md"}}
 
 
@@ -128,8 +128,19 @@ MIN_TIMED_SECONDS = 2.0     # a K-step region is repeated until this much has be
 MAX_REPEATS = 40
 
 
+def placement(wl: synth.Workload, world: int, sharded: bool) -> str:
+    """How the workload's replicas are placed on the GPUs of the run this line stands for (the same words in both arms)."""
+    if world == 1:
+        return f"all {wl.W} replicas on one GPU"
+    if sharded:
+        return (f"{wl.W // world} of {wl.W} replicas per GPU, every message broadcast into every GPU's pool "
+                f"on a communication stream")
+    return f"{world} independent copies of the one-GPU job, no exchange between them"
+
+
 def config_of(wl: synth.Workload, world: int, parallelism: str) -> dict:
-    """The `config` object of the JSON line: the same keys, from the workload alone, in both arms."""
+    """The `config` object of the JSON line: the same keys and values, from the workload and the placement alone, in
+    both arms."""
     stride = -(-wl.d // 8) * 8
     return {"workload": wl.name, "V": wl.V, "d": wl.d, "window": wl.window, "k": wl.k, "batch": wl.batch,
             "replicas": wl.W, "max_delay": wl.max_delay, "reduction": "mean" if wl.reduction else "sum",
@@ -293,13 +304,11 @@ def run_sharded(args):
     if ctx.tensair_sync() != B.OK:
         raise SystemExit("the device reported an error during the benchmark: " + ctx.tensair_last_error())
     P = wl.pairs_per_batch
-    placement = (f"{Wl} of {wl.W} replicas per GPU, every message broadcast into every GPU's pool on a communication stream"
-                 if world > 1 else f"all {wl.W} replicas on one GPU (sharded code path, nothing to exchange)")
     out = {
         "metric": METRIC, "value": wl.W * P * K / (ms_dev * 1e-3), "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": scaling, "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": config_of(wl, world, placement),
+        "config": config_of(wl, world, placement(wl, world, True)),
         "timing": {"regions": len(regions_dev), "steps_per_region": K, "reported": "median region",
                    "ms_per_step_min": round(min(regions_dev) / K, 5), "ms_per_step_max": round(max(regions_dev) / K, 5),
                    "timed_seconds": round(sum(regions_dev) / 1e3, 3)},
@@ -578,7 +587,7 @@ def run_ours(args):
         "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K, "warmup": Wm,
         "ms_per_step": ms_dev / K, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": config_of(wl, world, f"{world} independent replica group{'s' if world > 1 else ''}, no exchange between them"),
+        "config": config_of(wl, world, placement(wl, world, False)),
         "timing": {"regions": len(regions_dev), "steps_per_region": K, "reported": "median region",
                    "ms_per_step_min": round(min(regions_dev) / K, 5), "ms_per_step_max": round(max(regions_dev) / K, 5),
                    "timed_seconds": round(sum(regions_dev) / 1e3, 3)},
@@ -668,7 +677,7 @@ def run_reference(args):
         "impl": "reference", "metric": METRIC, "value": value, "unit": UNIT, "n_gpus": world, "steps": K,
         "warmup": Wm, "ms_per_step": dt / K * 1e3, "higher_is_better": True, "scaling": "weak", "vs_baseline": None,
         "dtype": "f64", "data": "synthetic",
-        "config": config_of(wl, world, "CPU oracle on rank 0's host cores, all replicas in one process"),
+        "config": config_of(wl, world, placement(wl, world, not args.replicas_only)),
         "cpu_baseline": {"value": value, "unit": UNIT, "cores": oracle.threads(), "kind": "oracle", "sample": sample},
         "e2e": {"value": value, "unit": UNIT, "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
     }))
