@@ -9,7 +9,8 @@ applies the messages that are due.  The default workload is the V = 1M, d = 300,
 
 One JSON line is printed by rank 0.  `value` is measured with the batches already in device memory;
 `e2e` is the same metric through tensair_train_batch_host with the batches in pinned host memory and
-every replica's loss copied back (tensair_read_loss_async) and read after the step's one synchronisation.
+every replica's loss copied back every step (tensair_read_loss_async) and read on the host one step later, behind an
+event, so that the GPU does not wait for the host; the error word is read once per timed region.
 `roofline` describes the kernel with the largest share of device time, timed with CUDA events inside the library in a separate pass.  `cpu_baseline`
 is the CPU oracle timed on a bounded sample of the same workload on this host's cores.
 
@@ -358,7 +359,9 @@ def run_ours(args):
                     max_grad_buffer=wl.max_grad_buffer)
     toks_dev = torch.from_numpy(toks_np).cuda()
     toks_pin = torch.from_numpy(toks_np).pin_memory()
-    losses_pin = torch.zeros(wl.W, dtype=torch.float64).pin_memory()
+    losses_pin = torch.zeros((2, wl.W), dtype=torch.float64).pin_memory()      # two steps' losses: one landing, one being read
+    loss_events = [torch.cuda.Event(), torch.cuda.Event()]
+    pending_loss = [None]
     step_losses = []
     n_rows = {}
 
@@ -376,7 +379,7 @@ def run_ours(args):
             elif host:
                 # the loss of every replica travels back asynchronously; the step ends with one synchronisation
                 _, inf = ctx.tensair_train_batch_host(i, toks_pin[b, i], t)
-                ctx.tensair_read_loss_async(losses_pin.data_ptr() + 8 * i)
+                ctx.tensair_read_loss_async(losses_pin.data_ptr() + 8 * (wl.W * (t & 1) + i))
             else:
                 _, inf = ctx.tensair_train_batch(i, toks_dev[b, i], t, want_info=info)
             if inf is not None:
@@ -389,9 +392,14 @@ def run_ours(args):
         else:
             ctx.tensair_apply_step(t)                         # all replicas' due messages in one pass
         if host and not wl.routed:
-            if ctx.tensair_sync() != B.OK:
-                raise SystemExit("the device reported a bad token during the benchmark")
-            step_losses.append(float(losses_pin.sum()))
+            # The losses of step t are read on the host while step t + 1 runs: an event marks the end of the step's
+            # copies, and the host waits for the event of the step before, so the GPU never waits for the host.
+            slot = t & 1
+            loss_events[slot].record(ctx.stream)
+            if pending_loss[0] is not None:
+                loss_events[slot ^ 1].synchronize()
+                step_losses.append(float(losses_pin[slot ^ 1].sum()))
+            pending_loss[0] = slot
 
     def barrier():
         torch.cuda.synchronize()
@@ -409,6 +417,11 @@ def run_ours(args):
         ev1.record()
         barrier()
         wall1 = time.time()
+        if host and pending_loss[0] is not None:             # the last step's losses, and the error word
+            step_losses.append(float(losses_pin[pending_loss[0]].sum()))
+            pending_loss[0] = None
+            if ctx.tensair_sync() != B.OK:
+                raise SystemExit("the device reported an error during the benchmark: " + ctx.tensair_last_error())
         ms = ev0.elapsed_time(ev1)
         if world > 1:
             ms = max_over_ranks(ms, dist, "cuda")
@@ -592,7 +605,7 @@ def run_ours(args):
                    "ms_per_step_min": round(min(regions_dev) / K, 5), "ms_per_step_max": round(max(regions_dev) / K, 5),
                    "timed_seconds": round(sum(regions_dev) / 1e3, 3)},
         "e2e": {"value": e2e_value, "unit": UNIT, "ms_per_step": ms_e2e / K, "regions": len(regions_e2e),
-                "h2d_bytes_per_step": (1 if wl.routed else wl.W) * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4) if wl.routed else wl.W * 8 + 4},
+                "h2d_bytes_per_step": (1 if wl.routed else wl.W) * wl.batch * 4, "d2h_bytes_per_step": wl.W * (8 + 16 + 4) if wl.routed else wl.W * 8},
         "gpu_launches": int(launches),
         "clocks": sampler.summary(wall0, wall1),
         "roofline": roofline,
