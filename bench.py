@@ -227,6 +227,9 @@ def run_sharded(args):
     if wl.routed or wl.max_grad_buffer != 1:
         raise SystemExit("the sharded placement needs an unrouted workload with maxGradBuffer 1")
     wl, Wl, scaling = sharded_workload(wl, world)
+    B.tensair_tune("early_prepare", 2)                    # resident, complete batches (see run_ours)
+    for item in filter(None, args.tune.split(",")):
+        B.tensair_tune(item.split("=")[0], int(item.split("=")[1]))
     K, Wm = args.steps, max(args.warmup, 3)
     nb = stream_batches(wl)
     toks_all, counts = rank_streams(wl, 0, nb)                   # the one-process job's streams; this rank takes its replicas'
@@ -236,6 +239,7 @@ def run_sharded(args):
                     first_replica=rank * Wl)
     grp = ShardedReplicas(ctx, rank, world, Wl, dist if world > 1 else None, count_device="cuda")
     toks_dev = torch.from_numpy(toks_np).cuda()
+    torch.cuda.synchronize()                              # the batches are complete before the first call names them
     toks_pin = torch.from_numpy(toks_np).pin_memory()
     losses_pin = torch.zeros(Wl, dtype=torch.float64).pin_memory()
 
@@ -346,6 +350,9 @@ def run_ours(args):
     if world > 1:
         dist.init_process_group("nccl", device_id=torch.device("cuda", local))
     wl = pick_workload(args.workload, args.override)
+    # the batches are resident in device memory, complete, long before they are trained on: the library may sample and
+    # sort a batch ahead of its turn on the stream
+    B.tensair_tune("early_prepare", 2)
     for item in filter(None, args.tune.split(",")):
         B.tensair_tune(item.split("=")[0], int(item.split("=")[1]))
     K, Wm = args.steps, max(args.warmup, 3)
@@ -358,6 +365,7 @@ def run_ours(args):
                     max_delay=wl.max_delay, seed=wl.seed + rank, counts=counts, device=local, reduction=wl.reduction,
                     max_grad_buffer=wl.max_grad_buffer)
     toks_dev = torch.from_numpy(toks_np).cuda()
+    torch.cuda.synchronize()                              # the batches are complete before the first call names them
     toks_pin = torch.from_numpy(toks_np).pin_memory()
     losses_pin = torch.zeros((2, wl.W), dtype=torch.float64).pin_memory()      # two steps' losses: one landing, one being read
     loss_events = [torch.cuda.Event(), torch.cuda.Event()]
@@ -705,6 +713,9 @@ def run_sweep(args):
 
     peak, peak_kind = hbm_peak()
     steps = min(args.steps, 100)
+    B.tensair_tune("early_prepare", 2)                    # resident, complete batches (see run_ours)
+    for item in filter(None, args.tune.split(",")):
+        B.tensair_tune(item.split("=")[0], int(item.split("=")[1]))
     for wl in synth.SWEEP:
         nb = steps + 6
         stream = synth.token_stream(wl, 0, nb)
@@ -712,6 +723,7 @@ def run_sweep(args):
         ctx = B.Context(V=wl.V, d=wl.d, window=wl.window, k=wl.k, batch=wl.batch, W=1, lr=wl.lr, seed=wl.seed,
                         counts=counts, reduction=wl.reduction)
         toks = torch.from_numpy(stream).cuda()
+        torch.cuda.synchronize()
         rows = []
         for t in range(3):
             _, info = ctx.tensair_train_batch(0, toks[t], t, want_info=True)

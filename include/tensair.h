@@ -18,8 +18,9 @@
  *   - "device pointer" means memory of the GPU named in tensair_config.device; "host pointer" means
  *     ordinary process memory (pinned or pageable).
  *   - All GPU work is enqueued on the stream given at tensair_init, in call order (inside one call the
- *     library may fork part of the work onto an internal stream and join it again before the call's
- *     last kernel; to the caller's stream the call is one ordered piece of work).  Calls are
+ *     library may fork part of the work onto internal streams and join it again before the call's
+ *     last kernel; to the caller's stream the call is one ordered piece of work - what it has done is
+ *     done when the stream has passed the call; part of it may have started earlier).  Calls are
  *     asynchronous unless stated; a context must be used from one thread at a time.
  *   - The library allocates no device memory: tables, message pool and scratch are caller-owned and
  *     must stay valid until tensair_destroy.
@@ -251,7 +252,13 @@ TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
  *              reaches maxGradBuffer) only every m-th batch of a replica sends: the sum of its last m
  *              messages over the union of their rows, each row's deltas added in fp32 in the order they
  *              were computed; tensair_read_message then holds only for those batch indices.
- * tokens_dev   device, int32[n_tokens], borrowed until the stream has passed this call; n_tokens <= batch.
+ * tokens_dev   device, int32[n_tokens], borrowed until the stream has passed this call; n_tokens <= batch.  They are
+ *              read in stream order (whatever the stream holds before this call may still be writing them), unless
+ *              the knob "early_prepare" of tensair_tune is 2: the caller then vouches that tokens_dev is complete
+ *              when the call is made (batches resident in device memory, a copy already waited for), and the
+ *              library samples and sorts the batch on an internal stream ahead of the batch's turn on the caller's
+ *              stream - beside the batches before it or beside the message application.  Results do not depend on
+ *              the knob.
  * batch_index  the global step t of this batch (< 2^32); it selects the random draws and the message slot.
  * loss_out     host, nullable.  Non-NULL: receives the sum of the batch's pair losses and the call synchronises.
  * info         host, nullable.  Non-NULL: filled, and the call synchronises.
@@ -264,8 +271,10 @@ TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
 TENSAIR_API int tensair_train_batch(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_dev, uint32_t n_tokens,
                         uint64_t batch_index, double* loss_out, tensair_msg_info* info);
 
-/* Same step with the batch in HOST memory: copies tokens_host to the device on the stream first
- * (asynchronously if the memory is pinned).  tokens_host must stay valid until the stream passes. */
+/* Same step with the batch in HOST memory: copies tokens_host to the device first (asynchronously if the memory is
+ * pinned).  Host memory is complete when the call is made, so (unless the knob "early_prepare" is 0) the copy, the
+ * sampling and the sort of the batch run on an internal stream ahead of the batch's turn on the caller's stream.
+ * tokens_host must stay valid until the stream passes. */
 TENSAIR_API int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, const int32_t* tokens_host, uint32_t n_tokens,
                              uint64_t batch_index, double* loss_out, tensair_msg_info* info);
 
@@ -433,7 +442,10 @@ TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
  * "fused_blocks_per_sm" = blocks per multiprocessor of that pass, "overlap_sort" = 0 keeps the sort of a batch on the caller's stream instead of an internal second stream,
  * "overlap_long_rows" = 0 keeps the sums of the rows with many contributions, the message's bucket index and the
  * loss sum on the caller's stream instead of beside the short-row sums on the second stream,
- * "device_alias_build" = 0 makes tensair_update_sampler build the table on the host. */
+ * "device_alias_build" = 0 makes tensair_update_sampler build the table on the host,
+ * "early_prepare" = 0 / 1 / 2: a batch's sampling and sort run ahead of its turn on an internal third stream never /
+ * when its tokens come from host memory (default) / also for device tokens, which the caller then vouches are complete
+ * when the call is made. */
 TENSAIR_API int tensair_tune(const char* name, int value);
 TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);
 

@@ -17,6 +17,8 @@ inline uint64_t round_up(uint64_t x, uint64_t a) { return (x + a - 1) / a * a; }
 struct Carve {
     uint64_t err, loss, long_counters, counts, alias_tab, tok, rows, items_a, items_b, rec, terms, gin_pos, loss_pos, hist,
         tile_counts, seg_start, long_rows, chunk_items, partials, merge_counts, topk, owner, owned, n_owned, alias_state, alias_work, total;
+    // buffer sets of the batches prepared ahead of their turn (tokens, row ids, sort buffers, histograms, error word)
+    uint64_t set_base, set_bytes, set_tok, set_rows, set_items_a, set_items_b, set_hist, set_err;
     uint64_t slot_bytes, bucket_off, ids_off, delta_off;
     uint32_t stride, max_pairs, max_contrib, max_items, max_long, max_chunks;
     uint32_t max_rows;    // most rows the message of ONE batch can have (bounds the per-batch lists)
@@ -41,6 +43,17 @@ struct tensair_ctx {
     cudaEvent_t ev_fork = nullptr, ev_join = nullptr;
     tensair::Launcher L_side;
     tensair::Launcher L;
+    // Third stream: the sampling and the sort of a batch need only its tokens and the sampler table, so they run here,
+    // ahead of the batch's turn on the caller's stream (beside the previous batches' kernels or the message application).
+    static constexpr int kPrepSets = 4;
+    cudaStream_t prep = nullptr;
+    tensair::Launcher L_prep;
+    cudaEvent_t ev_call = nullptr, ev_sampler = nullptr;
+    cudaEvent_t ev_prepared[kPrepSets] = {}, ev_sorted[kPrepSets] = {}, ev_set_free[kPrepSets] = {};
+    bool set_used[kPrepSets] = {};
+    bool sampler_rebuilt = false;    // ev_sampler has been recorded at least once
+    int next_set = 0, last_prepared = -1;
+    const uint32_t* last_rows = nullptr;   // row ids of the most recent batch (parity tap)
     uint64_t launches = 0;
     tensair::Profiler prof;
     float* tables;
@@ -59,6 +72,9 @@ struct tensair_ctx {
     struct Staging { tensair::MsgHeader hdr; double loss; uint32_t err; } *stage = nullptr;
 
     template <class T> T* at(uint64_t off) const { return reinterpret_cast<T*>(scratch + off); }
+    template <class T> T* in_set(int set, uint64_t off) const {
+        return reinterpret_cast<T*>(scratch + cv.set_base + (uint64_t)set * cv.set_bytes + off);
+    }
     float* table_of(uint32_t replica) const { return tables + (size_t)replica * 2 * cfg.V * cv.stride; }
     uint8_t* slot_ptr(uint32_t slot) const { return pool + (size_t)slot * cv.slot_bytes; }
     tensair::MsgHeader* slot_hdr(uint32_t slot) const { return reinterpret_cast<tensair::MsgHeader*>(slot_ptr(slot)); }

@@ -98,7 +98,14 @@ __global__ void __launch_bounds__(kFwdWarps * 32)
 k_forward(const int32_t* __restrict__ tok, uint32_t n, uint32_t V, uint32_t d, uint32_t stride, uint32_t w,
           uint32_t k, uint32_t chunk_rows, uint32_t warp_stage, const float* __restrict__ table, const uint32_t* __restrict__ rows,
           Rec* __restrict__ rec, double* __restrict__ gin_pos, double* __restrict__ loss_pos, uint32_t* __restrict__ err,
-          const uint32_t* __restrict__ owned, const uint32_t* __restrict__ n_owned, Limits lim) {
+          const uint32_t* __restrict__ owned, const uint32_t* __restrict__ n_owned, const uint32_t* __restrict__ batch_err,
+          Limits lim) {
+    // A batch prepared ahead of its turn raised its own error word (a later batch must not stop an earlier one that is
+    // still at work); this, the batch's first kernel on the caller's stream, hands it on to the sticky word.
+    if (batch_err && *batch_err) {
+        if (blockIdx.x == 0 && threadIdx.x == 0) atomicOr(err, *batch_err);
+        return;
+    }
     if (*err) return;
     extern __shared__ __align__(128) unsigned char smem_raw[];
     const uint32_t lane = threadIdx.x & 31, wib = threadIdx.x >> 5;
@@ -301,7 +308,7 @@ void set_forward_shape(int rows, int blocks_per_sm) {
 
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err,
-                           const uint32_t* owned, const uint32_t* n_owned) {
+                           const uint32_t* owned, const uint32_t* n_owned, const uint32_t* batch_err, bool sort_runs_beside) {
     if (n < 2) return cudaSuccess;
     if (L.device < 0 || L.device >= kMaxDevices) return cudaErrorInvalidDevice;
     const size_t row = (size_t)s.stride * 4;
@@ -348,13 +355,13 @@ cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, co
             attr_set = true;                                                                                        \
         }                                                                                                           \
         uint32_t grid = blocks;                                                                                     \
-        if (g_forward_blocks <= 0 && grid_shape().overlap_sort && room_for >= 1 &&                                  \
+        if (g_forward_blocks <= 0 && grid_shape().overlap_sort && sort_runs_beside && room_for >= 1 &&              \
             grid > (uint32_t)(L.sms * room_for))                                                                    \
             grid = (uint32_t)(L.sms * room_for);                                                                    \
         k_forward<NV, CR, NR, VW><<<grid, kFwdWarps * 32, smem, L.stream>>>(tok, n, s.V, s.d, s.stride, s.w, s.k,   \
                                                                             chunk_rows, warp_stage, table, rows,    \
                                                                             rec, gin_pos, loss_pos, err, owned,     \
-                                                                            n_owned, L.lim);                        \
+                                                                            n_owned, batch_err, L.lim);             \
     } while (0)
     // k = 5 (six rows per pair) is common enough to have whole chunks of its own
 #define TENSAIR_FWD_ROWS(NV, VW)                                                     \

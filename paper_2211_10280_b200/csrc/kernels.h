@@ -50,6 +50,7 @@ constexpr int kMaxDevices = 64;   // per-device launch state (function attribute
 struct GridShape {
     int fuse_apply = 1;              // apply the messages due for a receiver in one pass over its table
     int overlap_sort = 1;            // run the radix sort on a second stream while the forward kernel runs
+    int early_prepare = 1;           // sample and sort a batch on a third stream ahead of its turn: 0 never, 1 when the tokens come from host memory, 2 also for device tokens (the caller vouches that they are complete when the call is made)
     int overlap_long_rows = 1;       // sum the long rows (and index the message, sum the loss) on it while the short rows are summed
     int device_alias_build = 1;      // rebuild the sampler's alias table on the device (0: on the host, with a synchronisation)
     int reduce_blocks_per_sm = 64;
@@ -108,7 +109,8 @@ uint32_t sort_hist_words(uint32_t n);
 // forward.cu
 cudaError_t launch_forward(const Launcher& L, const int32_t* tok, uint32_t n, const Shape& s, const float* table,
                            const uint32_t* rows, Rec* rec, double* gin_pos, double* loss_pos, uint32_t* err,
-                           const uint32_t* owned, const uint32_t* n_owned);
+                           const uint32_t* owned, const uint32_t* n_owned, const uint32_t* batch_err = nullptr,
+                           bool sort_runs_beside = true);
 void set_forward_shape(int rows, int blocks_per_sm);
 cudaError_t launch_loss_sum(const Launcher& L, const double* loss_pos, uint32_t n, double* loss, const uint32_t* err,
                             const uint8_t* owner);

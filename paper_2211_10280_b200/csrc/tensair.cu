@@ -72,6 +72,19 @@ void carve(const tensair_config& c, Carve& k) {
     k.n_owned = take(4);
     k.alias_state = take(sizeof(AliasState));
     k.alias_work = take(alias_work_bytes(c.V));
+    // buffer sets of the batches prepared ahead of their turn: offsets inside a set, then the sets themselves
+    {
+        uint64_t in = 0;
+        auto part = [&in](uint64_t bytes) { const uint64_t at = in; in = round_up(in + bytes, 256); return at; };
+        k.set_err = part(4);
+        k.set_tok = part((uint64_t)c.batch * 4);
+        k.set_rows = part((uint64_t)k.max_contrib * 4);
+        k.set_items_a = part((uint64_t)k.max_items * 8);
+        k.set_items_b = part((uint64_t)k.max_items * 8);
+        k.set_hist = part((uint64_t)sort_hist_words(k.max_items) * 4);
+        k.set_bytes = in;
+    }
+    k.set_base = take((uint64_t)tensair_ctx::kPrepSets * k.set_bytes);
     k.total = off;
     k.bucket_off = kHeaderBytes;
     k.ids_off = round_up(k.bucket_off + (uint64_t)(bucket_count(c.V) + 1) * 4, 256);
@@ -135,8 +148,9 @@ int upload_sampler(tensair_ctx* ctx, const uint64_t* counts_host) {
 
 // routed: the replica trains only the centre positions whose word the hash partitioner gives it (Section 4.3);
 // pair indices, negative draws (replica tag 0) and the mean's denominator stay those of the whole batch.
+// tok_host != nullptr: the batch is in host memory (complete when the call is made) and is copied to the device here.
 int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint32_t n, uint64_t batch_index,
-               double* loss_out, tensair_msg_info* info, bool routed = false) {
+               double* loss_out, tensair_msg_info* info, bool routed = false, const int32_t* tok_host = nullptr) {
     const tensair_config& c = ctx->cfg;
     const Carve& cv = ctx->cv;
     // maxGradBuffer = 1: the batch's message is built in its send slot and filed at once.  Otherwise it is built
@@ -164,6 +178,50 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
     uint8_t* owner = routed ? ctx->at<uint8_t>(cv.owner) : nullptr;
     uint32_t* owned = routed ? ctx->at<uint32_t>(cv.owned) : nullptr;
     uint32_t* n_owned = routed ? ctx->at<uint32_t>(cv.n_owned) : nullptr;
+    // The sampling and the sort of a batch need only its tokens and the sampler table, not the model: with the tokens
+    // known to be complete (host memory, or the caller's word for device memory) they run on a third stream into a
+    // buffer set of their own, ahead of the batch's turn on the caller's stream - beside the kernels of the batches
+    // before it or beside the message application - and the forward kernel then has the machine to itself.
+    const bool early = !routed && n_items && ctx->prep &&
+                       (grid_shape().early_prepare >= 2 || (grid_shape().early_prepare == 1 && tok_host));
+    const uint32_t* rows_of_batch = ctx->at<uint32_t>(cv.rows);
+    item_t* sorted = nullptr;
+    int set = -1;
+    if (early) {
+        set = ctx->next_set;
+        ctx->next_set = (set + 1) % tensair_ctx::kPrepSets;
+        // the set's previous batch must have read its sorted items; the sampler table must be the current one
+        if (ctx->set_used[set]) TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->prep, ctx->ev_set_free[set], 0));
+        if (ctx->sampler_rebuilt) TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->prep, ctx->ev_sampler, 0));
+        uint32_t* batch_err = ctx->in_set<uint32_t>(set, cv.set_err);
+        if (tok_host) {
+            int32_t* staged = ctx->in_set<int32_t>(set, cv.set_tok);
+            TENSAIR_CUDA(ctx, cudaMemcpyAsync(staged, tok_host, (size_t)n * 4, cudaMemcpyHostToDevice, ctx->prep));
+            tok_dev = staged;
+        }
+        TENSAIR_CUDA(ctx, cudaMemsetAsync(batch_err, 0, 4, ctx->prep));
+        uint32_t* rows = ctx->in_set<uint32_t>(set, cv.set_rows);
+        TENSAIR_CUDA(ctx, launch_prepare(ctx->L_prep, tok_dev, n, ctx->shape, me, (uint32_t)batch_index, c.seed,
+                                         ctx->at<uint2>(cv.alias_tab), rows, ctx->in_set<item_t>(set, cv.set_items_a),
+                                         ctx->at<unsigned long long>(cv.counts), batch_err, nullptr, true, false));
+        TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_prepared[set], ctx->prep));
+        TENSAIR_CUDA(ctx, launch_sort(ctx->L_prep, ctx->in_set<item_t>(set, cv.set_items_a), ctx->in_set<item_t>(set, cv.set_items_b),
+                                      n_items, bits_for(2 * c.V), ctx->in_set<uint32_t>(set, cv.set_hist), &sorted));
+        TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_sorted[set], ctx->prep));
+        ctx->last_prepared = set;
+        rows_of_batch = rows;
+        TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_prepared[set], 0));
+        TENSAIR_CUDA(ctx, launch_forward(ctx->L, tok_dev, n, ctx->shape, table, rows, ctx->at<Rec>(cv.rec),
+                                         ctx->at<double>(cv.gin_pos), ctx->at<double>(cv.loss_pos), err, nullptr, nullptr,
+                                         batch_err, false));
+        TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_sorted[set], 0));
+        ctx->set_used[set] = true;
+    } else {
+    if (tok_host) {
+        int32_t* staged = ctx->at<int32_t>(cv.tok);
+        if (n) TENSAIR_CUDA(ctx, cudaMemcpyAsync(staged, tok_host, (size_t)n * 4, cudaMemcpyHostToDevice, ctx->stream));
+        tok_dev = staged;
+    }
     // A routed batch needs the owner of every centre word before anything else, and that kernel checks the token ids
     // as well; otherwise the prepare kernel checks them itself.  A batch with pairs has its tokens counted by the
     // first kernel of the message build (by then the whole batch is known to be valid), a shorter one here.
@@ -173,7 +231,10 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
                                      ctx->at<uint2>(cv.alias_tab), ctx->at<uint32_t>(cv.rows),
                                      ctx->at<item_t>(cv.items_a), ctx->at<unsigned long long>(cv.counts), err, owner,
                                      !routed && n_items, !n_items));
+    }
+    ctx->last_rows = rows_of_batch;
     if (n_items) {
+        if (!early) {
         // The sort needs only the items written by the prepare kernel and the forward kernel does not
         // touch them: the two run side by side (the sort is latency-bound and leaves the machine idle).
         const bool fork = ctx->side && grid_shape().overlap_sort;
@@ -181,7 +242,6 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
             TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_fork, ctx->stream));
             TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->side, ctx->ev_fork, 0));
         }
-        item_t* sorted = nullptr;
         TENSAIR_CUDA(ctx, launch_sort(fork ? ctx->L_side : ctx->L, ctx->at<item_t>(cv.items_a), ctx->at<item_t>(cv.items_b),
                                       n_items, bits_for(2 * c.V), ctx->at<uint32_t>(cv.hist), &sorted));
         TENSAIR_CUDA(ctx, launch_forward(ctx->L, tok_dev, n, ctx->shape, table, ctx->at<uint32_t>(cv.rows),
@@ -191,12 +251,15 @@ int train_impl(tensair_ctx* ctx, uint32_t replica, const int32_t* tok_dev, uint3
             TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_join, ctx->side));
             TENSAIR_CUDA(ctx, cudaStreamWaitEvent(ctx->stream, ctx->ev_join, 0));
         }
+        }
         TENSAIR_CUDA(ctx, launch_heads(ctx->L, sorted, n_items, c.V, ctx->at<uint32_t>(cv.tile_counts), hdr,
                                        ctx->slot_ids(slot), ctx->at<uint32_t>(cv.seg_start),
                                        ctx->at<uint32_t>(cv.long_counters), ctx->at<Rec>(cv.rec),
                                        ctx->at<Rec>(cv.terms), err, ctx->at<LongRow>(cv.long_rows),
                                        ctx->at<ChunkItem>(cv.chunk_items), tok_dev, n,
                                        ctx->at<unsigned long long>(cv.counts), owner));
+        // the set's sorted items are dead once the heads kernels have gathered the terms
+        if (early) TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_set_free[set], ctx->stream));
         // The few rows with many contributions, the message's bucket index and the loss are small latency-bound
         // kernels; they touch nothing the short-row kernel writes, so they run beside it on the second stream.
         const bool beside = ctx->side && grid_shape().overlap_long_rows;
@@ -371,6 +434,14 @@ int tensair_init_sharded(const tensair_config* cfg, const tensair_buffers* bufs,
         if (ctx->ev_fork) cudaEventDestroy(ctx->ev_fork);
         if (ctx->ev_join) cudaEventDestroy(ctx->ev_join);
         if (ctx->side) cudaStreamDestroy(ctx->side);
+        if (ctx->ev_call) cudaEventDestroy(ctx->ev_call);
+        if (ctx->ev_sampler) cudaEventDestroy(ctx->ev_sampler);
+        for (int i = 0; i < tensair_ctx::kPrepSets; ++i) {
+            if (ctx->ev_prepared[i]) cudaEventDestroy(ctx->ev_prepared[i]);
+            if (ctx->ev_sorted[i]) cudaEventDestroy(ctx->ev_sorted[i]);
+            if (ctx->ev_set_free[i]) cudaEventDestroy(ctx->ev_set_free[i]);
+        }
+        if (ctx->prep) cudaStreamDestroy(ctx->prep);
         delete ctx;
         return code;
     };
@@ -391,6 +462,17 @@ int tensair_init_sharded(const tensair_config* cfg, const tensair_buffers* bufs,
         return bail(TENSAIR_ECUDA);
     ctx->L_side = ctx->L;
     ctx->L_side.stream = ctx->side;
+    if (cudaStreamCreateWithPriority(&ctx->prep, cudaStreamNonBlocking, prio_high) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_call, cudaEventDisableTiming) != cudaSuccess ||
+        cudaEventCreateWithFlags(&ctx->ev_sampler, cudaEventDisableTiming) != cudaSuccess)
+        return bail(TENSAIR_ECUDA);
+    for (int i = 0; i < tensair_ctx::kPrepSets; ++i)
+        if (cudaEventCreateWithFlags(&ctx->ev_prepared[i], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_sorted[i], cudaEventDisableTiming) != cudaSuccess ||
+            cudaEventCreateWithFlags(&ctx->ev_set_free[i], cudaEventDisableTiming) != cudaSuccess)
+            return bail(TENSAIR_ECUDA);
+    ctx->L_prep = ctx->L;
+    ctx->L_prep.stream = ctx->prep;
 
     const uint32_t V = cfg->V, stride = ctx->cv.stride;
     const size_t replica_floats = (size_t)2 * V * stride;
@@ -435,6 +517,17 @@ void tensair_destroy(tensair_ctx* ctx) {
         cudaEventDestroy(ctx->ev_join);
         cudaStreamDestroy(ctx->side);
     }
+    if (ctx->prep) {
+        cudaStreamSynchronize(ctx->prep);
+        cudaEventDestroy(ctx->ev_call);
+        cudaEventDestroy(ctx->ev_sampler);
+        for (int i = 0; i < tensair_ctx::kPrepSets; ++i) {
+            cudaEventDestroy(ctx->ev_prepared[i]);
+            cudaEventDestroy(ctx->ev_sorted[i]);
+            cudaEventDestroy(ctx->ev_set_free[i]);
+        }
+        cudaStreamDestroy(ctx->prep);
+    }
     delete ctx->sched;
     delete ctx;
 }
@@ -466,10 +559,7 @@ int tensair_train_batch_host(tensair_ctx* ctx, uint32_t replica, const int32_t* 
         return TENSAIR_EINVAL;
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return TENSAIR_ECUDA;
-    int32_t* tok = ctx->at<int32_t>(ctx->cv.tok);
-    if (n_tokens)
-        TENSAIR_CUDA(ctx, cudaMemcpyAsync(tok, tokens_host, (size_t)n_tokens * 4, cudaMemcpyHostToDevice, ctx->stream));
-    return train_impl(ctx, replica, tok, n_tokens, batch_index, loss_out, info);
+    return train_impl(ctx, replica, nullptr, n_tokens, batch_index, loss_out, info, false, tokens_host);
 }
 
 int tensair_apply_messages(tensair_ctx* ctx, uint32_t replica, uint64_t step, uint32_t* n_applied) {
@@ -684,9 +774,15 @@ int tensair_update_sampler(tensair_ctx* ctx) {
     DeviceGuard guard(ctx->cfg.device);
     if (!guard.ok) return TENSAIR_ECUDA;
     if (grid_shape().device_alias_build) {
+        // Every batch prepared ahead so far has been waited for by the caller's stream (its forward kernel follows its
+        // sampling), so the table may be rewritten here; the batches prepared from now on wait for this event.
         TENSAIR_CUDA(ctx, launch_alias_build(ctx->L, ctx->at<unsigned long long>(ctx->cv.counts), ctx->cfg.V,
                                              ctx->at<AliasState>(ctx->cv.alias_state), ctx->at<uint8_t>(ctx->cv.alias_work),
                                              ctx->at<uint2>(ctx->cv.alias_tab)));
+        if (ctx->prep) {
+            TENSAIR_CUDA(ctx, cudaEventRecord(ctx->ev_sampler, ctx->stream));
+            ctx->sampler_rebuilt = true;
+        }
         return TENSAIR_OK;
     }
     std::vector<uint64_t> counts(ctx->cfg.V);
@@ -772,7 +868,7 @@ int tensair_read_negatives(tensair_ctx* ctx, uint32_t* host_neg, uint32_t* n_pai
     if (host_neg && ctx->last_pairs) {
         const uint32_t k = ctx->cfg.k;
         // rows are stored per pair as [positive, k negatives]
-        TENSAIR_CUDA(ctx, cudaMemcpy2D(host_neg, (size_t)k * 4, ctx->at<uint32_t>(ctx->cv.rows) + 1, (size_t)(k + 1) * 4,
+        TENSAIR_CUDA(ctx, cudaMemcpy2D(host_neg, (size_t)k * 4, (ctx->last_rows ? ctx->last_rows : ctx->at<uint32_t>(ctx->cv.rows)) + 1, (size_t)(k + 1) * 4,
                                        (size_t)k * 4, ctx->last_pairs, cudaMemcpyDeviceToHost));
     }
     return TENSAIR_OK;
@@ -848,6 +944,7 @@ int tensair_tune(const char* name, int value) {
     else if (!std::strcmp(name, "fused_blocks_per_sm") && value > 0) { grid_shape().fused_blocks_per_sm = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "fuse_apply")) { grid_shape().fuse_apply = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "overlap_sort")) { grid_shape().overlap_sort = value; return TENSAIR_OK; }
+    else if (!std::strcmp(name, "early_prepare") && value >= 0 && value <= 2) { grid_shape().early_prepare = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "overlap_long_rows")) { grid_shape().overlap_long_rows = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "device_alias_build")) { grid_shape().device_alias_build = value; return TENSAIR_OK; }
     else if (!std::strcmp(name, "reduce_blocks_per_sm") && value > 0) { grid_shape().reduce_blocks_per_sm = value; return TENSAIR_OK; }

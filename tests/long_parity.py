@@ -37,6 +37,7 @@ def run(wl: synth.Workload, steps: int, check_every: int, tol: float = 1e-3, rep
     counts = None if wl.drift_every else synth.stream_counts(synth.all_streams(wl), wl.V)
     o, g = make_pair(wl, counts=counts)
     dstreams = [torch.from_numpy(np.ascontiguousarray(s, dtype=np.int32)).cuda() for s in streams]
+    torch.cuda.synchronize()
     checked = list(range(wl.W)) if replicas_checked is None else list(replicas_checked)
     checks, t_oracle, t_gpu, loss_first, loss_last = [], 0.0, 0.0, None, None
     rebuilds = 0

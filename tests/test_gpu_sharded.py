@@ -27,7 +27,11 @@ def torch():
 
 
 def dev(torch, a):
-    return torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+    """The batch in device memory, complete when this returns (so that the suite can also run with the knob that lets
+    the library start on a batch's tokens ahead of the stream: TENSAIR_TUNE=early_prepare=2)."""
+    t = torch.from_numpy(np.ascontiguousarray(a, dtype=np.int32)).cuda()
+    torch.cuda.current_stream().synchronize()
+    return t
 
 
 def shard_contexts(wl, counts, world, local):

@@ -43,6 +43,7 @@ def test_static_scratch_entry_point_matches_train_batch_on_two_calls_in_a_row():
                  seed=wl.seed, counts=counts, init_in=t_in, init_out=t_out, reduction=wl.reduction)
     for b in range(2):
         toks = torch.from_numpy(stream[b]).cuda()
+        torch.cuda.synchronize()
         loss_ref, info_ref = ref.tensair_train_batch(0, toks, b, want_loss=True, want_info=True)
         torch.cuda.synchronize()
         free_before = torch.cuda.mem_get_info()[0]
