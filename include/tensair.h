@@ -256,9 +256,9 @@ TENSAIR_API void tensair_destroy(tensair_ctx* ctx);
  *              read in stream order (whatever the stream holds before this call may still be writing them), unless
  *              the knob "early_prepare" of tensair_tune is 2: the caller then vouches that tokens_dev is complete
  *              when the call is made (batches resident in device memory, a copy already waited for), and the
- *              library samples and sorts the batch on an internal stream ahead of the batch's turn on the caller's
- *              stream - beside the batches before it or beside the message application.  Results do not depend on
- *              the knob.
+ *              library samples and sorts a batch (of up to "early_prepare_max_items" sort items) on an internal stream
+ *              ahead of the batch's turn on the caller's stream - beside the batches before it or beside the message
+ *              application.  Results do not depend on the knobs.
  * batch_index  the global step t of this batch (< 2^32); it selects the random draws and the message slot.
  * loss_out     host, nullable.  Non-NULL: receives the sum of the batch's pair losses and the call synchronises.
  * info         host, nullable.  Non-NULL: filled, and the call synchronises.
@@ -445,7 +445,8 @@ TENSAIR_API int tensair_profile(tensair_ctx* ctx, int enable);
  * "device_alias_build" = 0 makes tensair_update_sampler build the table on the host,
  * "early_prepare" = 0 / 1 / 2: a batch's sampling and sort run ahead of its turn on an internal third stream never /
  * when its tokens come from host memory (default) / also for device tokens, which the caller then vouches are complete
- * when the call is made. */
+ * when the call is made; "early_prepare_max_items" = largest batch, in sort items (two per token plus window pairs
+ * times (k+1)), that is prepared ahead (default 2^20: larger batches gain nothing from it). */
 TENSAIR_API int tensair_tune(const char* name, int value);
 TENSAIR_API int tensair_profile_read(tensair_ctx* ctx, uint32_t max_kinds, tensair_kernel_time* out, uint32_t* n_kinds);
 

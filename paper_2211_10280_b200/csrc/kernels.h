@@ -53,6 +53,7 @@ struct GridShape {
     int early_prepare = 1;           // sample and sort a batch on a third stream ahead of its turn: 0 never, 1 when the tokens come from host memory, 2 also for device tokens (the caller vouches that they are complete when the call is made)
     int overlap_long_rows = 1;       // sum the long rows (and index the message, sum the loss) on it while the short rows are summed
     int device_alias_build = 1;      // rebuild the sampler's alias table on the device (0: on the host, with a synchronisation)
+    int early_prepare_max_items = 1 << 20;   // ... for batches of at most this many sort items (larger ones gain nothing from it)
     int reduce_blocks_per_sm = 64;
     int apply_blocks_per_sm = 64;
     int fused_blocks_per_sm = 256;
