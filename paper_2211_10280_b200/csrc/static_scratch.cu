@@ -144,6 +144,7 @@ extern "C" int tensair_train_batch_static(tensair_ctx* ctx, uint32_t replica, co
     ctx->last_n = n_tokens;
     ctx->last_pairs = pairs;
     ctx->have_last = true;
+    ctx->last_rows = ctx->at<uint32_t>(cv.rows);      // where this call left its row ids (parity tap)
     if (loss_out || info) {
         TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->loss, ctx->at<double>(cv.loss), 8, cudaMemcpyDeviceToHost, ctx->stream));
         TENSAIR_CUDA(ctx, cudaMemcpyAsync(&ctx->stage->hdr, hdr, sizeof(MsgHeader), cudaMemcpyDeviceToHost, ctx->stream));

@@ -74,6 +74,18 @@ def test_static_scratch_entry_point_matches_train_batch_on_two_calls_in_a_row():
     assert l_new == pytest.approx(l_ref, rel=1e-12)
     assert np.array_equal(new.tensair_read_message(0, 2)[0], ref.tensair_read_message(0, 2)[0])
     assert rel_err(new.tensair_read_embeddings(0, 1), ref.tensair_read_embeddings(0, 1)) <= TOL
+    # after a batch from host memory (which the library prepares ahead of its turn, in buffers of its own) the entry
+    # point still works in its array and the taps follow the last call
+    for ctx in (ref, new):
+        ctx.tensair_train_batch_host(0, np.ascontiguousarray(stream[1]), 3)
+    toks = torch.from_numpy(stream[0]).cuda()
+    torch.cuda.synchronize()
+    l_ref, _ = ref.tensair_train_batch(0, toks, 4, want_loss=True)
+    l_new, _ = new.tensair_train_batch_static(0, toks, 4, want_loss=True)
+    assert l_new == pytest.approx(l_ref, rel=1e-12)
+    assert np.array_equal(new.tensair_read_negatives(), ref.tensair_read_negatives())
+    for which in (0, 1):
+        assert rel_err(new.tensair_read_embeddings(0, which), ref.tensair_read_embeddings(0, which)) <= TOL
 
 
 def test_static_scratch_entry_point_rejects_what_does_not_fit():
