@@ -8,15 +8,15 @@ namespace tensair {
 
 enum KernelKind {
     K_VALIDATE, K_PREPARE, K_SORT_HIST, K_SORT_SCAN, K_SORT_SCATTER, K_FORWARD, K_LOSS_SUM, K_HEADS_COUNT,
-    K_HEADS_SCAN, K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
-    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_ALIAS_BUILD, K_HEADS_LONG,
+    K_HEADS_WRITE, K_REDUCE_ROWS, K_REDUCE_CHUNKS, K_REDUCE_LONG, K_APPLY_INPUT_ROWS,
+    K_APPLY_MESSAGE, K_INIT_TABLE, K_BUCKET_INDEX, K_APPLY_FUSED, K_COSINE, K_MERGE, K_TOPK, K_ALIAS_BUILD,
     K_APPLY_STEP, K_KINDS
 };
 inline const char* kernel_name(int kind) {
     static const char* const names[K_KINDS] = {
         "validate", "prepare", "sort_hist", "sort_scan", "sort_scatter", "forward", "loss_sum", "heads_count",
-        "heads_scan", "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
-        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted", "alias_build", "heads_long_rows",
+        "heads_write", "reduce_rows", "reduce_chunks", "reduce_long", "apply_input_rows",
+        "apply_message", "init_table", "bucket_index", "apply_fused", "cosine_difference", "merge", "top_drifted", "alias_build",
         "apply_step"};
     return kind >= 0 && kind < K_KINDS ? names[kind] : "?";
 }
