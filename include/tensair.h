@@ -318,8 +318,9 @@ TENSAIR_API int tensair_route(uint64_t seed, uint32_t W, uint32_t token, uint32_
  *     histograms): e.g. V = 20,000, d = 64, window 5, k = 5, batch 1,024 needs 4 MiB; batch 8,192 at
  *     d = 300, k = 15 needs 180 MiB and is refused.
  *   - The first call on a device looks up the array's device address (once per device, with that device
- *     current, under a lock, so first calls from several threads are safe).  Make that first call before
- *     any stream capture begins.
+ *     current, under a lock, so first calls from several threads are safe); where the driver loads modules
+ *     lazily, it may reserve the array's 32 MiB only then, so the device's free memory can change at that first
+ *     call and at no later one.  Make that first call before any stream capture begins.
  *   - All calls, from all contexts of the process on one GPU, share the one array.  It keeps the last
  *     call's contents; the call clears what it needs to be zero itself.  Two calls that may overlap on
  *     the GPU (contexts on different streams) race on it: serialise them.
